@@ -1,0 +1,186 @@
+/*
+ * trimkv.h -- C ABI of the B200 (sm_100a) decode hot path of global retention-based
+ * KV-cache eviction ("Make Each Token Count", DBTrimKV).
+ *
+ * One handle owns a budgeted, paged KV cache for a fixed batch of independent
+ * sequences.  Per decode step the caller appends the new token's K/V (with its
+ * retention, produced by the library's gate kernel or supplied), runs attention over
+ * the ragged per-(layer, KV-head) pools, and calls score_and_evict, which re-scores
+ * every cached entry, keeps the budget's worth of best entries across ALL layers and
+ * heads of a sequence and compacts the pools.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory on the current device; "host" pointers
+ *     are ordinary host memory.  All tensors are row-major and contiguous.
+ *   - The caller owns every buffer it passes; the library copies what it keeps and
+ *     holds no caller pointer after the stream work of the call has run.
+ *   - Calls that take `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     only enqueue work.  Argument and state errors are returned at once; errors found
+ *     by kernels (non-finite retention, page pool exhausted, a bounded wait that gave
+ *     up) are latched in a device error word and reported by trimkv_sync_status and
+ *     by the trimkv_get_* calls, which synchronise.
+ *   - No exceptions, no abort, no device trap.  There is no CPU fallback.
+ *   - Every sequence of the batch advances in lock step: each append adds the same
+ *     number of tokens to every sequence.
+ *   - Positions are 1-based token indices i per sequence, as in the paper (C_t = {1..t}).
+ *   - Not thread-safe per handle; handles are independent.
+ */
+#ifndef TRIMKV_H_
+#define TRIMKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TRIMKV_API __attribute__((visibility("default")))
+#else
+#define TRIMKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct trimkv trimkv_t; /* opaque; owns all device memory it allocates */
+
+typedef enum trimkv_status {
+    TRIMKV_OK = 0,
+    TRIMKV_E_ARG = 1,         /* bad argument (NULL, out of range, misaligned)              */
+    TRIMKV_E_STATE = 2,       /* call order violated (e.g. layers hold different token counts) */
+    TRIMKV_E_NOMEM = 3,       /* device allocation failed or page pool exhausted             */
+    TRIMKV_E_CUDA = 4,        /* a CUDA runtime call failed                                   */
+    TRIMKV_E_NONFINITE = 5,   /* NaN retention value met by a kernel                          */
+    TRIMKV_E_TIMEOUT = 6,     /* a bounded device-side wait gave up                           */
+    TRIMKV_E_UNSUPPORTED = 7  /* shape outside what the kernels handle                        */
+} trimkv_status;
+
+#define TRIMKV_DTYPE_BF16 0
+#define TRIMKV_DTYPE_F32 1
+
+typedef struct trimkv_config {
+    int64_t budget_entries; /* M_global per sequence, in entries = tokens' worth x layers x kv_heads
+                               (Sec. 5.2 "global budget of M x #layers x #heads")               */
+    int32_t layers;         /* L                                                               */
+    int32_t kv_heads;       /* H                                                               */
+    int32_t q_heads;        /* Hq, a multiple of H (GQA group g = Hq / H)                      */
+    int32_t head_dim;       /* d, a multiple of 8                                              */
+    int32_t hidden;         /* D, gate input width; 0 = no gate (retention must be supplied)   */
+    int32_t max_batch;      /* B, sequences held by the handle; every call covers all of them  */
+    int32_t page_size;      /* entries per page; must be 64                                    */
+    int32_t gate_hidden;    /* d_g, hidden width of Proj (Sec. 5.1: 512)                       */
+    int32_t gate_embed;     /* d_e, output width of Proj, input of the shared readout          */
+    int32_t horizon;        /* lookahead T - t (Sec. 5.1: 2); 0 = infinite horizon             */
+    int32_t kv_dtype;       /* TRIMKV_DTYPE_BF16 or TRIMKV_DTYPE_F32 (K, V, q and out)         */
+    int32_t max_chunk;      /* largest n_new of one append (1 for pure decode)                 */
+    int32_t reserved;       /* set to 0                                                        */
+    int64_t max_pool_pages; /* cap on pages of one (layer, head) pool; 0 = a pool may take all */
+} trimkv_config;
+
+/* Fill *cfg with defaults (batch 1, q_heads = kv_heads, bf16, no gate, page 64, d_g 512,
+ * d_e 64, horizon 2, max_chunk 512) for the given budget and shape. */
+TRIMKV_API void trimkv_default_config(trimkv_config* cfg, int64_t budget_entries, int layers, int kv_heads, int head_dim);
+
+/* Budgeted cache (Sec. 2.1, Eq. (2): at most M retained entries) with default
+ * configuration.  Returns NULL on failure (see trimkv_last_error). */
+TRIMKV_API trimkv_t* trimkv_create(int64_t budget_entries, int layers, int kv_heads, int head_dim);
+
+/* Same with explicit configuration.  *out receives the handle. */
+TRIMKV_API trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out);
+
+/* Frees everything the handle owns.  NULL is allowed. */
+TRIMKV_API void trimkv_destroy(trimkv_t* h);
+
+/* Empties the cache (all pools, token counters) but keeps gate weights.  Synchronises. */
+TRIMKV_API trimkv_status trimkv_reset(trimkv_t* h);
+
+/* Gate parameters of one layer (Sec. 4.1, Sec. 5.1): Proj_{l,h}(x) = W2[h] act(W1 x + b1) + b2[h],
+ * act = SiLU.  Device pointers, fp32: W1 [d_g, D], b1 [d_g], W2 [H, d_e, d_g], b2 [H, d_e].
+ * Copied; synchronises. */
+TRIMKV_API trimkv_status trimkv_set_gate(trimkv_t* h, int layer, const float* W1, const float* b1, const float* W2,
+                              const float* b2);
+
+/* The readout shared by every layer and head (Sec. 4.1: (w_g, b_g) tied): device w_g [d_e], scalar b_g. */
+TRIMKV_API trimkv_status trimkv_set_shared_projection(trimkv_t* h, const float* w_g, float b_g);
+
+/* Retention gate alone (Sec. 4.1): for x [B, n_new, D] fp32 (device) compute, per row and KV head,
+ *   s = w_g . Proj_{layer,h}(x) + b_g,  beta = sigmoid(s),  lambda = ln beta,
+ *   c = ln sum_{k<horizon} beta^k   (the beta-only factor of Eq. (global_score)).
+ * Any of beta/lambda/c (device, fp32 [B, n_new, H]) may be NULL.  Changes no cache state. */
+TRIMKV_API trimkv_status trimkv_gate(trimkv_t* h, int layer, int n_new, const float* x, float* beta, float* lambda, float* c,
+                          void* stream);
+
+/* Append n_new tokens to every pool of `layer` (a token's retention is estimated once, when it
+ * enters the cache, Sec. 3.2).  k, v: device [B, n_new, H, d] in kv_dtype.
+ * Retention: x != NULL -> gate on x [B, n_new, D] fp32; else lambda [B, n_new, H] fp32 (<= 0) is
+ * required and c [B, n_new, H] is optional (NULL -> derived from lambda on the device in fp32).
+ * Token j of the call gets position tokens(layer) + j + 1.  n_new <= max_chunk. */
+TRIMKV_API trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, const float* lambda, const float* c,
+                            const void* k, const void* v, void* stream);
+
+/* One eviction round at time t = tokens appended so far (Sec. 4.2): for every sequence, score
+ * every entry, S = (t + 1 - i) * lambda + c in fp32 (log of Eq. (global_score)), keep the
+ * budget_entries highest over all layers and heads (ties: older position, then lower layer, then
+ * lower head are kept), drop the rest and compact the pools.  No-op while within budget.
+ * TRIMKV_E_STATE unless every layer holds the same number of tokens. */
+TRIMKV_API trimkv_status trimkv_score_and_evict(trimkv_t* h, void* stream);
+
+/* Decode attention of one layer over the retained entries (Sec. 2.1 / Eq. (1) with r in {0,1}):
+ * q, out: device [B, Hq, d] in kv_dtype; query head j reads the pool of KV head j / g; softmax
+ * scale 1/sqrt(d); an empty pool gives zeros. */
+TRIMKV_API trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const void* q, void* out, void* stream);
+
+/* One whole decode step for all layers at once (the benchmark path): gate on x [L, B, D] fp32
+ * (or lambda [L, B, H] if x == NULL), append k, v [L, B, H, d], attention of q [L, B, Hq, d] into
+ * out [L, B, Hq, d], then score_and_evict. */
+TRIMKV_API trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
+                                     const void* q, void* out, void* stream);
+
+/* Pool lengths to host memory, int32 [B, L, H].  Synchronises; reports latched device errors. */
+TRIMKV_API trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host);
+
+/* Positions kept in pool (seq, layer, head), ascending, to host pos_out[0..cap); *n = pool length
+ * (also when it exceeds cap, in which case TRIMKV_E_ARG is returned).  Synchronises. */
+TRIMKV_API trimkv_status trimkv_get_kept(trimkv_t* h, int seq, int layer, int head, int32_t* pos_out_host, int cap, int* n);
+
+/* Entries of pool (seq, layer, head) in storage order to host arrays (each may be NULL):
+ * pos int32 [n], lambda/c fp32 [n], k/v [n, d] in kv_dtype.  *n as above.  Synchronises. */
+TRIMKV_API trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap, int* n, int32_t* pos_host,
+                              float* lambda_host, float* c_host, void* k_host, void* v_host);
+
+/* Per-sequence figures of the last selection, int64 [B, 4] to host:
+ * {histogram passes used, candidates resolved exactly, entries evicted, bin shift}.  Synchronises. */
+TRIMKV_API trimkv_status trimkv_get_select_stats(trimkv_t* h, int64_t* out_host);
+
+/* Waits for the handle's enqueued work (device synchronise) and returns the latched device error,
+ * TRIMKV_OK if none.  The latch is cleared by trimkv_reset. */
+TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);
+
+/* Per-phase device timing (CUDA events recorded on the call's stream around each phase of append,
+ * decode_attention, decode_step_all and score_and_evict).  trimkv_profile(h, 1) starts recording,
+ * trimkv_profile(h, 0) stops; both synchronise and discard earlier records.  trimkv_profile_read
+ * synchronises, writes to host ms[8] the summed milliseconds and to count[8] the number of recorded
+ * intervals per phase {0 gate, 1 append, 2 attention plan, 3 attention main kernel, 4 attention merge,
+ * 5 score+select, 6 compact, 7 unused}, and clears the records. */
+TRIMKV_API trimkv_status trimkv_profile(trimkv_t* h, int enable);
+TRIMKV_API trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host);
+
+/* Message of the calling thread's last failed call; never NULL. */
+TRIMKV_API const char* trimkv_last_error(void);
+
+/* Number of kernels this library has launched in the calling process so far. */
+TRIMKV_API int64_t trimkv_kernel_launches(void);
+
+/* ---- standalone global selection over a flat score array (Sec. 4.2's ranking alone) ---------
+ * Keeps the k_keep largest of n fp32 scores (device); ties: lower index kept.  keep_bits: device
+ * uint64 [(n + 63) / 64], bit (i % 64) of word i / 64 set iff score i is kept.  workspace: device
+ * scratch of at least trimkv_select_workspace_bytes(n) bytes, 256-byte aligned, contents ignored.
+ * NaN scores are not allowed (latched as TRIMKV_E_NONFINITE in the status word).
+ * status_out: device int32, set to a trimkv_status by the kernels (may be NULL). */
+TRIMKV_API size_t trimkv_select_workspace_bytes(int64_t n);
+TRIMKV_API trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
+                                 size_t workspace_bytes, int32_t* status_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRIMKV_H_ */

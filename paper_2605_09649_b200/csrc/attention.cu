@@ -1,0 +1,536 @@
+// Decode attention over the ragged per-(layer, head) pools (Sec. 2.1 softmax attention restricted to
+// the retained set, Eq. (1) with r in {0,1}; GQA: query head j reads the pool of KV head j / g).
+//
+// bf16, d = 128 path ("split-KV"): the pools of the call are cut into work items of a fixed number of
+// 32-entry tiles.  Each warp is an independent worker: lane 0 streams its tiles' K and V rows from HBM
+// to shared memory with bulk asynchronous copies (cp.async.bulk + mbarrier, 3 stages of 16 KB per warp),
+// the warp computes S^T = K Q^T and O^T += V^T P^T with mma.sync m16n8k16 (the GQA group is the N
+// dimension, so no tensor-core work is spent on padding rows), keeps an online softmax in registers with
+// warp-shuffle reductions over the entries, and writes (m, l, O) partials.  A second kernel merges the
+// partials of each pool.  The kernel is bound by HBM bandwidth: every K/V byte is read once.
+//
+// Any other shape / fp32 uses a plain one-warp-per-query-head kernel.
+#include <algorithm>
+
+#include "trimkv_internal.cuh"
+
+namespace tkv {
+
+namespace {
+
+constexpr int TILE = 32;                       // entries per pipeline stage
+constexpr int ATT_WARPS = 4;
+constexpr int ATT_STAGES = 3;
+constexpr int ROWB = 256;                      // bytes per K or V row (d = 128, bf16)
+constexpr int STAGE_BYTES = 2 * TILE * ROWB;   // K tile + V tile
+constexpr int ATT_SMEM = ATT_WARPS * ATT_STAGES * STAGE_BYTES + 256;
+constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Returns false if the wait gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (unsigned it = 0; it < WAIT_LIMIT; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), .y = hi
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------ work plan
+// Scope = pools of layers [layer0, layer0 + nlayers): scope index si = (lb * B + b) * H + h.
+__device__ __forceinline__ long long scope_pool(const CacheView& cv, int layer0, int si) {
+    const int h = si % cv.H;
+    const int b = (si / cv.H) % cv.B;
+    const int lb = si / (cv.H * cv.B);
+    return ((long long)b * cv.L + layer0 + lb) * cv.H + h;
+}
+
+// One CTA of 1024 threads: items per pool = ceil(ceil(len / TILE) / tpi); exclusive prefix over the scope;
+// item table {scope index, first tile}.
+__global__ void __launch_bounds__(1024)
+attn_plan_kernel(CacheView cv, int layer0, int n_scope, int tpi, int32_t* __restrict__ item_prefix,
+                 int2* __restrict__ item_desc, long long max_items) {
+    __shared__ int wsum[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (n_scope + 1023) / 1024;
+    const int s0 = tid * per, s1 = min(n_scope, s0 + per);
+    int local = 0;
+    for (int si = s0; si < s1; ++si) {
+        const int len = cv.len[scope_pool(cv, layer0, si)];
+        const int tiles = (len + TILE - 1) / TILE;
+        local += (tiles + tpi - 1) / tpi;
+    }
+    int incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    int off = 0, total = 0;
+    for (int w = 0; w < 32; ++w) {
+        if (w < warp) off += wsum[w];
+        total += wsum[w];
+    }
+    int run = off + incl - local;
+    for (int si = s0; si < s1; ++si) {
+        const int len = cv.len[scope_pool(cv, layer0, si)];
+        const int tiles = (len + TILE - 1) / TILE;
+        const int items = (tiles + tpi - 1) / tpi;
+        item_prefix[si] = run;
+        for (int c = 0; c < items; ++c)
+            if (run + c < max_items) item_desc[run + c] = make_int2(si, c * tpi);
+        run += items;
+    }
+    if (tid == 0) {
+        item_prefix[n_scope] = total;
+        if (total > max_items) latch_error(cv.err, TRIMKV_E_NOMEM);
+    }
+}
+
+// ------------------------------------------------------------------ bf16 / d = 128 worker kernel
+struct ItemCtx {
+    int item;        // global item index, -1 = none
+    int si;          // scope index
+    int b;           // sequence
+    int first_tile;  // first tile of the item inside its pool
+    int ntile;       // tiles in the item
+    int len;         // pool length
+    int page_id;     // lane i holds the physical page of the item's i-th page
+};
+
+template <int NT>   // NT = ceil(g / 8): column tiles of 8 query heads
+__global__ void __launch_bounds__(ATT_WARPS * 32, 1)
+attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, const int32_t* __restrict__ item_prefix,
+                const int2* __restrict__ item_desc, const __nv_bfloat16* __restrict__ q, float* __restrict__ part_o,
+                float* __restrict__ part_ml, float scale_log2, long long max_items) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    unsigned char* wbuf = smem_raw + (size_t)warp * ATT_STAGES * STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + (size_t)ATT_WARPS * ATT_STAGES * STAGE_BYTES) + warp * ATT_STAGES;
+
+    // stale shared memory must hold finite values: masked entries still multiply V rows by zero
+    for (int i = lane * 16; i < ATT_STAGES * STAGE_BYTES; i += 32 * 16)
+        *reinterpret_cast<uint4*>(wbuf + i) = make_uint4(0u, 0u, 0u, 0u);
+    if (lane == 0) {
+        for (int s = 0; s < ATT_STAGES; ++s) mbar_init(bars + s, 1);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+
+    const int total_items = min((long long)item_prefix[n_scope], max_items);
+    const int gw = blockIdx.x * ATT_WARPS + warp;
+    const int GW = gridDim.x * ATT_WARPS;
+
+    auto load_item = [&](int item) -> ItemCtx {
+        ItemCtx c;
+        c.item = -1; c.si = 0; c.b = 0; c.first_tile = 0; c.ntile = 0; c.len = 0; c.page_id = 0;
+        if (item >= total_items) return c;
+        const int2 dsc = item_desc[item];
+        c.item = item;
+        c.si = dsc.x;
+        c.first_tile = dsc.y;
+        const long long pool = scope_pool(cv, layer0, c.si);
+        c.b = (c.si / cv.H) % cv.B;
+        c.len = cv.len[pool];
+        const int tiles = (c.len + TILE - 1) / TILE;
+        c.ntile = min(tpi, tiles - c.first_tile);
+        const int npage_item = (c.ntile + 1) / 2;
+        c.page_id = (lane < npage_item) ? cv.block_table[pool * cv.maxpp + c.first_tile / 2 + lane] : 0;
+        return c;
+    };
+
+    ItemCtx prod = load_item(gw), cons = prod;
+    int prod_tile = 0;
+    unsigned issued = 0, consumed = 0;
+    bool failed = false;
+
+    auto issue_one = [&]() {   // issue the producer cursor's tile into stage (issued % STAGES), advance
+        if (prod.item < 0) return;
+        const int tt = prod_tile;
+        const int page = __shfl_sync(0xffffffffu, prod.page_id, tt >> 1);
+        const int half = (prod.first_tile + tt) & 1;
+        if (lane == 0) {
+            const unsigned s = issued % ATT_STAGES;
+            unsigned char* dst = wbuf + (size_t)s * STAGE_BYTES;
+            const char* ksrc = cv.kv + kv_row_offset(cv, prod.b, page, 0, half * TILE);
+            const char* vsrc = cv.kv + kv_row_offset(cv, prod.b, page, 1, half * TILE);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_expect_tx(bars + s, STAGE_BYTES);
+            bulk_g2s(dst, ksrc, TILE * ROWB, bars + s);
+            bulk_g2s(dst + TILE * ROWB, vsrc, TILE * ROWB, bars + s);
+        }
+        ++issued;
+        if (++prod_tile == prod.ntile) {
+            prod = load_item(prod.item + GW);
+            prod_tile = 0;
+        }
+    };
+
+    for (int s = 0; s < ATT_STAGES - 1; ++s) issue_one();
+
+    // per-item state
+    uint32_t bq[NT][8][2];
+    float o[NT][8][4];
+    float m_run[NT][2], l_run[NT][2];
+
+    while (cons.item >= 0 && !failed) {
+        // ---- item prologue: Q fragments (B operand of S^T = K Q^T: k = d, n = query head)
+        const int h = cons.si % cv.H;
+        const int lbb = cons.si / cv.H;   // lb * B + b
+        const __nv_bfloat16* qb = q + ((size_t)lbb * Hq + (size_t)h * g) * 128;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int head = nt * 8 + (lane >> 2);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                uint32_t v0 = 0u, v1 = 0u;
+                if (head < g) {
+                    const __nv_bfloat16* p = qb + (size_t)head * 128 + ks * 16 + 2 * (lane & 3);
+                    v0 = *reinterpret_cast<const uint32_t*>(p);
+                    v1 = *reinterpret_cast<const uint32_t*>(p + 8);
+                }
+                bq[nt][ks][0] = v0;
+                bq[nt][ks][1] = v1;
+            }
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) { o[nt][dt][0] = o[nt][dt][1] = o[nt][dt][2] = o[nt][dt][3] = 0.f; }
+            m_run[nt][0] = m_run[nt][1] = -INFINITY;
+            l_run[nt][0] = l_run[nt][1] = 0.f;
+        }
+
+        for (int tt = 0; tt < cons.ntile; ++tt) {
+            issue_one();    // refill the stage freed by the previous tile
+            const unsigned s = consumed % ATT_STAGES;
+            if (!mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u)) { failed = true; break; }
+            ++consumed;
+            const uint32_t kbase = smem_u32(wbuf + (size_t)s * STAGE_BYTES);
+            const uint32_t vbase = kbase + TILE * ROWB;
+            const int valid = min(TILE, cons.len - (cons.first_tile + tt) * TILE);
+
+            // ---- S^T[entry][head] = K Q^T
+            float sacc[2][NT][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) sacc[mt][nt][0] = sacc[mt][nt][1] = sacc[mt][nt][2] = sacc[mt][nt][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const int row = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                    const int chunk = (2 * ks + (lane >> 4)) ^ (row & 7);
+                    uint32_t a[4];
+                    ldsm_x4(a, kbase + row * ROWB + chunk * 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma_bf16(sacc[mt][nt], a, bq[nt][ks][0], bq[nt][ks][1]);
+                }
+            }
+            // ---- online softmax over the entries (rows); this thread owns heads 2*(lane&3), +1 of each nt
+            uint32_t pb[2][NT][2];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const int r0 = mt * 16 + (lane >> 2);
+                    float* sc = sacc[mt][nt];
+                    sc[0] = (r0 < valid) ? sc[0] * scale_log2 : -INFINITY;
+                    sc[1] = (r0 < valid) ? sc[1] * scale_log2 : -INFINITY;
+                    sc[2] = (r0 + 8 < valid) ? sc[2] * scale_log2 : -INFINITY;
+                    sc[3] = (r0 + 8 < valid) ? sc[3] * scale_log2 : -INFINITY;
+                    mx0 = fmaxf(mx0, fmaxf(sc[0], sc[2]));
+                    mx1 = fmaxf(mx1, fmaxf(sc[1], sc[3]));
+                }
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);
+                const float f0 = exp2f(m_run[nt][0] - mn0), f1 = exp2f(m_run[nt][1] - mn1);   // 0 on the first tile
+                m_run[nt][0] = mn0;
+                m_run[nt][1] = mn1;
+                float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    float* sc = sacc[mt][nt];
+                    const __nv_bfloat162 plo = __floats2bfloat162_rn(exp2f(sc[0] - mn0), exp2f(sc[1] - mn1));
+                    const __nv_bfloat162 phi = __floats2bfloat162_rn(exp2f(sc[2] - mn0), exp2f(sc[3] - mn1));
+                    ls0 += __low2float(plo) + __low2float(phi);     // sum what the tensor cores will see
+                    ls1 += __high2float(plo) + __high2float(phi);
+                    pb[mt][nt][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&plo));
+                    pb[mt][nt][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&phi));
+                }
+                l_run[nt][0] = l_run[nt][0] * f0 + ls0;
+                l_run[nt][1] = l_run[nt][1] * f1 + ls1;
+#pragma unroll
+                for (int dt = 0; dt < 8; ++dt) {
+                    o[nt][dt][0] *= f0; o[nt][dt][1] *= f1; o[nt][dt][2] *= f0; o[nt][dt][3] *= f1;
+                }
+            }
+            // ---- O^T[d][head] += V^T P^T
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const int row = mt * 16 + (lane & 7) + (lane >> 4) * 8;
+                    const int chunk = (2 * dt + ((lane >> 3) & 1)) ^ (row & 7);
+                    uint32_t a[4];
+                    ldsm_x4_trans(a, vbase + row * ROWB + chunk * 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) mma_bf16(o[nt][dt], a, pb[mt][nt][0], pb[mt][nt][1]);
+                }
+            }
+            __syncwarp();   // all lanes are done reading this stage before it is refilled
+        }
+        if (failed) break;
+
+        // ---- item epilogue: partial (m, l, O)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float l0 = l_run[nt][0], l1 = l_run[nt][1];
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+            }
+            const int head0 = nt * 8 + 2 * (lane & 3);
+            if ((lane >> 2) == 0) {
+                if (head0 < g) {
+                    part_ml[((size_t)cons.item * g + head0) * 2 + 0] = m_run[nt][0];
+                    part_ml[((size_t)cons.item * g + head0) * 2 + 1] = l0;
+                }
+                if (head0 + 1 < g) {
+                    part_ml[((size_t)cons.item * g + head0 + 1) * 2 + 0] = m_run[nt][1];
+                    part_ml[((size_t)cons.item * g + head0 + 1) * 2 + 1] = l1;
+                }
+            }
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+                const int dr = dt * 16 + (lane >> 2);
+                if (head0 < g) {
+                    float* po = part_o + ((size_t)cons.item * g + head0) * 128;
+                    po[dr] = o[nt][dt][0];
+                    po[dr + 8] = o[nt][dt][2];
+                }
+                if (head0 + 1 < g) {
+                    float* po = part_o + ((size_t)cons.item * g + head0 + 1) * 128;
+                    po[dr] = o[nt][dt][1];
+                    po[dr + 8] = o[nt][dt][3];
+                }
+            }
+        }
+        cons = load_item(cons.item + GW);
+    }
+
+    if (failed) {
+        latch_error(cv.err, TRIMKV_E_TIMEOUT);
+        // drain: wait (bounded) for the copies still in flight before leaving shared memory
+        while (consumed < issued) {
+            const unsigned s = consumed % ATT_STAGES;
+            mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u);
+            ++consumed;
+        }
+    }
+}
+
+// Merge the partials of every pool in scope: out = sum_i 2^(m_i - M) O_i / sum_i 2^(m_i - M) l_i.
+__global__ void __launch_bounds__(128)
+attn_merge_kernel(CacheView cv, int g, int Hq, const int32_t* __restrict__ item_prefix, const float* __restrict__ part_o,
+                  const float* __restrict__ part_ml, __nv_bfloat16* __restrict__ out) {
+    const int si = blockIdx.x;
+    const int h = si % cv.H;
+    const int lbb = si / cv.H;
+    const int i0 = item_prefix[si], i1 = item_prefix[si + 1];
+    const int d = threadIdx.x;   // 128 threads = one per output column
+    for (int j = 0; j < g; ++j) {
+        float M = -INFINITY;
+        for (int it = i0; it < i1; ++it) M = fmaxf(M, part_ml[((size_t)it * g + j) * 2]);
+        float num = 0.f, den = 0.f;
+        for (int it = i0; it < i1; ++it) {
+            const float w = exp2f(part_ml[((size_t)it * g + j) * 2] - M);
+            den += w * part_ml[((size_t)it * g + j) * 2 + 1];
+            num += w * part_o[((size_t)it * g + j) * 128 + d];
+        }
+        const float r = (i1 > i0 && den > 0.f) ? num / den : 0.f;
+        out[((size_t)lbb * Hq + (size_t)h * g + j) * 128 + d] = __float2bfloat16_rn(r);
+    }
+}
+
+// ------------------------------------------------------------------ plain kernel: any d, fp32 or bf16
+template <typename T>
+__device__ __forceinline__ float to_f32(T v);
+template <>
+__device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T>
+__device__ __forceinline__ T from_f32(float v);
+template <>
+__device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// One warp per (pool in scope, query head of its group).  Lanes split d; per entry one warp reduction.
+template <typename T, int MAXD>
+__global__ void __launch_bounds__(128)
+attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T* __restrict__ q, T* __restrict__ out,
+                  float scale) {
+    const int wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (wid >= n_scope * g) return;
+    const int si = wid / g, j = wid % g;
+    const int h = si % cv.H, lbb = si / cv.H, b = lbb % cv.B;
+    const long long pool = scope_pool(cv, layer0, si);
+    const int n = cv.len[pool];
+    const int d = cv.d;
+    constexpr int PER = MAXD / 32;
+    const int epc = 16 / (int)sizeof(T);          // elements per 16-byte chunk
+    float qr[PER], acc[PER];
+    const T* qp = q + ((size_t)lbb * Hq + (size_t)h * g + j) * d;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int dd = lane + 32 * i;
+        qr[i] = dd < d ? to_f32<T>(qp[dd]) * scale : 0.f;
+        acc[i] = 0.f;
+    }
+    float m = -INFINITY, l = 0.f;
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    for (int e = 0; e < n; ++e) {
+        const int page = bt[e / PAGE], off = e % PAGE;
+        const T* kr = reinterpret_cast<const T*>(cv.kv + kv_row_offset(cv, b, page, 0, off));
+        const T* vr = reinterpret_cast<const T*>(cv.kv + kv_row_offset(cv, b, page, 1, off));
+        float s = 0.f;
+        int pidx[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int dd = lane + 32 * i;
+            pidx[i] = phys_chunk(cv, dd / epc, off) * epc + dd % epc;
+            if (dd < d) s = fmaf(qr[i], to_f32<T>(kr[pidx[i]]), s);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        const float mn = fmaxf(m, s);
+        const float f = __expf(m - mn), p = __expf(s - mn);
+        l = l * f + p;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int dd = lane + 32 * i;
+            if (dd < d) acc[i] = acc[i] * f + p * to_f32<T>(vr[pidx[i]]);
+        }
+        m = mn;
+    }
+    T* op = out + ((size_t)lbb * Hq + (size_t)h * g + j) * d;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int dd = lane + 32 * i;
+        if (dd < d) op[dd] = from_f32<T>(n > 0 ? acc[i] / l : 0.f);
+    }
+}
+
+}  // namespace
+
+void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
+                      long long tiles_estimate, long long tiles_upper, const void* q, void* out, cudaStream_t st,
+                      PhaseMarker* pm) {
+    const int n_scope = nlayers * cv.B * cv.H;
+    const int g = Hq / cv.H;
+    const float scale = 1.0f / sqrtf((float)cv.d);
+    if (is_bf16 && cv.d == 128 && g <= 16) {
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaFuncSetAttribute(attn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            cudaFuncSetAttribute(attn_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            attr_set = true;
+        }
+        int dev = 0, sms = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const long long workers = (long long)sms * ATT_WARPS;
+        long long tpi = tiles_estimate / (workers * 24);       // ~24 items per worker for balance
+        const long long room = ab.max_items - n_scope;          // items <= tiles / tpi + n_scope must fit
+        if (room > 0) tpi = std::max(tpi, (tiles_upper + room - 1) / room);
+        tpi = (tpi + 1) & ~1LL;
+        if (tpi < 2) tpi = 2;
+        if (tpi > 64) tpi = 64;
+        if (pm) pm->mark(PH_ATTN_PLAN, 0, st);
+        attn_plan_kernel<<<1, 1024, 0, st>>>(cv, layer0, n_scope, (int)tpi, ab.item_prefix, ab.item_desc, ab.max_items);
+        if (pm) { pm->mark(PH_ATTN_PLAN, 1, st); pm->mark(PH_ATTN_MAIN, 0, st); }
+        const float scale_log2 = scale * 1.4426950408889634f;
+        if (g <= 8)
+            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, g, Hq, ab.item_prefix,
+                                                                      ab.item_desc, (const __nv_bfloat16*)q, ab.part_o,
+                                                                      ab.part_ml, scale_log2, ab.max_items);
+        else
+            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, g, Hq, ab.item_prefix,
+                                                                      ab.item_desc, (const __nv_bfloat16*)q, ab.part_o,
+                                                                      ab.part_ml, scale_log2, ab.max_items);
+        if (pm) { pm->mark(PH_ATTN_MAIN, 1, st); pm->mark(PH_ATTN_MERGE, 0, st); }
+        attn_merge_kernel<<<n_scope, 128, 0, st>>>(cv, g, Hq, ab.item_prefix, ab.part_o, ab.part_ml, (__nv_bfloat16*)out);
+        if (pm) pm->mark(PH_ATTN_MERGE, 1, st);
+        count_launch(3);
+    } else {
+        const int warps = n_scope * g;
+        const int grid = (warps + 3) / 4;
+        if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
+        if (is_bf16)
+            attn_plain_kernel<__nv_bfloat16, 256><<<grid, 128, 0, st>>>(cv, layer0, n_scope, g, Hq, (const __nv_bfloat16*)q,
+                                                                         (__nv_bfloat16*)out, scale);
+        else
+            attn_plain_kernel<float, 256><<<grid, 128, 0, st>>>(cv, layer0, n_scope, g, Hq, (const float*)q, (float*)out,
+                                                                scale);
+        if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
+        count_launch();
+    }
+}
+
+}  // namespace tkv

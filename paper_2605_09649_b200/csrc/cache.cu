@@ -1,0 +1,278 @@
+// Paged per-(layer, head) KV pools (Sec. 4.2 "Implementation details": fixed-size pages, one block
+// table per head, variable logical length per head): append of new tokens and compaction after an
+// eviction round.
+#include "trimkv_internal.cuh"
+
+namespace tkv {
+
+namespace {
+
+// One CTA per pool: take pages from the sequence's free stack if the pool grows past its last page,
+// then copy the new rows (K, V, retention metadata) to their slots.
+__global__ void __launch_bounds__(256)
+append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* __restrict__ lam_in,
+              const float* __restrict__ c_in, int horizon, const char* __restrict__ k_in,
+              const char* __restrict__ v_in) {
+    __shared__ int s_old;
+    __shared__ int s_fail;
+    const int h = blockIdx.x % cv.H;
+    const int b = (blockIdx.x / cv.H) % cv.B;
+    const int lb = blockIdx.x / (cv.H * cv.B);
+    const int layer = layer0 + lb;
+    const int pool_local = layer * cv.H + h;
+    const long long pool = (long long)b * cv.L * cv.H + pool_local;
+    int32_t* bt = cv.block_table + pool * cv.maxpp;
+
+    if (threadIdx.x == 0) {
+        const int old = cv.len[pool];
+        const long long nw = (long long)old + n_new;
+        const long long p_old = (old + PAGE - 1) / PAGE, p_new = (nw + PAGE - 1) / PAGE;
+        int fail = 0;
+        if (p_new > cv.maxpp) {
+            fail = 1;
+        } else if (p_new > p_old) {
+            const int need = (int)(p_new - p_old);
+            const int prev = atomicSub(&cv.free_count[b], need);
+            if (prev < need) {
+                atomicAdd(&cv.free_count[b], need);
+                fail = 1;
+            } else {
+                const int32_t* stack = cv.free_stack + (size_t)b * cv.P_seq;
+                for (int j = 0; j < need; ++j) {
+                    const int page = stack[prev - 1 - j];
+                    bt[p_old + j] = page;
+                    cv.owner[(size_t)b * cv.P_seq + page] = make_int2(pool_local, (int)(p_old + j));
+                }
+            }
+        }
+        if (fail) latch_error(cv.err, TRIMKV_E_NOMEM);
+        s_old = old;
+        s_fail = fail;
+    }
+    __syncthreads();
+    if (s_fail) return;
+    const int old = s_old;
+
+    // rows: [lb][b][j][h][d]
+    const int rc = cv.row_bytes / 16;                  // 16-byte chunks per row
+    const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
+    const int total = n_new * rc * 2;
+    for (int w = threadIdx.x; w < total; w += blockDim.x) {
+        const int ci = w % rc;
+        const int part = (w / rc) & 1;
+        const int j = w / (2 * rc);
+        const int idx = old + j;
+        const int page = bt[idx / PAGE];
+        const int off = idx % PAGE;
+        const char* src = (part ? v_in : k_in) + (in_row0 + (size_t)j * cv.H) * cv.row_bytes + (size_t)ci * 16;
+        char* dst = cv.kv + kv_row_offset(cv, b, page, part, off) + (size_t)phys_chunk(cv, ci, off) * 16;
+        *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    }
+    for (int j = threadIdx.x; j < n_new; j += blockDim.x) {
+        const int idx = old + j;
+        const int page = bt[idx / PAGE];
+        const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + idx % PAGE;
+        const size_t mi = (in_row0 + (size_t)j * cv.H);
+        const float lm = lam_in[mi];
+        const float cc = c_in ? c_in[mi] : horizon_term_f32(lm, horizon);
+        if (lm != lm || cc != cc) latch_error(cv.err, TRIMKV_E_NONFINITE);
+        cv.lam[slot] = lm;
+        cv.c[slot] = cc;
+        cv.pos[slot] = (int32_t)(pos0 + j + 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) cv.len[pool] = old + n_new;
+}
+
+__device__ __forceinline__ u64 bits_below(int n) {   // mask with the lowest n bits set, n in [0, 64]
+    return n >= 64 ? ~0ull : ((1ull << n) - 1ull);
+}
+
+// Block-wide exclusive scan of a 64-bit value over 256 threads; returns the exclusive prefix and the total.
+__device__ __forceinline__ u64 block_exscan_256(u64 v, u64* total, u64* warp_tot /*[8] shared*/) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    u64 incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        u64 t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    u64 off = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        const u64 t = warp_tot[w];
+        if (w < warp) off += t;
+        tot += t;
+    }
+    *total = tot;
+    return off + incl - v;
+}
+
+// One CTA per pool.  Entries flagged in evict_mask are removed: with n' = n - E survivors, the E' holes
+// at logical index < n' are filled, in ascending order, by the survivors at index >= n' (ascending), so
+// only as many rows move as there are holes.  Pages past the new end return to the free stack.
+__global__ void __launch_bounds__(256)
+compact_kernel(CacheView cv, int32_t* __restrict__ hole, int32_t* __restrict__ mover, int32_t* __restrict__ cursor,
+               long long e_max) {
+    __shared__ u64 warp_tot[8];
+    __shared__ long long s_base;
+    __shared__ int s_freebase;
+    const long long pool = blockIdx.x;
+    const int b = (int)(pool / ((long long)cv.L * cv.H));
+    const int n = cv.len[pool];
+    if (n == 0) return;
+    const int np = (n + PAGE - 1) / PAGE;
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    const u64* masks = cv.evict_mask + (size_t)b * cv.P_seq;
+
+    // phase 1: number of evicted entries
+    u64 e_local = 0;
+    for (int lp = threadIdx.x; lp < np; lp += blockDim.x) {
+        const u64 valid = bits_below(min(PAGE, n - lp * PAGE));
+        e_local += __popcll(masks[bt[lp]] & valid);
+    }
+    u64 E;
+    block_exscan_256(e_local, &E, warp_tot);
+    if (E == 0) return;
+    const int n2 = n - (int)E;
+
+    if (threadIdx.x == 0) {
+        const long long base = (long long)atomicAdd(cursor + b, (int)E);
+        s_base = base;
+        if (base + (long long)E > e_max) latch_error(cv.err, TRIMKV_E_NOMEM);
+    }
+    __syncthreads();
+    if (s_base + (long long)E > e_max) return;
+    int32_t* hl = hole + (size_t)b * e_max + s_base;
+    int32_t* ml = mover + (size_t)b * e_max + s_base;
+
+    // phase 2: ordered lists of holes (evicted, index < n2) and movers (kept, index >= n2)
+    long long run_h = 0, run_m = 0;
+    for (int base = 0; base < np; base += blockDim.x) {
+        const int lp = base + threadIdx.x;
+        u64 hb = 0, mb = 0;
+        int page = 0;
+        if (lp < np) {
+            page = bt[lp];
+            const u64 valid = bits_below(min(PAGE, n - lp * PAGE));
+            const u64 m = masks[page] & valid;
+            const u64 below = bits_below(max(0, min(PAGE, n2 - lp * PAGE)));   // indices < n2 within this page
+            hb = m & below;
+            mb = ~m & valid & ~below;
+        }
+        const u64 packed = ((u64)__popcll(hb) << 32) | (u64)__popcll(mb);
+        u64 tot;
+        const u64 ex = block_exscan_256(packed, &tot, warp_tot);
+        long long ho = run_h + (long long)(ex >> 32), mo = run_m + (long long)(ex & 0xffffffffu);
+        while (hb) {
+            const int bit = __ffsll((long long)hb) - 1;
+            hb &= hb - 1;
+            hl[ho++] = page * PAGE + bit;
+        }
+        while (mb) {
+            const int bit = __ffsll((long long)mb) - 1;
+            mb &= mb - 1;
+            ml[mo++] = page * PAGE + bit;
+        }
+        run_h += (long long)(tot >> 32);
+        run_m += (long long)(tot & 0xffffffffu);
+    }
+    __syncthreads();
+    if (run_h != run_m) {                       // cannot happen; guards the copy loop against bad masks
+        if (threadIdx.x == 0) latch_error(cv.err, TRIMKV_E_STATE);
+        return;
+    }
+
+    // phase 3: move rows (K, V by 16-byte chunks; metadata by one thread per move)
+    const int rc = cv.row_bytes / 16;
+    const long long work = run_h * (2 * rc + 1);
+    for (long long w = threadIdx.x; w < work; w += blockDim.x) {
+        const long long j = w / (2 * rc + 1);
+        const int r = (int)(w % (2 * rc + 1));
+        const int src = ml[j], dst = hl[j];
+        const int sp = src / PAGE, so = src % PAGE, dp = dst / PAGE, dof = dst % PAGE;
+        if (r == 2 * rc) {
+            const size_t ss = ((size_t)b * cv.P_seq + sp) * PAGE + so, ds = ((size_t)b * cv.P_seq + dp) * PAGE + dof;
+            cv.lam[ds] = cv.lam[ss];
+            cv.c[ds] = cv.c[ss];
+            cv.pos[ds] = cv.pos[ss];
+        } else {
+            const int part = r / rc, ci = r % rc;
+            const char* s = cv.kv + kv_row_offset(cv, b, sp, part, so) + (size_t)phys_chunk(cv, ci, so) * 16;
+            char* d = cv.kv + kv_row_offset(cv, b, dp, part, dof) + (size_t)phys_chunk(cv, ci, dof) * 16;
+            *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(s);
+        }
+    }
+    __syncthreads();
+
+    // phase 4: new length, release pages past the end
+    const int np2 = (n2 + PAGE - 1) / PAGE;
+    const int nfree = np - np2;
+    if (threadIdx.x == 0) {
+        cv.len[pool] = n2;
+        s_freebase = nfree > 0 ? atomicAdd(&cv.free_count[b], nfree) : 0;
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < nfree; j += blockDim.x) {
+        const int page = bt[np2 + j];
+        cv.free_stack[(size_t)b * cv.P_seq + s_freebase + j] = page;
+        cv.owner[(size_t)b * cv.P_seq + page] = make_int2(-1, 0);
+    }
+}
+
+// Copies one pool's entries, in storage order, to dense device buffers (undoing the chunk permutation).
+__global__ void gather_pool_kernel(CacheView cv, int b, long long pool, int n, int32_t* pos, float* lam, float* c,
+                                   char* k, char* v) {
+    const int rc = cv.row_bytes / 16;
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    const long long work = (long long)n * (2 * rc + 1);
+    for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < work;
+         w += (long long)gridDim.x * blockDim.x) {
+        const int i = (int)(w / (2 * rc + 1));
+        const int r = (int)(w % (2 * rc + 1));
+        const int page = bt[i / PAGE], off = i % PAGE;
+        if (r == 2 * rc) {
+            const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
+            if (pos) pos[i] = cv.pos[s];
+            if (lam) lam[i] = cv.lam[s];
+            if (c) c[i] = cv.c[s];
+        } else {
+            const int part = r / rc, ci = r % rc;
+            char* dst = part ? v : k;
+            if (dst) {
+                const char* s = cv.kv + kv_row_offset(cv, b, page, part, off) + (size_t)phys_chunk(cv, ci, off) * 16;
+                *reinterpret_cast<uint4*>(dst + (size_t)i * cv.row_bytes + (size_t)ci * 16) =
+                    *reinterpret_cast<const uint4*>(s);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
+                   const float* c, int horizon, const void* k, const void* v, cudaStream_t st) {
+    const int grid = nlayers * cv.B * cv.H;
+    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v);
+    count_launch();
+}
+
+void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max,
+                    cudaStream_t st) {
+    const long long pools = (long long)cv.B * cv.L * cv.H;
+    compact_kernel<<<(unsigned)pools, 256, 0, st>>>(cv, hole, mover, cursor, e_max);
+    count_launch();
+}
+
+void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
+                        void* v, int n, cudaStream_t st) {
+    if (n <= 0) return;
+    const long long pool = ((long long)seq * cv.L + layer) * cv.H + head;
+    gather_pool_kernel<<<64, 256, 0, st>>>(cv, seq, pool, n, pos, lam, c, (char*)k, (char*)v);
+    count_launch();
+}
+
+}  // namespace tkv

@@ -1,0 +1,177 @@
+// Internal declarations shared by the translation units of the trimkv library.
+// Not part of the public ABI.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "trimkv.h"
+
+namespace tkv {
+
+// ------------------------------------------------------------------ constants
+constexpr int PAGE = 64;                 // entries per page
+constexpr int NB = 4096;                 // histogram bins: 0 = below range, 1..NB-2 regular, NB-1 = above range (not counted)
+constexpr int REG_BINS = NB - 2;
+constexpr int ZOOM_BITS = 11;            // a zoom maps the surviving key range onto <= 2^11 regular bins
+constexpr int MAX_HIST_PASSES = 3;       // histogram passes per selection; the last one resolves unconditionally
+constexpr int INIT_SHIFT = 64 - ZOOM_BITS;
+
+typedef unsigned long long u64;
+
+// Per-sequence selection state (device resident, persists between calls so that the first
+// histogram pass of a call can be centred on the previous call's threshold).
+struct SelState {
+    u64 lo;            // key at the lower edge of regular bin 1
+    u64 kmin, kmax;    // min / max key seen during the running pass
+    u64 cand_lo;       // candidate range [cand_lo, cand_hi]: keys below are evicted, above are kept
+    u64 cand_hi;
+    long long n_below; // number of keys < cand_lo
+    int shift;         // bin width = 2^shift keys
+    int resolved;      // 1 once the candidate range is final for this call
+    int passes;        // histogram passes run in this call
+    unsigned int cand_count;   // candidates appended by the filter pass
+    unsigned int cand_expected;
+    int pad;
+};
+
+struct Cand {          // one candidate of the exact resolution stage
+    u64 key;
+    u64 slot;          // slot index inside the sequence (page * 64 + offset) or flat index
+};
+
+// Order-preserving map of a float onto uint32 (smaller float -> smaller integer); -0 is folded onto +0.
+__device__ __forceinline__ uint32_t orderable_key(float s) {
+    s = __fadd_rn(s, 0.0f);
+    uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Retention score in log space: S = c + age * lambda with one fp32 multiply and one fp32 add,
+// each rounded to nearest even and never contracted into an FMA.
+__device__ __forceinline__ float retention_score(float lam, float c, float age) {
+    return __fadd_rn(c, __fmul_rn(age, lam));
+}
+
+// Eviction-order key: entries with the SMALLEST keys are evicted first.
+//   high 32 bits: orderable score; low 32 bits: ~tie, where a larger tie (newer position, then higher
+//   layer*H+head) is evicted first among equal scores.
+__device__ __forceinline__ u64 make_key(float score, uint32_t tie) {
+    return ((u64)orderable_key(score) << 32) | (u64)(~tie);
+}
+
+// c = ln sum_{k<horizon} exp(k * lambda): the beta-only factor of the retention score (horizon 0 = infinite).
+__device__ __forceinline__ float horizon_term_f32(float lam, int horizon) {
+    if (horizon == 1) return 0.0f;
+    if (horizon == 0) return -logf(-expm1f(lam));
+    float acc = 1.0f;
+    for (int k = 1; k < horizon; ++k) acc += expf((float)k * lam);
+    return logf(acc);
+}
+
+__device__ __forceinline__ int bin_of(u64 key, u64 lo, int shift) {
+    if (key < lo) return 0;
+    u64 idx = (key - lo) >> shift;
+    return idx >= (u64)REG_BINS ? NB - 1 : (int)idx + 1;
+}
+
+// ------------------------------------------------------------------ cache geometry
+// KV storage: kv[b][page][2][PAGE][row_bytes]; part 0 = K rows, part 1 = V rows of the page.
+// bf16 rows whose length is a multiple of 128 bytes are stored with their 16-byte chunks permuted
+// inside each 128-byte group: physical chunk = logical chunk ^ (slot_in_page & 7).  A linear bulk copy of
+// a page to shared memory is then bank-conflict free for 8-row matrix loads.
+struct CacheView {
+    char* kv;
+    float* lam;
+    float* c;
+    int32_t* pos;
+    int2* owner;           // [B][P_seq] {pool_local or -1, logical page index}
+    int32_t* block_table;  // [B*L*H][maxpp]
+    int32_t* len;          // [B*L*H]
+    int32_t* free_stack;   // [B][P_seq]
+    int32_t* free_count;   // [B]
+    u64* evict_mask;       // [B][P_seq]
+    int32_t* err;          // latched device status
+    long long P_seq;       // pages per sequence
+    long long maxpp;       // block-table row length
+    int B, L, H, d;
+    int row_bytes;         // d * sizeof(element)
+    int swizzle;           // 1 if rows are chunk-permuted
+    int pool_bits;         // bits that hold layer*H+head in the tie-break word
+};
+
+__device__ __forceinline__ size_t kv_row_offset(const CacheView& cv, int b, long long page, int part, int off) {
+    return ((((size_t)b * cv.P_seq + page) * 2 + part) * PAGE + off) * (size_t)cv.row_bytes;
+}
+__device__ __forceinline__ int phys_chunk(const CacheView& cv, int chunk, int off) {
+    return cv.swizzle ? (chunk ^ (off & 7)) : chunk;
+}
+
+__device__ __forceinline__ void latch_error(int32_t* err, int code) {
+    if (err) atomicCAS(err, 0, code);
+}
+
+// ------------------------------------------------------------------ launchers (host)
+struct GateParams {
+    const float* W1;  // [L][dg][D]
+    const float* b1;  // [L][dg]
+    const float* W2;  // [L][H][de][dg]
+    const float* b2;  // [L][H][de]
+    const float* w_g; // [de]
+    float b_g;
+    int D, dg, de, H, horizon;
+};
+
+// rows_per_layer rows of x per layer, layers [layer0, layer0 + nlayers).
+void launch_gate(const GateParams& gp, const float* x, float* u_scratch, int layer0, int nlayers, int rows_per_layer,
+                 float* beta, float* lam, float* c, cudaStream_t st);
+
+void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
+                   const float* c, int horizon, const void* k, const void* v, cudaStream_t st);
+
+struct SelectBuffers {
+    SelState* sel;        // [B]
+    uint32_t* hist;       // [B][NB]
+    unsigned int* done;   // [B]
+    Cand* cand;           // [B][cand_cap]
+    long long cand_cap;
+    long long* stats;     // [B][4]
+};
+
+// compact_cursor [B]: zeroed by the selection for the compaction that follows.
+void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, long long k_evict,
+                         int32_t* compact_cursor, cudaStream_t st);
+void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max, cudaStream_t st);
+
+void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,
+                         int32_t* err, cudaStream_t st);
+void launch_invert_mask(const u64* evict_mask, u64* keep_bits, long long n, cudaStream_t st);
+void launch_select_state_init(SelState* sel, int B, cudaStream_t st);
+
+struct AttnBuffers {
+    int32_t* item_prefix;  // [pools_in_scope + 1]
+    int2* item_desc;       // [max_items] {scope index, first tile}
+    float* part_o;         // [max_items][g][d]
+    float* part_ml;        // [max_items][g][2]
+    long long max_items;
+};
+
+// Optional per-phase timing: mark(phase, 0) before and mark(phase, 1) after a phase's launches.
+enum Phase { PH_GATE = 0, PH_APPEND = 1, PH_ATTN_PLAN = 2, PH_ATTN_MAIN = 3, PH_ATTN_MERGE = 4, PH_SELECT = 5,
+             PH_COMPACT = 6, PH_COUNT = 8 };
+struct PhaseMarker {
+    virtual void mark(int phase, int end, cudaStream_t st) = 0;
+    virtual ~PhaseMarker() {}
+};
+
+void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
+                      long long tiles_estimate, long long tiles_upper, const void* q, void* out, cudaStream_t st,
+                      PhaseMarker* pm);
+
+void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
+                        void* v, int n, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace tkv

@@ -1,0 +1,574 @@
+// Host side of the trimkv C ABI: handle, device memory, call-order checks, kernel orchestration.
+#include <algorithm>
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "trimkv_internal.cuh"
+
+namespace tkv {
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace tkv
+
+using namespace tkv;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+trimkv_status fail(trimkv_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+#define CUDA_TRY(expr)                                                                                     \
+    do {                                                                                                   \
+        cudaError_t e__ = (expr);                                                                          \
+        if (e__ != cudaSuccess)                                                                            \
+            return fail(e__ == cudaErrorMemoryAllocation ? TRIMKV_E_NOMEM : TRIMKV_E_CUDA, "%s: %s", #expr, \
+                        cudaGetErrorString(e__));                                                          \
+    } while (0)
+
+int ceil_log2(long long v) {
+    int b = 0;
+    while ((1LL << b) < v) ++b;
+    return b;
+}
+
+}  // namespace
+
+struct Profiler : public tkv::PhaseMarker {
+    bool on = false;
+    std::vector<cudaEvent_t> pool;                 // reusable events
+    size_t used = 0;
+    std::vector<std::pair<int, std::pair<cudaEvent_t, cudaEvent_t>>> recs;
+    cudaEvent_t open_ev[tkv::PH_COUNT] = {};
+    cudaEvent_t get() {
+        if (used == pool.size()) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+            pool.push_back(e);
+        }
+        return pool[used++];
+    }
+    void mark(int phase, int end, cudaStream_t st) override {
+        if (!on || recs.size() >= (1u << 18)) return;
+        cudaEvent_t e = get();
+        if (!e) return;
+        cudaEventRecord(e, st);
+        if (!end) open_ev[phase] = e;
+        else if (open_ev[phase]) { recs.push_back({phase, {open_ev[phase], e}}); open_ev[phase] = nullptr; }
+    }
+    void clear() { recs.clear(); used = 0; for (auto& e : open_ev) e = nullptr; }
+    ~Profiler() override { for (cudaEvent_t e : pool) cudaEventDestroy(e); }
+};
+
+struct trimkv {
+    trimkv_config cfg;
+    Profiler prof;
+    int B, L, H, Hq, g, d, D, dg, de, elt;
+    long long M, P_seq, maxpp, slots_seq, e_max, n_max;
+    int pool_bits;
+    long long max_pos;
+    CacheView cv;
+    SelectBuffers sb;
+    AttnBuffers ab;
+    int32_t *hole, *mover, *cursor;
+    float *W1, *b1, *W2, *b2, *w_g, *u, *g_lam, *g_c;
+    float b_g;
+    bool shared_set;
+    std::vector<char> gate_set;
+    std::vector<long long> tokens;   // per layer
+    long long entries;               // per sequence (all sequences advance together)
+    long long rows_max;
+    std::vector<void*> allocs;
+};
+
+namespace {
+
+template <class T>
+trimkv_status dev_alloc(trimkv* h, T** p, size_t count, bool zero) {
+    void* q = nullptr;
+    size_t bytes = std::max<size_t>(count * sizeof(T), 256);
+    cudaError_t e = cudaMalloc(&q, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(TRIMKV_E_NOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+    }
+    h->allocs.push_back(q);
+    if (zero) {
+        e = cudaMemset(q, 0, bytes);
+        if (e != cudaSuccess) return fail(TRIMKV_E_CUDA, "cudaMemset: %s", cudaGetErrorString(e));
+    }
+    *p = reinterpret_cast<T*>(q);
+    return TRIMKV_OK;
+}
+
+trimkv_status init_cache_state(trimkv* h) {
+    // free stacks: pops take the lowest page ids first
+    std::vector<int32_t> stack((size_t)h->B * h->P_seq);
+    for (int b = 0; b < h->B; ++b)
+        for (long long p = 0; p < h->P_seq; ++p) stack[(size_t)b * h->P_seq + p] = (int32_t)(h->P_seq - 1 - p);
+    CUDA_TRY(cudaMemcpy(h->cv.free_stack, stack.data(), stack.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    std::vector<int32_t> cnt(h->B, (int32_t)h->P_seq);
+    CUDA_TRY(cudaMemcpy(h->cv.free_count, cnt.data(), cnt.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    std::vector<int2> own((size_t)h->B * h->P_seq, make_int2(-1, 0));
+    CUDA_TRY(cudaMemcpy(h->cv.owner, own.data(), own.size() * sizeof(int2), cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemset(h->cv.len, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
+    CUDA_TRY(cudaMemset(h->cv.err, 0, sizeof(int32_t)));
+    CUDA_TRY(cudaMemset(h->sb.hist, 0, (size_t)h->B * NB * sizeof(uint32_t)));
+    CUDA_TRY(cudaMemset(h->sb.done, 0, (size_t)h->B * sizeof(unsigned)));
+    CUDA_TRY(cudaMemset(h->sb.stats, 0, (size_t)h->B * 4 * sizeof(long long)));
+    CUDA_TRY(cudaMemset(h->cursor, 0, (size_t)h->B * sizeof(int32_t)));
+    launch_select_state_init(h->sb.sel, h->B, 0);
+    CUDA_TRY(cudaDeviceSynchronize());
+    std::fill(h->tokens.begin(), h->tokens.end(), 0LL);
+    h->entries = 0;
+    return TRIMKV_OK;
+}
+
+trimkv_status check_handle(trimkv_t* h) { return h ? TRIMKV_OK : fail(TRIMKV_E_ARG, "NULL handle"); }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+trimkv_status device_status(trimkv* h) {
+    int32_t code = 0;
+    CUDA_TRY(cudaMemcpy(&code, h->cv.err, sizeof(code), cudaMemcpyDeviceToHost));
+    if (code != 0) return fail((trimkv_status)code, "device-side error %d latched by a kernel", code);
+    return TRIMKV_OK;
+}
+
+GateParams gate_params(const trimkv* h) {
+    GateParams gp;
+    gp.W1 = h->W1; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.b_g = h->b_g;
+    gp.D = h->D; gp.dg = h->dg; gp.de = h->de; gp.H = h->H; gp.horizon = h->cfg.horizon;
+    return gp;
+}
+
+trimkv_status gate_ready(const trimkv* h, int layer0, int nlayers) {
+    if (h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
+    if (!h->shared_set) return fail(TRIMKV_E_STATE, "shared projection not set");
+    for (int l = layer0; l < layer0 + nlayers; ++l)
+        if (!h->gate_set[l]) return fail(TRIMKV_E_STATE, "gate of layer %d not set", l);
+    return TRIMKV_OK;
+}
+
+trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
+    const long long t = h->tokens[0];
+    for (int l = 1; l < h->L; ++l)
+        if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layer %d holds %lld tokens, layer 0 holds %lld", l, h->tokens[l], t);
+    const long long k = h->entries - h->M;
+    if (k <= 0) return TRIMKV_OK;
+    PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
+    if (pm) pm->mark(PH_SELECT, 0, st);
+    launch_select_cache(h->cv, h->sb, t, h->entries, k, h->cursor, st);
+    if (pm) { pm->mark(PH_SELECT, 1, st); pm->mark(PH_COMPACT, 0, st); }
+    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
+    if (pm) pm->mark(PH_COMPACT, 1, st);
+    h->entries = h->M;
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, void* out, cudaStream_t st) {
+    const long long tiles = (h->entries * h->B / 32) * nlayers / h->L + (long long)nlayers * h->B * h->H;
+    const long long tiles_upper = h->entries * h->B / 32 + (long long)nlayers * h->B * h->H;
+    launch_attention(h->cv, h->ab, layer0, nlayers, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, tiles, tiles_upper, q,
+                     out, st, h->prof.on ? &h->prof : nullptr);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void trimkv_default_config(trimkv_config* cfg, int64_t budget_entries, int layers, int kv_heads, int head_dim) {
+    if (!cfg) return;
+    memset(cfg, 0, sizeof(*cfg));
+    cfg->budget_entries = budget_entries;
+    cfg->layers = layers;
+    cfg->kv_heads = kv_heads;
+    cfg->q_heads = kv_heads;
+    cfg->head_dim = head_dim;
+    cfg->hidden = 0;
+    cfg->max_batch = 1;
+    cfg->page_size = PAGE;
+    cfg->gate_hidden = 512;
+    cfg->gate_embed = 64;
+    cfg->horizon = 2;
+    cfg->kv_dtype = TRIMKV_DTYPE_BF16;
+    cfg->max_chunk = 512;
+    cfg->max_pool_pages = 0;
+}
+
+trimkv_t* trimkv_create(int64_t budget_entries, int layers, int kv_heads, int head_dim) {
+    trimkv_config cfg;
+    trimkv_default_config(&cfg, budget_entries, layers, kv_heads, head_dim);
+    trimkv_t* h = nullptr;
+    if (trimkv_create_ex(&cfg, &h) != TRIMKV_OK) return nullptr;
+    return h;
+}
+
+trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
+    if (!cfg || !out) return fail(TRIMKV_E_ARG, "NULL argument");
+    *out = nullptr;
+    if (cfg->budget_entries < 1 || cfg->layers < 1 || cfg->kv_heads < 1 || cfg->head_dim < 8 || cfg->max_batch < 1 ||
+        cfg->max_chunk < 1)
+        return fail(TRIMKV_E_ARG, "budget, layers, kv_heads, head_dim, max_batch and max_chunk must be positive");
+    if (cfg->page_size != PAGE) return fail(TRIMKV_E_UNSUPPORTED, "page_size must be %d", PAGE);
+    if (cfg->q_heads < cfg->kv_heads || cfg->q_heads % cfg->kv_heads) return fail(TRIMKV_E_ARG, "q_heads must be a multiple of kv_heads");
+    if (cfg->kv_dtype != TRIMKV_DTYPE_BF16 && cfg->kv_dtype != TRIMKV_DTYPE_F32) return fail(TRIMKV_E_ARG, "unknown kv_dtype");
+    if (cfg->head_dim % 8 || cfg->head_dim > 256) return fail(TRIMKV_E_UNSUPPORTED, "head_dim must be a multiple of 8, at most 256");
+    if (cfg->horizon < 0 || cfg->horizon > 64) return fail(TRIMKV_E_ARG, "horizon must be in [0, 64]");
+    if (cfg->hidden < 0 || (cfg->hidden > 0 && (cfg->hidden % 4 || cfg->gate_hidden < 4 || cfg->gate_hidden % 4 || cfg->gate_embed < 1)))
+        return fail(TRIMKV_E_ARG, "hidden and gate_hidden must be multiples of 4, gate_embed positive");
+    if ((long long)cfg->layers * cfg->kv_heads > 65536) return fail(TRIMKV_E_UNSUPPORTED, "layers * kv_heads too large");
+
+    trimkv* h = new (std::nothrow) trimkv();
+    if (!h) return fail(TRIMKV_E_NOMEM, "host allocation failed");
+    h->cfg = *cfg;
+    h->B = cfg->max_batch; h->L = cfg->layers; h->H = cfg->kv_heads; h->Hq = cfg->q_heads; h->g = h->Hq / h->H;
+    h->d = cfg->head_dim; h->D = cfg->hidden; h->dg = cfg->gate_hidden; h->de = cfg->gate_embed;
+    h->elt = cfg->kv_dtype == TRIMKV_DTYPE_BF16 ? 2 : 4;
+    h->M = cfg->budget_entries;
+    const long long LH = (long long)h->L * h->H;
+    h->e_max = (long long)cfg->max_chunk * LH;
+    h->n_max = h->M + h->e_max;
+    h->P_seq = (h->n_max + PAGE - 1) / PAGE + LH + 8;
+    h->maxpp = cfg->max_pool_pages > 0 ? std::min<long long>(cfg->max_pool_pages, h->P_seq) : h->P_seq;
+    h->slots_seq = h->P_seq * PAGE;
+    h->pool_bits = std::max(1, ceil_log2(LH));
+    h->max_pos = std::min<long long>((1LL << 24) - 1, (1LL << (32 - h->pool_bits)) - 1);
+    h->tokens.assign(h->L, 0);
+    h->gate_set.assign(h->L, 0);
+    h->shared_set = false;
+    h->b_g = 0.f;
+    h->entries = 0;
+    h->W1 = h->b1 = h->W2 = h->b2 = h->w_g = h->u = h->g_lam = h->g_c = nullptr;
+
+    CacheView& cv = h->cv;
+    memset(&cv, 0, sizeof(cv));
+    cv.P_seq = h->P_seq; cv.maxpp = h->maxpp; cv.B = h->B; cv.L = h->L; cv.H = h->H; cv.d = h->d;
+    cv.row_bytes = h->d * h->elt;
+    cv.swizzle = (cfg->kv_dtype == TRIMKV_DTYPE_BF16 && cv.row_bytes % 128 == 0) ? 1 : 0;
+    cv.pool_bits = h->pool_bits;
+    const size_t pools = (size_t)h->B * LH;
+    const size_t slots = (size_t)h->B * h->slots_seq;
+    trimkv_status s = TRIMKV_OK;
+    auto A = [&](trimkv_status r) { if (s == TRIMKV_OK) s = r; };
+    A(dev_alloc(h, &cv.kv, slots * 2 * cv.row_bytes, true));
+    A(dev_alloc(h, &cv.lam, slots, true));
+    A(dev_alloc(h, &cv.c, slots, true));
+    A(dev_alloc(h, &cv.pos, slots, true));
+    A(dev_alloc(h, &cv.owner, (size_t)h->B * h->P_seq, false));
+    A(dev_alloc(h, &cv.block_table, pools * h->maxpp, true));
+    A(dev_alloc(h, &cv.len, pools, true));
+    A(dev_alloc(h, &cv.free_stack, (size_t)h->B * h->P_seq, false));
+    A(dev_alloc(h, &cv.free_count, (size_t)h->B, false));
+    A(dev_alloc(h, &cv.evict_mask, (size_t)h->B * h->P_seq, true));
+    A(dev_alloc(h, &cv.err, 1, true));
+    SelectBuffers& sb = h->sb;
+    sb.cand_cap = h->n_max;
+    A(dev_alloc(h, &sb.sel, (size_t)h->B, true));
+    A(dev_alloc(h, &sb.hist, (size_t)h->B * NB, true));
+    A(dev_alloc(h, &sb.done, (size_t)h->B, true));
+    A(dev_alloc(h, &sb.cand, (size_t)h->B * sb.cand_cap, false));
+    A(dev_alloc(h, &sb.stats, (size_t)h->B * 4, true));
+    A(dev_alloc(h, &h->hole, (size_t)h->B * h->e_max, false));
+    A(dev_alloc(h, &h->mover, (size_t)h->B * h->e_max, false));
+    A(dev_alloc(h, &h->cursor, (size_t)h->B, true));
+    AttnBuffers& ab = h->ab;
+    const long long tiles_max = (long long)h->B * (h->n_max / 32 + 2 * LH);
+    ab.max_items = std::max<long long>(592LL * 32, tiles_max / 32) + 2 * (long long)pools;
+    A(dev_alloc(h, &ab.item_prefix, pools + 1, true));
+    A(dev_alloc(h, &ab.item_desc, (size_t)ab.max_items, false));
+    A(dev_alloc(h, &ab.part_o, (size_t)ab.max_items * h->g * h->d, false));
+    A(dev_alloc(h, &ab.part_ml, (size_t)ab.max_items * h->g * 2, false));
+    h->rows_max = std::max<long long>((long long)h->B * cfg->max_chunk, (long long)h->L * h->B);
+    A(dev_alloc(h, &h->g_lam, (size_t)h->rows_max * h->H, false));
+    A(dev_alloc(h, &h->g_c, (size_t)h->rows_max * h->H, false));
+    if (h->D > 0) {
+        A(dev_alloc(h, &h->W1, (size_t)h->L * h->dg * h->D, false));
+        A(dev_alloc(h, &h->b1, (size_t)h->L * h->dg, false));
+        A(dev_alloc(h, &h->W2, (size_t)h->L * h->H * h->de * h->dg, false));
+        A(dev_alloc(h, &h->b2, (size_t)h->L * h->H * h->de, false));
+        A(dev_alloc(h, &h->w_g, (size_t)h->de, false));
+        A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg, false));
+    }
+    if (s == TRIMKV_OK) s = init_cache_state(h);
+    if (s != TRIMKV_OK) {
+        char keep[sizeof(g_err)];
+        memcpy(keep, g_err, sizeof(keep));
+        trimkv_destroy(h);
+        memcpy(g_err, keep, sizeof(keep));
+        return s;
+    }
+    *out = h;
+    return TRIMKV_OK;
+}
+
+void trimkv_destroy(trimkv_t* h) {
+    if (!h) return;
+    cudaDeviceSynchronize();
+    for (void* p : h->allocs) cudaFree(p);
+    delete h;
+}
+
+trimkv_status trimkv_reset(trimkv_t* h) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    return init_cache_state(h);
+}
+
+trimkv_status trimkv_set_gate(trimkv_t* h, int layer, const float* W1, const float* b1, const float* W2, const float* b2) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
+    if (layer < 0 || layer >= h->L || !W1 || !b1 || !W2 || !b2) return fail(TRIMKV_E_ARG, "bad layer or NULL weights");
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(h->W1 + (size_t)layer * h->dg * h->D, W1, (size_t)h->dg * h->D * 4, cudaMemcpyDeviceToDevice));
+    CUDA_TRY(cudaMemcpy(h->b1 + (size_t)layer * h->dg, b1, (size_t)h->dg * 4, cudaMemcpyDeviceToDevice));
+    CUDA_TRY(cudaMemcpy(h->W2 + (size_t)layer * h->H * h->de * h->dg, W2, (size_t)h->H * h->de * h->dg * 4, cudaMemcpyDeviceToDevice));
+    CUDA_TRY(cudaMemcpy(h->b2 + (size_t)layer * h->H * h->de, b2, (size_t)h->H * h->de * 4, cudaMemcpyDeviceToDevice));
+    CUDA_TRY(cudaDeviceSynchronize());
+    h->gate_set[layer] = 1;
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_set_shared_projection(trimkv_t* h, const float* w_g, float b_g) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
+    if (!w_g) return fail(TRIMKV_E_ARG, "NULL w_g");
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(h->w_g, w_g, (size_t)h->de * 4, cudaMemcpyDeviceToDevice));
+    CUDA_TRY(cudaDeviceSynchronize());
+    h->b_g = b_g;
+    h->shared_set = true;
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_gate(trimkv_t* h, int layer, int n_new, const float* x, float* beta, float* lambda, float* c,
+                          void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (layer < 0 || layer >= h->L || n_new < 1 || !x || !aligned16(x)) return fail(TRIMKV_E_ARG, "bad layer, n_new or x (x must be 16-byte aligned)");
+    if ((long long)h->B * n_new > h->rows_max) return fail(TRIMKV_E_ARG, "n_new exceeds max_chunk");
+    if (trimkv_status s = gate_ready(h, layer, 1)) return s;
+    launch_gate(gate_params(h), x, h->u, layer, 1, h->B * n_new, beta, lambda, c, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, const float* lambda, const float* c,
+                            const void* k, const void* v, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (layer < 0 || layer >= h->L) return fail(TRIMKV_E_ARG, "layer out of range");
+    if (n_new < 1 || n_new > h->cfg.max_chunk) return fail(TRIMKV_E_ARG, "n_new must be in [1, max_chunk]");
+    if (!k || !v || !aligned16(k) || !aligned16(v)) return fail(TRIMKV_E_ARG, "k and v must be non-NULL and 16-byte aligned");
+    if (!x && !lambda) return fail(TRIMKV_E_ARG, "either x or lambda is required");
+    if (h->tokens[layer] + n_new > h->max_pos) return fail(TRIMKV_E_UNSUPPORTED, "position limit %lld reached", h->max_pos);
+    cudaStream_t st = (cudaStream_t)stream;
+    const float* lam = lambda;
+    const float* cc = c;
+    if (x) {
+        if (!aligned16(x)) return fail(TRIMKV_E_ARG, "x must be 16-byte aligned");
+        if (trimkv_status s = gate_ready(h, layer, 1)) return s;
+        if (h->prof.on) h->prof.mark(PH_GATE, 0, st);
+        launch_gate(gate_params(h), x, h->u, layer, 1, h->B * n_new, nullptr, h->g_lam, h->g_c, st);
+        if (h->prof.on) h->prof.mark(PH_GATE, 1, st);
+        lam = h->g_lam;
+        cc = h->g_c;
+    }
+    if (h->prof.on) h->prof.mark(PH_APPEND, 0, st);
+    launch_append(h->cv, layer, 1, n_new, h->tokens[layer], lam, cc, h->cfg.horizon, k, v, st);
+    if (h->prof.on) h->prof.mark(PH_APPEND, 1, st);
+    CUDA_TRY(cudaGetLastError());
+    h->tokens[layer] += n_new;
+    h->entries += (long long)n_new * h->H;
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_score_and_evict(trimkv_t* h, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    return evict_impl(h, (cudaStream_t)stream);
+}
+
+trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const void* q, void* out, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (layer < 0 || layer >= h->L || !q || !out || !aligned16(q) || !aligned16(out)) return fail(TRIMKV_E_ARG, "bad layer, q or out");
+    return attention_impl(h, layer, 1, q, out, (cudaStream_t)stream);
+}
+
+trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
+                                     const void* q, void* out, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!k || !v || !q || !out || (!x && !lambda)) return fail(TRIMKV_E_ARG, "NULL argument");
+    if (!aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out) || (x && !aligned16(x))) return fail(TRIMKV_E_ARG, "buffers must be 16-byte aligned");
+    const long long t = h->tokens[0];
+    for (int l = 1; l < h->L; ++l)
+        if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layers hold different token counts");
+    if (t + 1 > h->max_pos) return fail(TRIMKV_E_UNSUPPORTED, "position limit %lld reached", h->max_pos);
+    cudaStream_t st = (cudaStream_t)stream;
+    const float* lam = lambda;
+    const float* cc = nullptr;
+    if (x) {
+        if (trimkv_status s = gate_ready(h, 0, h->L)) return s;
+        if (h->prof.on) h->prof.mark(PH_GATE, 0, st);
+        launch_gate(gate_params(h), x, h->u, 0, h->L, h->B, nullptr, h->g_lam, h->g_c, st);
+        if (h->prof.on) h->prof.mark(PH_GATE, 1, st);
+        lam = h->g_lam;
+        cc = h->g_c;
+    }
+    if (h->prof.on) h->prof.mark(PH_APPEND, 0, st);
+    launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, st);
+    if (h->prof.on) h->prof.mark(PH_APPEND, 1, st);
+    for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
+    h->entries += (long long)h->L * h->H;
+    if (trimkv_status s = attention_impl(h, 0, h->L, q, out, st)) return s;
+    return evict_impl(h, st);
+}
+
+trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!out_host) return fail(TRIMKV_E_ARG, "NULL output");
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(out_host, h->cv.len, (size_t)h->B * h->L * h->H * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return device_status(h);
+}
+
+trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap, int* n, int32_t* pos_host,
+                              float* lambda_host, float* c_host, void* k_host, void* v_host) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (seq < 0 || seq >= h->B || layer < 0 || layer >= h->L || head < 0 || head >= h->H || !n || cap < 0)
+        return fail(TRIMKV_E_ARG, "pool index out of range or NULL n");
+    CUDA_TRY(cudaDeviceSynchronize());
+    const long long pool = ((long long)seq * h->L + layer) * h->H + head;
+    int32_t len = 0;
+    CUDA_TRY(cudaMemcpy(&len, h->cv.len + pool, sizeof(len), cudaMemcpyDeviceToHost));
+    *n = len;
+    if (len > cap) return fail(TRIMKV_E_ARG, "pool holds %d entries, capacity %d", len, cap);
+    if (len == 0) return device_status(h);
+    const size_t rb = (size_t)h->d * h->elt;
+    char* tmp = nullptr;
+    const size_t meta = ((size_t)len * 4 + 255) / 256 * 256;
+    const size_t kvb = ((size_t)len * rb + 255) / 256 * 256;
+    CUDA_TRY(cudaMalloc((void**)&tmp, 3 * meta + 2 * kvb));
+    int32_t* dpos = (int32_t*)tmp;
+    float* dlam = (float*)(tmp + meta);
+    float* dc = (float*)(tmp + 2 * meta);
+    char* dk = tmp + 3 * meta;
+    char* dv = dk + kvb;
+    launch_gather_pool(h->cv, seq, layer, head, dpos, dlam, dc, k_host ? dk : nullptr, v_host ? dv : nullptr, len, 0);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess && pos_host) e = cudaMemcpy(pos_host, dpos, (size_t)len * 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && lambda_host) e = cudaMemcpy(lambda_host, dlam, (size_t)len * 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && c_host) e = cudaMemcpy(c_host, dc, (size_t)len * 4, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && k_host) e = cudaMemcpy(k_host, dk, (size_t)len * rb, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && v_host) e = cudaMemcpy(v_host, dv, (size_t)len * rb, cudaMemcpyDeviceToHost);
+    cudaFree(tmp);
+    if (e != cudaSuccess) return fail(TRIMKV_E_CUDA, "get_pool: %s", cudaGetErrorString(e));
+    return device_status(h);
+}
+
+trimkv_status trimkv_get_kept(trimkv_t* h, int seq, int layer, int head, int32_t* pos_out_host, int cap, int* n) {
+    if (!pos_out_host) return fail(TRIMKV_E_ARG, "NULL output");
+    trimkv_status s = trimkv_get_pool(h, seq, layer, head, cap, n, pos_out_host, nullptr, nullptr, nullptr, nullptr);
+    if (s == TRIMKV_OK) std::sort(pos_out_host, pos_out_host + *n);
+    return s;
+}
+
+trimkv_status trimkv_get_select_stats(trimkv_t* h, int64_t* out_host) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!out_host) return fail(TRIMKV_E_ARG, "NULL output");
+    CUDA_TRY(cudaDeviceSynchronize());
+    CUDA_TRY(cudaMemcpy(out_host, h->sb.stats, (size_t)h->B * 4 * sizeof(long long), cudaMemcpyDeviceToHost));
+    return device_status(h);
+}
+
+trimkv_status trimkv_sync_status(trimkv_t* h) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    return device_status(h);
+}
+
+trimkv_status trimkv_profile(trimkv_t* h, int enable) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    h->prof.clear();
+    h->prof.on = enable != 0;
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!ms_host || !count_host) return fail(TRIMKV_E_ARG, "NULL output");
+    CUDA_TRY(cudaDeviceSynchronize());
+    for (int i = 0; i < PH_COUNT; ++i) { ms_host[i] = 0.0; count_host[i] = 0; }
+    for (auto& r : h->prof.recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.second.first, r.second.second) == cudaSuccess) {
+            ms_host[r.first] += ms;
+            count_host[r.first] += 1;
+        }
+    }
+    h->prof.clear();
+    return TRIMKV_OK;
+}
+
+const char* trimkv_last_error(void) { return g_err; }
+
+int64_t trimkv_kernel_launches(void) { return (int64_t)tkv::g_launches.load(std::memory_order_relaxed); }
+
+// ---- standalone selection ---------------------------------------------------------------------------
+static long long select_cand_cap(int64_t n) {
+    long long cap = n / 1024;
+    if (cap < 16384) cap = 16384;
+    return cap;
+}
+static const size_t SEL_HDR = 1024;   // SelState, done counter, stats
+
+size_t trimkv_select_workspace_bytes(int64_t n) {
+    if (n < 0) return 0;
+    return SEL_HDR + (size_t)NB * sizeof(uint32_t) + (size_t)select_cand_cap(n) * sizeof(Cand) + 256;
+}
+
+trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
+                                 size_t workspace_bytes, int32_t* status_out, void* stream) {
+    if (n < 0 || k_keep < 0 || n > 0xFFFFFFFFLL) return fail(TRIMKV_E_ARG, "n must be in [0, 2^32), k_keep >= 0");
+    if (n == 0) return TRIMKV_OK;
+    if (!scores || !keep_bits || !workspace || !aligned16(scores) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return fail(TRIMKV_E_ARG, "NULL or misaligned buffer (scores 16 B, workspace 256 B)");
+    if (workspace_bytes < trimkv_select_workspace_bytes(n)) return fail(TRIMKV_E_ARG, "workspace too small");
+    cudaStream_t st = (cudaStream_t)stream;
+    const long long words = (n + 63) / 64;
+    if (status_out) CUDA_TRY(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
+    const long long k_evict = n - std::min<long long>(k_keep, n);
+    if (k_evict == 0 || k_evict == n) {
+        CUDA_TRY(cudaMemsetAsync(keep_bits, k_evict == 0 ? 0x00 : 0xFF, (size_t)words * 8, st));
+        launch_invert_mask((const u64*)keep_bits, (u64*)keep_bits, n, st);   // 0 -> all kept, 1s -> none kept
+        CUDA_TRY(cudaGetLastError());
+        return TRIMKV_OK;
+    }
+    char* ws = (char*)workspace;
+    SelectBuffers sb;
+    sb.sel = (SelState*)ws;
+    sb.done = (unsigned*)(ws + 256);
+    sb.stats = (long long*)(ws + 512);
+    sb.hist = (uint32_t*)(ws + SEL_HDR);
+    sb.cand = (Cand*)(ws + SEL_HDR + (size_t)NB * sizeof(uint32_t));
+    sb.cand_cap = select_cand_cap(n);
+    CUDA_TRY(cudaMemsetAsync(ws, 0, SEL_HDR + (size_t)NB * sizeof(uint32_t), st));
+    launch_select_state_init(sb.sel, 1, st);
+    launch_select_array(scores, n, k_evict, (u64*)keep_bits, sb, status_out, st);
+    launch_invert_mask((const u64*)keep_bits, (u64*)keep_bits, n, st);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+}  // extern "C"
