@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Decode-step benchmark of the retention-eviction hot path.
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: retention gates for all
+layers, append of the new token's K/V, GQA decode attention over the ragged pools, then score + global
+selection + compaction (trimkv_decode_step_all).  At N = 1 the workload is the Llama-3-8B-shaped decode:
+32 layers, 8 KV / 32 query heads, d 128, hidden 4096, bf16 K/V, batch 8, 32K-token context fed in
+512-token chunks, budget 4096 tokens' worth (1,048,576 entries per sequence).  With N > 1 every rank holds
+its own batch of sequences (independent budgets, no data-path collective): weak scaling.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode tokens/s at fixed global KV budget (step time in ms_per_step, % of HBM peak in roofline)"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(w, entries_per_seq):
+    """Bytes one decode step must move (per rank): every kept K/V row once, the per-entry retention metadata
+    (lambda, c, position: 12 B) twice (histogram pass + filter pass), the gate weights once."""
+    kv = w.batch * entries_per_seq * 2 * w.head_dim * (2 if w.kv_dtype == "bf16" else 4)
+    meta = 2 * w.batch * entries_per_seq * 12
+    gate = w.layers * (w.hidden * w.gate_hidden + w.kv_heads * w.gate_embed * w.gate_hidden + w.gate_hidden
+                       + w.kv_heads * w.gate_embed) * 4
+    return {"kv": kv, "meta": meta, "gate": gate, "total": kv + meta + gate}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.QUERY}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(w, steps, seed=0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: ONE sequence whose cache is at its
+    budget (M_global entries spread evenly over the pools, seeded N(0,1) K/V, seeded retention), running `steps`
+    whole decode steps (gate, append, attention over all pools, score + full sort + eviction).  Returns
+    (seconds per step, threads used, description)."""
+    import numpy as np
+    from oracle import trimkv_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([int(t.get("num_threads", 1)) for t in threadpool_info()] + [1])
+    except Exception:
+        threads = 1
+    r = np.random.default_rng(seed)
+    oc = orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, w.head_dim, w.horizon)
+    per_pool = w.budget_entries // (w.layers * w.kv_heads)
+    t0 = w.context
+    pos = np.arange(t0 - per_pool + 1, t0 + 1, dtype=np.int64)
+    for l in range(w.layers):
+        for h in range(w.kv_heads):
+            lam = (-np.exp(-(w.b_g + 0.05 * r.standard_normal(per_pool)))).astype(np.float32)
+            oc.pos[l][h] = pos.copy()
+            oc.lam[l][h] = lam
+            oc.c[l][h] = orc.horizon_term_from_lambda32(lam, w.horizon)
+            oc.K[l][h] = r.standard_normal((per_pool, w.head_dim))
+            oc.V[l][h] = r.standard_normal((per_pool, w.head_dim))
+        oc.tokens[l] = t0
+    params = []
+    for l in range(w.layers):
+        params.append((r.standard_normal((w.gate_hidden, w.hidden)) * 0.02, np.zeros(w.gate_hidden),
+                       r.standard_normal((w.kv_heads, w.gate_embed, w.gate_hidden)) * 0.02,
+                       np.zeros((w.kv_heads, w.gate_embed))))
+    oc.set_gate(params, r.standard_normal(w.gate_embed) * 0.02, w.b_g)
+    times = []
+    for _ in range(steps):
+        x = r.standard_normal((w.layers, 1, w.hidden))
+        k = r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim))
+        v = r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim))
+        q = r.standard_normal((w.layers, w.q_heads, w.head_dim))
+        a = time.perf_counter()
+        for l in range(w.layers):
+            oc.append(l, k[l], v[l], x=x[l])
+            oc.decode_attention(l, q[l])
+        oc.score_and_evict()
+        times.append(time.perf_counter() - a)
+    desc = (f"1 of {w.batch} sequences at budget ({w.budget_entries} entries), {steps} whole decode steps "
+            f"(gate+append+attention over all {w.layers * w.kv_heads} pools+score+full sort)")
+    return sum(times) / len(times), threads, desc
+
+
+def run_reference(args, w):
+    from paper_2605_09649_b200 import dist_util
+    rank, _, world = dist_util.env_world()
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 8))
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, 1)
+    sec, threads, desc = oracle_sample(w, steps)
+    value = 1.0 / sec                       # one sequence advances one token per oracle step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded N(0,1) hidden states, K/V, random-init gates)",
+        "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
+                   "head_dim": w.head_dim, "hidden": w.hidden, "batch": w.batch, "budget_entries_per_seq": w.budget_entries,
+                   "context": w.context},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------- CUDA arm
+def run_ours(args, w):
+    import torch
+    from paper_2605_09649_b200 import binding, dist_util, workloads
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = dist_util.init("nccl") if int(os.environ.get("WORLD_SIZE", "1")) > 1 else (0, 0, 1)
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    seed = args.seed + 1000 * rank                      # every rank owns different sequences
+    K, W = args.steps, args.warmup
+
+    cache = binding.TrimKV.from_workload(w)
+    per_layer, w_g = workloads.gate_params(w, seed, device=dev)
+    for l, p in enumerate(per_layer):
+        cache.set_gate(l, *p)
+    cache.set_shared_projection(w_g, w.b_g)
+    bank = workloads.ProjectionBank(w, seed, device=dev)
+
+    # ---- untimed: chunked prefill with eviction after every chunk
+    t_setup = time.time()
+    done = 0
+    while done < w.context:
+        n = min(w.chunk, w.context - done)
+        for l in range(w.layers):
+            x = workloads.hidden_states(w, seed, l, done, n, device=dev)
+            _, k, v = workloads.project_qkv(w, bank, l, x)
+            cache.append(l, k, v, x=x)
+        cache.score_and_evict()
+        done += n
+    cache.sync_status()
+    entries = int(cache.lengths()[0].sum())
+    t_setup = time.time() - t_setup
+
+    # ---- per-step inputs, resident in HBM before the timed region
+    def step_inputs(i):
+        xs, ks, vs, qs = [], [], [], []
+        for l in range(w.layers):
+            x = workloads.hidden_states(w, seed, l, w.context + i, 1, device=dev)
+            q, k, v = workloads.project_qkv(w, bank, l, x)
+            xs.append(x[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0]); qs.append(q[:, 0])
+        return [torch.stack(t).contiguous() for t in (xs, ks, vs, qs)]
+
+    n_in = W + K
+    inputs = [step_inputs(i) for i in range(n_in)]
+    out = torch.empty_like(inputs[0][3])
+    torch.cuda.synchronize()
+
+    def step(i):
+        X, Kt, Vt, Q = inputs[i]
+        cache.decode_step_all(Kt, Vt, Q, out, x=X)
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = binding.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(K):
+        step(W + i)
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    launches = binding.kernel_launches() - launches0
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    cache.sync_status()
+    ms_step = dist_util.max_over_ranks(ms_total / K, device=dev)
+    tokens_per_step = dist_util.sum_over_ranks(w.batch, device=dev)
+    value = tokens_per_step / (ms_step * 1e-3)
+
+    # ---- per-phase device time over the same K steps (second pass, CUDA events around each phase on the launch stream)
+    extra = [step_inputs(n_in + i) for i in range(K)]
+    cache.profile(True)
+    for i in range(K):
+        X, Kt, Vt, Q = extra[i]
+        cache.decode_step_all(Kt, Vt, Q, out, x=X)
+    phases = cache.profile_read()
+    cache.profile(False)
+
+    # ---- end to end: host buffers in, host result out, copies inside the timed region
+    host_in = [[t.cpu().pin_memory() for t in step_inputs(n_in + K + i)] for i in range(K)]
+    dev_in = [torch.empty_like(t, device=dev) for t in host_in[0]]
+    host_out = torch.empty_like(out, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host_in[0])
+    d2h = host_out.numel() * host_out.element_size()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    e0.record()
+    for i in range(K):
+        for dst, src in zip(dev_in, host_in[i]):
+            dst.copy_(src, non_blocking=True)
+        cache.decode_step_all(dev_in[1], dev_in[2], dev_in[3], out, x=dev_in[0])
+        host_out.copy_(out, non_blocking=True)
+        torch.cuda.current_stream().synchronize()         # the caller needs the step's result before the next token
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier()
+    e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1) / K, device=dev)
+    e2e_value = tokens_per_step / (e2e_ms * 1e-3)
+    cache.sync_status()
+    lens = cache.lengths()
+    assert int(lens[0].sum()) == min(w.budget_entries, entries), "budget invariant violated"
+
+    if rank != 0:
+        cache.close()
+        return
+    peak, peak_kind = load_peaks()
+    ab = algorithmic_bytes(w, entries + w.layers * w.kv_heads)
+    attn_ms, attn_n = phases["attn_main"]
+    attn_ms_per = attn_ms / max(attn_n, 1)
+    achieved = ab["kv"] / (attn_ms_per * 1e-3) / 1e9 if attn_ms_per > 0 else 0.0
+    step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
+    cpu = None
+    if not args.no_cpu_baseline:
+        sec, threads, desc = oracle_sample(w, 3 if w.budget_entries > 100000 else 8)
+        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "f32",
+        "data": "synthetic (seeded N(0,1) hidden states; K/V/Q from random-init projections; random-init gates)",
+        "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
+                   "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
+                   "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk,
+                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g,
+                   "parallelism": f"sequences sharded over {world} rank(s), no collective",
+                   "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1)},
+        "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": ab["kv"], "avg_launch_ms": attn_ms_per,
+                     "step": {"algorithmic_bytes": ab, "achieved_gbs": step_gbs, "frac_of_peak": step_gbs / peak,
+                              "frac_of_8tbs_nominal": step_gbs / 8000.0},
+                     "phase_ms_per_step": {k: v[0] / K for k, v in phases.items()}},
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    cache.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=32)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_32k")
+    ap.add_argument("--context", type=int, default=None, help="override the prompt length (development only)")
+    ap.add_argument("--b-g", type=float, default=None, help="override the shared gate bias")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2605_09649_b200 import workloads
+    w = workloads.WORKLOADS[args.workload]
+    if args.context is not None:
+        w = w.replace(context=args.context)
+    if args.b_g is not None:
+        w = w.replace(b_g=args.b_g)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
