@@ -180,6 +180,27 @@ TRIMKV_API size_t trimkv_select_workspace_bytes(int64_t n);
 TRIMKV_API trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
                                  size_t workspace_bytes, int32_t* status_out, void* stream);
 
+/* ---- the same selection for callers that cannot allocate ------------------------------------
+ * (No counterpart in the paper: this entry point exists for the sake of the caller's environment.)
+ * Some users of this library run where device allocation is off limits at call time: inside a
+ * serving loop whose memory was carved up at start-up, under an allocator they do not control, or in
+ * a host framework that forbids cudaMalloc after initialisation.  They cannot size and provide the
+ * workspace that trimkv_select_topk wants.  This variant does the identical selection (same result,
+ * bit for bit) with its scratch memory in an array built into the library image, and itself calls no
+ * cudaMalloc, cudaFree or any other allocating routine.  The caller still passes scores, keep_bits
+ * and status_out (device memory, as for trimkv_select_topk).
+ *   - Limit: n <= TRIMKV_SELECT_STATIC_MAX_N scores; a larger n is refused with
+ *     TRIMKV_E_UNSUPPORTED and a message in trimkv_last_error.  The array takes about 274 KB of
+ *     device memory on every GPU that loads the library, until the process exits.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the last call left in it; each call
+ *     clears, on `stream`, the part that must start at zero.  Two calls whose GPU work may overlap
+ *     (different streams, or different threads or handles on one device) race on it: serialise them. */
+#define TRIMKV_SELECT_STATIC_MAX_N (1 << 24)
+TRIMKV_API trimkv_status trimkv_select_topk_static(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits,
+                                        int32_t* status_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

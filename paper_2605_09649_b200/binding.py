@@ -24,7 +24,7 @@ EXPORTS = [
     "trimkv_set_shared_projection", "trimkv_gate", "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention",
     "trimkv_decode_step_all", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
-    "trimkv_select_topk",
+    "trimkv_select_topk", "trimkv_select_topk_static",
 ]
 
 
@@ -85,10 +85,12 @@ def lib() -> C.CDLL:
     L.trimkv_select_workspace_bytes.argtypes = [i64]
     L.trimkv_select_workspace_bytes.restype = C.c_size_t
     L.trimkv_select_topk.argtypes = [vp, i64, i64, vp, vp, C.c_size_t, vp, vp]
+    L.trimkv_select_topk_static.argtypes = [vp, i64, i64, vp, vp, vp]
     for name in ("trimkv_create_ex", "trimkv_reset", "trimkv_set_gate", "trimkv_set_shared_projection", "trimkv_gate",
                  "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention", "trimkv_decode_step_all",
                  "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
-                 "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_select_topk"):
+                 "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_select_topk",
+                 "trimkv_select_topk_static"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -274,4 +276,19 @@ def select_topk(scores: torch.Tensor, k_keep: int, keep_bits: Optional[torch.Ten
         status = torch.zeros(1, dtype=torch.int32, device=scores.device)
     _check(lib().trimkv_select_topk(_ptr(scores, torch.float32), n, k_keep, _ptr(keep_bits), _ptr(workspace),
                                     workspace.numel(), _ptr(status), _stream()))
+    return keep_bits, status
+
+
+SELECT_STATIC_MAX_N = 1 << 24
+
+
+def select_topk_static(scores: torch.Tensor, k_keep: int, keep_bits: torch.Tensor, status: torch.Tensor):
+    """trimkv_select_topk_static: the same selection, for callers that cannot allocate device memory when
+    they call (a serving loop with a fixed memory plan, a framework that bans cudaMalloc after start-up).
+    The scratch lives inside the library; the caller passes every buffer: keep_bits (int64 words,
+    ceil(n / 64) of them) and status (int32[1]).  At most SELECT_STATIC_MAX_N scores.  Calls share the
+    scratch, so do not let two of them overlap on the GPU."""
+    n = scores.numel()
+    _check(lib().trimkv_select_topk_static(_ptr(scores, torch.float32), n, k_keep, _ptr(keep_bits), _ptr(status),
+                                           _stream()))
     return keep_bits, status

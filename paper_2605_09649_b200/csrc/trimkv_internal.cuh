@@ -174,4 +174,7 @@ void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32
 
 void count_launch(int n = 1);
 
+// Sets the calling thread's message returned by trimkv_last_error (printf format).
+void set_last_error(const char* fmt, ...);
+
 }  // namespace tkv

@@ -44,6 +44,15 @@ int ceil_log2(long long v) {
 
 }  // namespace
 
+namespace tkv {
+void set_last_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+}  // namespace tkv
+
 struct Profiler : public tkv::PhaseMarker {
     bool on = false;
     std::vector<cudaEvent_t> pool;                 // reusable events
