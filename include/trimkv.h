@@ -72,7 +72,8 @@ typedef struct trimkv_config {
     int32_t horizon;        /* lookahead T - t (Sec. 5.1: 2); 0 = infinite horizon             */
     int32_t kv_dtype;       /* TRIMKV_DTYPE_BF16 or TRIMKV_DTYPE_F32 (K, V, q and out)         */
     int32_t max_chunk;      /* largest n_new of one append (1 for pure decode)                 */
-    int32_t reserved;       /* set to 0                                                        */
+    int32_t reserved;       /* 0; bit 0 = testing aid: distrust the selection's key sample, so that the
+                               exact single-CTA redo of the selection runs in every eviction round  */
     int64_t max_pool_pages; /* cap on pages of one (layer, head) pool; 0 = a pool may take all */
 } trimkv_config;
 
@@ -148,7 +149,8 @@ TRIMKV_API trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int he
                               float* lambda_host, float* c_host, void* k_host, void* v_host);
 
 /* Per-sequence figures of the last selection, int64 [B, 4] to host:
- * {histogram passes used, candidates resolved exactly, entries evicted, bin shift}.  Synchronises. */
+ * {1 if the exact redo ran (the sampled candidate range missed) else 0, candidates ranked exactly,
+ *  entries evicted, keys sampled}.  Synchronises. */
 TRIMKV_API trimkv_status trimkv_get_select_stats(trimkv_t* h, int64_t* out_host);
 
 /* Waits for the handle's enqueued work (device synchronise) and returns the latched device error,

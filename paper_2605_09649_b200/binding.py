@@ -130,7 +130,7 @@ class TrimKV:
 
     def __init__(self, budget_entries: int, layers: int, kv_heads: int, head_dim: int, *, q_heads: Optional[int] = None,
                  hidden: int = 0, batch: int = 1, gate_hidden: int = 512, gate_embed: int = 64, horizon: int = 2,
-                 kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0):
+                 kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0, distrust_sample: bool = False):
         L = lib()
         cfg = Config()
         L.trimkv_default_config(C.byref(cfg), budget_entries, layers, kv_heads, head_dim)
@@ -143,6 +143,7 @@ class TrimKV:
         cfg.kv_dtype = {"bf16": DTYPE_BF16, "f32": DTYPE_F32}[kv_dtype]
         cfg.max_chunk = max_chunk
         cfg.max_pool_pages = max_pool_pages
+        cfg.reserved = 1 if distrust_sample else 0     # testing aid: forces the selection's exact redo path
         self.cfg = cfg
         self.torch_dtype = torch.bfloat16 if kv_dtype == "bf16" else torch.float32
         self.B, self.L, self.H, self.Hq, self.d, self.D = batch, layers, kv_heads, cfg.q_heads, head_dim, hidden

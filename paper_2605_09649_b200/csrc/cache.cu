@@ -41,7 +41,6 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
                 for (int j = 0; j < need; ++j) {
                     const int page = stack[prev - 1 - j];
                     bt[p_old + j] = page;
-                    cv.owner[(size_t)b * cv.P_seq + page] = make_int2(pool_local, (int)(p_old + j));
                 }
             }
         }
@@ -80,8 +79,12 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
         cv.c[slot] = cc;
         cv.pos[slot] = (int32_t)(pos0 + j + 1);
     }
+    // page records of every page that received entries: owner pool, logical index, live entries
+    const int n2 = old + n_new;
+    for (int lp = old / PAGE + threadIdx.x; lp * PAGE < n2; lp += blockDim.x)
+        cv.owner[(size_t)b * cv.P_seq + bt[lp]] = make_int4(pool_local, lp, min(PAGE, n2 - lp * PAGE), 0);
     __syncthreads();
-    if (threadIdx.x == 0) cv.len[pool] = old + n_new;
+    if (threadIdx.x == 0) cv.len[pool] = n2;
 }
 
 __device__ __forceinline__ u64 bits_below(int n) {   // mask with the lowest n bits set, n in [0, 64]
@@ -219,8 +222,10 @@ compact_kernel(CacheView cv, int32_t* __restrict__ hole, int32_t* __restrict__ m
     for (int j = threadIdx.x; j < nfree; j += blockDim.x) {
         const int page = bt[np2 + j];
         cv.free_stack[(size_t)b * cv.P_seq + s_freebase + j] = page;
-        cv.owner[(size_t)b * cv.P_seq + page] = make_int2(-1, 0);
+        cv.owner[(size_t)b * cv.P_seq + page] = make_int4(-1, 0, 0, 0);
     }
+    if (threadIdx.x == 0 && np2 > 0)     // the new last page is the only kept page whose fill changed
+        cv.owner[(size_t)b * cv.P_seq + bt[np2 - 1]] = make_int4((int)(pool % ((long long)cv.L * cv.H)), np2 - 1, n2 - (np2 - 1) * PAGE, 0);
 }
 
 // Copies one pool's entries, in storage order, to dense device buffers (undoing the chunk permutation).

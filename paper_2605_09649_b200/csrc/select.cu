@@ -21,12 +21,11 @@ struct CacheSrc {
     CacheView cv;
     long long t1;   // t + 1
     __device__ long long pages() const { return cv.P_seq; }
-    // returns the valid-entry bits (4) of this lane; sets owned = page holds live entries
-    __device__ unsigned load4(int b, long long p, int e0, u64 (&key)[4], bool& owned) const {
-        const int2 ow = cv.owner[(size_t)b * cv.P_seq + p];
-        owned = ow.x >= 0;
-        if (!owned) return 0u;
-        const int fill = cv.len[(size_t)b * cv.L * cv.H + ow.x] - ow.y * PAGE;
+    // {pool, logical page, live entries, -}; pool < 0: the page is free
+    __device__ int4 info(int b, long long p) const { return __ldg(cv.owner + (size_t)b * cv.P_seq + p); }
+    // returns the valid-entry bits (4) of this lane
+    __device__ unsigned load4(int b, long long p, int e0, const int4& inf, u64 (&key)[4]) const {
+        if (inf.x < 0 || e0 >= inf.z) return 0u;
         const size_t s = ((size_t)b * cv.P_seq + p) * PAGE + e0;
         const float4 lm = *reinterpret_cast<const float4*>(cv.lam + s);
         const float4 cc = *reinterpret_cast<const float4*>(cv.c + s);
@@ -37,11 +36,11 @@ struct CacheSrc {
         unsigned vm = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (e0 + j < fill) {
+            if (e0 + j < inf.z) {
                 const float age = (float)(t1 - (long long)p4[j]);
                 const float S = retention_score(l4[j], c4[j], age);
                 if (S != S) latch_error(cv.err, TRIMKV_E_NONFINITE);
-                const uint32_t tie = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)ow.x;
+                const uint32_t tie = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)inf.x;
                 key[j] = make_key(S, tie);
                 vm |= 1u << j;
             }
@@ -55,8 +54,8 @@ struct ArraySrc {
     long long n;
     int32_t* err;
     __device__ long long pages() const { return (n + PAGE - 1) / PAGE; }
-    __device__ unsigned load4(int, long long p, int e0, u64 (&key)[4], bool& owned) const {
-        owned = true;
+    __device__ int4 info(int, long long) const { return make_int4(0, 0, PAGE, 0); }
+    __device__ unsigned load4(int, long long p, int e0, const int4&, u64 (&key)[4]) const {
         const long long i0 = p * PAGE + e0;
         float v[4];
         unsigned vm = 0;
@@ -189,32 +188,47 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
     unsigned under = 0;
     int cur_bin = -1;
     unsigned cur_cnt = 0;
-    for (long long pp = p0 + warp * 2; pp < p1; pp += (blockDim.x >> 5) * 2) {
-        const long long page = pp + sub;
-        if (page < p1) {
-            u64 key[4];
-            bool owned;
-            const unsigned vm = src.load4(b, page, e0, key, owned);
+    auto tally = [&](const u64 (&key)[4], unsigned vm) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (vm & (1u << j)) {
-                    kmin = key[j] < kmin ? key[j] : kmin;
-                    kmax = key[j] > kmax ? key[j] : kmax;
-                    const int bin = bin_of(key[j], lo, shift);
-                    if (bin == 0) {
-                        ++under;
-                    } else if (bin < NB - 1) {
-                        if (bin == cur_bin) {
-                            ++cur_cnt;
-                        } else {
-                            if (cur_cnt) atomicAdd(&sh[cur_bin], cur_cnt);
-                            cur_bin = bin;
-                            cur_cnt = 1;
-                        }
+        for (int j = 0; j < 4; ++j) {
+            if (vm & (1u << j)) {
+                kmin = key[j] < kmin ? key[j] : kmin;
+                kmax = key[j] > kmax ? key[j] : kmax;
+                const int bin = bin_of(key[j], lo, shift);
+                if (bin == 0) {
+                    ++under;
+                } else if (bin < NB - 1) {
+                    if (bin == cur_bin) {
+                        ++cur_cnt;
+                    } else {
+                        if (cur_cnt) atomicAdd(&sh[cur_bin], cur_cnt);
+                        cur_bin = bin;
+                        cur_cnt = 1;
                     }
                 }
             }
         }
+    };
+    // Each half-warp takes two pages per trip; the page records of the next trip are fetched one trip ahead,
+    // so the metadata loads of a trip depend on nothing that is still in flight.
+    const long long stride = (long long)(blockDim.x >> 5) * 4;
+    long long pp = p0 + warp * 4;
+    int4 infA = make_int4(-1, 0, 0, 0), infB = infA;
+    if (pp + sub < p1) infA = src.info(b, pp + sub);
+    if (pp + 2 + sub < p1) infB = src.info(b, pp + 2 + sub);
+    for (; pp < p1; pp += stride) {
+        const long long pgA = pp + sub, pgB = pp + 2 + sub, nx = pp + stride;
+        int4 nA = make_int4(-1, 0, 0, 0), nB = nA;
+        if (nx + sub < p1) nA = src.info(b, nx + sub);
+        if (nx + 2 + sub < p1) nB = src.info(b, nx + 2 + sub);
+        u64 keyA[4], keyB[4];
+        unsigned vmA = 0, vmB = 0;
+        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, keyA);
+        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, keyB);
+        tally(keyA, vmA);
+        tally(keyB, vmB);
+        infA = nA;
+        infB = nB;
     }
     if (cur_cnt) atomicAdd(&sh[cur_bin], cur_cnt);
 #pragma unroll
@@ -261,12 +275,15 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
 }
 
 // ------------------------------------------------------------------ filter: evict masks + candidates
-template <class Src>
+// COUNT_BELOW: also count the keys below the candidate range into st->n_below (the sample-bracket path, where
+// that count is not known beforehand).
+template <class Src, bool COUNT_BELOW>
 __global__ void __launch_bounds__(256)
 filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap,
               u64* __restrict__ evict_mask, long long mask_stride, int32_t* err) {
     const int b = blockIdx.y;
     SelState* st = sel + b;
+    unsigned below = 0;
     const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane >> 4, l16 = lane & 15, e0 = l16 * 4;
@@ -276,12 +293,7 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
     const long long p1 = min(P, p0 + chunk);
     Cand* cb = cand + (size_t)b * cand_cap;
 
-    for (long long pp = p0 + warp * 2; pp < p1; pp += (blockDim.x >> 5) * 2) {   // warp-uniform trip count
-        const long long page = pp + sub;
-        u64 key[4];
-        bool owned = false;
-        unsigned vm = 0;
-        if (page < p1) vm = src.load4(b, page, e0, key, owned);
+    auto emit = [&](long long page, const int4& inf, const u64 (&key)[4], unsigned vm) {   // called by all lanes
         unsigned ev = 0, cd = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -290,16 +302,18 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
                 else if (key[j] <= c_hi) cd |= 1u << j;
             }
         }
+        if (COUNT_BELOW) below += __popc(ev);
         // candidates: warp-aggregated append
-        const int nc = __popc(cd);
-        int incl = nc;
+        const unsigned any = __ballot_sync(0xffffffffu, cd != 0u);
+        if (any) {
+            const int nc = __popc(cd);
+            int incl = nc;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        const int tot = __shfl_sync(0xffffffffu, incl, 31);
-        if (tot > 0) {
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const int tot = __shfl_sync(0xffffffffu, incl, 31);
             unsigned base = 0;
             if (lane == 0) base = atomicAdd(&st->cand_count, (unsigned)tot);
             base = __shfl_sync(0xffffffffu, base, 0);
@@ -327,89 +341,369 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
             wlo |= __shfl_xor_sync(0xffffffffu, wlo, o);
             whi |= __shfl_xor_sync(0xffffffffu, whi, o);
         }
-        if (l16 == 0 && page < p1 && owned) evict_mask[(size_t)b * mask_stride + page] = ((u64)whi << 32) | (u64)wlo;
+        if (l16 == 0 && page < p1 && inf.x >= 0) evict_mask[(size_t)b * mask_stride + page] = ((u64)whi << 32) | (u64)wlo;
+    };
+    // Pages are visited from the end of the CTA's range backwards: the histogram pass went forwards, so the
+    // most recently read metadata (the likeliest to still sit in L2) comes first.  Warp-uniform trip count.
+    const long long stride = (long long)(blockDim.x >> 5) * 4;
+    long long pp = p0 + warp * 4;
+    const long long span = p1 - p0;
+    auto page_of = [&](long long q) { return p0 + (span - 1 - (q - p0)); };   // reversed index
+    int4 infA = make_int4(-1, 0, 0, 0), infB = infA;
+    if (pp + sub < p1) infA = src.info(b, page_of(pp + sub));
+    if (pp + 2 + sub < p1) infB = src.info(b, page_of(pp + 2 + sub));
+    for (; pp < p1; pp += stride) {
+        const long long qA = pp + sub, qB = pp + 2 + sub, nx = pp + stride;
+        int4 nA = make_int4(-1, 0, 0, 0), nB = nA;
+        if (nx + sub < p1) nA = src.info(b, page_of(nx + sub));
+        if (nx + 2 + sub < p1) nB = src.info(b, page_of(nx + 2 + sub));
+        const long long pgA = qA < p1 ? page_of(qA) : p1, pgB = qB < p1 ? page_of(qB) : p1;
+        u64 keyA[4], keyB[4];
+        unsigned vmA = 0, vmB = 0;
+        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, keyA);
+        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, keyB);
+        emit(pgA, infA, keyA, vmA);
+        emit(pgB, infB, keyB, vmB);
+        infA = nA;
+        infB = nB;
+    }
+    if (COUNT_BELOW) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
+        if (lane == 0 && below) atomicAdd(reinterpret_cast<unsigned long long*>(&st->n_below), (unsigned long long)below);
+    }
+}
+
+
+
+// ------------------------------------------------------------------ sample bracket (cache path)
+// One full pass suffices when a candidate range that surely holds the k-th smallest key is known beforehand.
+// A Bernoulli sample of the sequence's keys (a hash of the slot decides, about SAMPLE_MEAN keys) is sorted by one
+// CTA; the sample keys at ranks k*p -+ a margin of several standard deviations bound the range.  The filter pass
+// then counts the keys below the range, and the exact ranking verifies that the k-th key lay inside; if it did
+// not (probability below 1e-9 per call), a single-CTA exact selection redoes the sequence.
+constexpr int SAMPLE_CAP = 4096;
+constexpr int SAMPLE_MEAN = 3072;
+
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: spreads slot indices over 32 bits
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
+// One thread per page: samples each live slot with probability thresh / 2^32.
+__global__ void __launch_bounds__(256)
+sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, uint32_t thresh, uint32_t seed) {
+    const int b = blockIdx.y;
+    const long long page = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (page >= src.cv.P_seq) return;
+    const int4 inf = src.info(b, page);
+    if (inf.x < 0) return;
+    SelState* st = sel + b;
+    const CacheView& cv = src.cv;
+    const uint32_t base = (uint32_t)(page * PAGE) * 0x9E3779B1u + seed + (uint32_t)b * 0x85EBCA77u;
+    for (int off = 0; off < inf.z; ++off) {
+        if (thresh != 0xffffffffu && mix32(base + (uint32_t)off * 0x9E3779B1u) >= thresh) continue;
+        const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
+        const int pos = cv.pos[s];
+        const float S = retention_score(cv.lam[s], cv.c[s], (float)(src.t1 - (long long)pos));
+        const uint32_t tie = ((uint32_t)pos << cv.pool_bits) | (uint32_t)inf.x;
+        const unsigned w = atomicAdd(&st->sample_count, 1u);
+        if (w < SAMPLE_CAP) sample[(size_t)b * SAMPLE_CAP + w] = make_key(S, tie);
+    }
+}
+
+// One CTA per sequence: sorts the sample and sets the candidate range [cand_lo, cand_hi].
+__global__ void __launch_bounds__(1024)
+bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long long k_evict, long long n_total,
+               int distrust) {
+    __shared__ u64 sk[SAMPLE_CAP];
+    const int b = blockIdx.x;
+    SelState* st = sel + b;
+    const unsigned raw = st->sample_count;
+    const int ns = (int)min(raw, (unsigned)SAMPLE_CAP);
+    int n2 = 2;
+    while (n2 < ns) n2 <<= 1;
+    for (int i = threadIdx.x; i < n2; i += blockDim.x) sk[i] = i < ns ? sample[(size_t)b * SAMPLE_CAP + i] : ~0ull;
+    __syncthreads();
+    for (int k2 = 2; k2 <= n2; k2 <<= 1) {
+        for (int j = k2 >> 1; j > 0; j >>= 1) {
+            for (int p = threadIdx.x; p < (n2 >> 1); p += blockDim.x) {
+                const int i = 2 * p - (p & (j - 1));          // lower index of the p-th compare-exchange pair
+                const int q = i + j;
+                const bool asc = (i & k2) == 0;
+                const u64 a = sk[i], c = sk[q];
+                if ((a > c) == asc) { sk[i] = c; sk[q] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        u64 lo = 0ull, hi = ~0ull;
+        if (ns > 0 && !distrust) {
+            long long r_lo, r_hi;
+            if ((long long)raw == n_total) {          // every key was sampled: the k-th smallest is known exactly
+                r_lo = r_hi = k_evict;
+            } else {
+                const double mu = (double)k_evict * (double)ns / (double)n_total;   // expected sample rank of the k-th key
+                const double dev = 7.0 * sqrt(mu) + 8.0;
+                r_lo = (long long)floor(mu - dev);
+                r_hi = (long long)ceil(mu + dev) + 1;
+            }
+            if (r_lo >= 1) lo = sk[min(r_lo, (long long)ns) - 1];
+            if (r_hi <= ns) hi = sk[max(r_hi, 1LL) - 1];
+        } else if (distrust) {
+            lo = hi = ~0ull;    // test hook: a range that cannot hold the k-th key, so that the exact redo runs
+        }
+        st->cand_lo = lo;
+        st->cand_hi = hi;
+        st->n_below = 0;
+        st->cand_count = 0;
+        st->cand_expected = 0;
+        st->resolved = 0;
+        st->passes = ns;
     }
 }
 
 // ------------------------------------------------------------------ exact ranking of the candidates
+// One CTA per sequence.  STRICT (histogram path): the candidate range is known to hold the k-th key; any
+// inconsistency is an internal error.  Otherwise (sample-bracket path): an inconsistent count means the range
+// missed; resolved stays 0 and the exact redo kernel takes over.
+template <bool STRICT>
 __global__ void __launch_bounds__(1024)
 resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap, u64* __restrict__ evict_mask,
-               long long mask_stride, long long k_evict, unsigned cand_target, long long* __restrict__ stats,
+               long long mask_stride, long long k_evict, unsigned next_aim, long long* __restrict__ stats,
                int32_t* __restrict__ cursor, int32_t* err) {
-    __shared__ unsigned hist[256];
+    constexpr int DB = 11, NBIN = 1 << DB;
+    __shared__ unsigned hist[NBIN];
+    __shared__ unsigned wtot[32];
+    __shared__ u64 s_or[32], s_and[32];
     __shared__ u64 s_prefix;
     __shared__ long long s_r;
-    const int b = blockIdx.x;
+    __shared__ int s_found;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     SelState* st = sel + b;
     const Cand* cb = cand + (size_t)b * cand_cap;
-    const long long C = min((long long)st->cand_count, cand_cap);
+    const long long craw = (long long)st->cand_count;
+    const long long C = min(craw, cand_cap);
     long long r = k_evict - st->n_below;
-    const u64 lo = st->cand_lo, hi = st->cand_hi;
-    if (r < 0 || r > C || (long long)st->cand_expected != (long long)st->cand_count) {
-        if (threadIdx.x == 0) latch_error(err, TRIMKV_E_STATE);
-        r = r < 0 ? 0 : (r > C ? C : r);
+    const bool ok = r >= 0 && r <= C && craw <= cand_cap && (!STRICT || (long long)st->cand_expected == craw);
+    const int sample_n = st->passes;
+    if (!ok) {
+        if (STRICT) {
+            if (tid == 0) latch_error(err, TRIMKV_E_STATE);
+            r = r < 0 ? 0 : (r > C ? C : r);
+        } else {
+            if (tid == 0) {
+                st->resolved = 0;
+                st->sample_count = 0;
+                if (stats) { stats[b * 4 + 0] = 1; stats[b * 4 + 1] = C; stats[b * 4 + 2] = k_evict; stats[b * 4 + 3] = sample_n; }
+                if (cursor) cursor[b] = 0;
+            }
+            return;
+        }
     }
-    u64 tau = lo;
+    u64 tau = 0ull;
     if (r > 0) {
-        int top = (lo == hi) ? 0 : 64 - __clzll((long long)(lo ^ hi));   // number of low bits that differ
-        u64 prefix = top >= 64 ? 0ull : (lo >> top);
+        // bits in which the candidate keys differ
+        u64 vor = 0ull, vand = ~0ull;
+        for (long long i = tid; i < C; i += blockDim.x) {
+            const u64 key = cb[i].key;
+            vor |= key;
+            vand &= key;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            vor |= __shfl_xor_sync(0xffffffffu, vor, o);
+            vand &= __shfl_xor_sync(0xffffffffu, vand, o);
+        }
+        if (lane == 0) { s_or[warp] = vor; s_and[warp] = vand; }
+        __syncthreads();
+        vor = 0ull; vand = ~0ull;
+        for (int w = 0; w < 32; ++w) { vor |= s_or[w]; vand &= s_and[w]; }
+        const u64 diff = vor ^ vand;
+        int top = diff ? 64 - __clzll((long long)diff) : 0;    // number of low bits that differ
+        u64 prefix = top >= 64 ? 0ull : (vor >> top);
         while (top > 0) {
-            const int dbits = top < 8 ? top : 8;
+            const int dbits = top < DB ? top : DB;
             const int sh = top - dbits;
-            for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0u;
+            hist[tid] = 0u;
+            hist[tid + 1024] = 0u;
+            if (tid == 0) s_found = 0;
             __syncthreads();
-            for (long long i = threadIdx.x; i < C; i += blockDim.x) {
+            for (long long i = tid; i < C; i += blockDim.x) {
                 const u64 key = cb[i].key;
                 const bool match = top >= 64 ? true : ((key >> top) == prefix);
                 if (match) atomicAdd(&hist[(unsigned)((key >> sh) & ((1u << dbits) - 1u))], 1u);
             }
             __syncthreads();
-            if (threadIdx.x == 0) {
-                long long cum = 0, rr = r;
-                unsigned dv = 0;
-                for (unsigned q = 0; q < (1u << dbits); ++q) {
-                    if (rr <= cum + (long long)hist[q]) { dv = q; rr -= cum; break; }
-                    cum += hist[q];
-                }
-                s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)dv;
-                s_r = rr;
+            const unsigned h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+            unsigned incl = h0 + h1;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) wtot[warp] = incl;
+            __syncthreads();
+            unsigned off = 0;
+            for (int w = 0; w < warp; ++w) off += wtot[w];
+            const long long excl = (long long)off + incl - (h0 + h1);
+            if (r > excl && r <= excl + h0) {
+                s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid);
+                s_r = r - excl;
+                s_found = 1;
+            } else if (r > excl + h0 && r <= excl + h0 + h1) {
+                s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid + 1);
+                s_r = r - excl - h0;
+                s_found = 1;
             }
             __syncthreads();
+            if (!s_found) {                          // cannot happen with consistent counts
+                if (tid == 0) latch_error(err, TRIMKV_E_STATE);
+                break;
+            }
             prefix = s_prefix;
             r = s_r;
             top = sh;
+            __syncthreads();
         }
         tau = prefix;   // the r-th smallest candidate key: everything <= tau is evicted
-        for (long long i = threadIdx.x; i < C; i += blockDim.x) {
+        for (long long i = tid; i < C; i += blockDim.x) {
             const Cand cnd = cb[i];
             if (cnd.key <= tau)
                 atomicOr(evict_mask + (size_t)b * mask_stride + (cnd.slot >> 6), 1ull << (cnd.slot & 63));
         }
+    } else {
+        tau = st->cand_lo;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (tid == 0) {
         if (stats) {
-            stats[b * 4 + 0] = st->passes;
+            stats[b * 4 + 0] = STRICT ? st->passes : 0;
             stats[b * 4 + 1] = C;
             stats[b * 4 + 2] = k_evict;
-            stats[b * 4 + 3] = st->shift;
+            stats[b * 4 + 3] = STRICT ? st->shift : sample_n;
         }
-        // centre the next call's first histogram on this threshold; aim for ~cand_target/8 candidates
-        int shift = st->shift;
-        const int want = 31 - __clz((int)max(cand_target / 8u, 1u));
-        const int have = 31 - __clz((int)max((unsigned)min(C, 0x7fffffffLL), 1u));
-        shift += want - have;
-        shift = shift < 0 ? 0 : (shift > INIT_SHIFT ? INIT_SHIFT : shift);
-        const u64 half = (u64)(REG_BINS / 2) << shift;
-        st->lo = tau > half ? tau - half : 0ull;
-        st->shift = shift;
-        st->resolved = 0;
-        st->passes = 0;
+        if (STRICT) {
+            // centre the next call's first histogram on this threshold; aim for ~next_aim candidates
+            int shift = st->shift;
+            const int want = 31 - __clz((int)max(next_aim, 1u));
+            const int have = 31 - __clz((int)max((unsigned)min(C, 0x7fffffffLL), 1u));
+            shift += want - have;
+            shift = shift < 0 ? 0 : (shift > INIT_SHIFT ? INIT_SHIFT : shift);
+            const u64 half = (u64)(REG_BINS / 2) << shift;
+            st->lo = tau > half ? tau - half : 0ull;
+            st->shift = shift;
+            st->resolved = 0;
+            st->passes = 0;
+        } else {
+            st->resolved = 1;
+        }
         st->cand_count = 0;
+        st->sample_count = 0;
         st->kmin = ~0ull;
         st->kmax = 0ull;
         if (cursor) cursor[b] = 0;
     }
+}
+
+// Exact redo for a sequence whose sample bracket missed: one CTA radix-selects the k-th smallest key over all of
+// the sequence's entries (DB bits per sweep) and rewrites every eviction mask.  Slow and rare.
+__global__ void __launch_bounds__(1024)
+redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_mask, long long mask_stride,
+            long long k_evict, int32_t* err) {
+    constexpr int DB = 11, NBIN = 1 << DB;
+    __shared__ unsigned hist[NBIN];
+    __shared__ unsigned wtot[32];
+    __shared__ u64 s_prefix;
+    __shared__ long long s_r;
+    __shared__ int s_found;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    SelState* st = sel + b;
+    if (st->resolved) return;
+    const int sub = lane >> 4, l16 = lane & 15, e0 = l16 * 4;
+    const long long P = src.pages();
+    u64 prefix = 0ull;
+    long long r = k_evict;
+    int top = 64;
+    while (top > 0) {
+        const int dbits = top < DB ? top : DB;
+        const int sh = top - dbits;
+        hist[tid] = 0u;
+        hist[tid + 1024] = 0u;
+        if (tid == 0) s_found = 0;
+        __syncthreads();
+        for (long long pp = warp * 2; pp < P; pp += 64) {
+            const long long page = pp + sub;
+            if (page < P) {
+                const int4 inf = src.info(b, page);
+                u64 key[4];
+                const unsigned vm = src.load4(b, page, e0, inf, key);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (vm & (1u << j)) {
+                        const bool match = top >= 64 ? true : ((key[j] >> top) == prefix);
+                        if (match) atomicAdd(&hist[(unsigned)((key[j] >> sh) & ((1u << dbits) - 1u))], 1u);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        const unsigned h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+        unsigned incl = h0 + h1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) wtot[warp] = incl;
+        __syncthreads();
+        unsigned off = 0;
+        for (int w = 0; w < warp; ++w) off += wtot[w];
+        const long long excl = (long long)off + incl - (h0 + h1);
+        if (r > excl && r <= excl + h0) {
+            s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid);
+            s_r = r - excl;
+            s_found = 1;
+        } else if (r > excl + h0 && r <= excl + h0 + h1) {
+            s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid + 1);
+            s_r = r - excl - h0;
+            s_found = 1;
+        }
+        __syncthreads();
+        if (!s_found) {
+            if (tid == 0) latch_error(err, TRIMKV_E_STATE);
+            return;
+        }
+        prefix = s_prefix;
+        r = s_r;
+        top = sh;
+        __syncthreads();
+    }
+    const u64 tau = prefix;
+    for (long long pp = warp * 2; pp < P; pp += 64) {          // warp-uniform trip count
+        const long long page = pp + sub;
+        int4 inf = make_int4(-1, 0, 0, 0);
+        u64 key[4];
+        unsigned vm = 0;
+        if (page < P) {
+            inf = src.info(b, page);
+            vm = src.load4(b, page, e0, inf, key);
+        }
+        unsigned ev = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if ((vm & (1u << j)) && key[j] <= tau) ev |= 1u << j;
+        const unsigned nib = ev << (4 * (l16 & 7));
+        unsigned wlo = (l16 < 8) ? nib : 0u, whi = (l16 >= 8) ? nib : 0u;
+#pragma unroll
+        for (int o = 1; o < 16; o <<= 1) {
+            wlo |= __shfl_xor_sync(0xffffffffu, wlo, o);
+            whi |= __shfl_xor_sync(0xffffffffu, whi, o);
+        }
+        if (l16 == 0 && page < P && inf.x >= 0) evict_mask[(size_t)b * mask_stride + page] = ((u64)whi << 32) | (u64)wlo;
+    }
+    if (tid == 0) st->resolved = 1;
 }
 
 __global__ void state_init_kernel(SelState* sel, int B) {
@@ -417,7 +711,7 @@ __global__ void state_init_kernel(SelState* sel, int B) {
     if (b >= B) return;
     SelState s;
     s.lo = 0ull; s.kmin = ~0ull; s.kmax = 0ull; s.cand_lo = 0ull; s.cand_hi = 0ull; s.n_below = 0;
-    s.shift = INIT_SHIFT; s.resolved = 0; s.passes = 0; s.cand_count = 0; s.cand_expected = 0; s.pad = 0;
+    s.shift = INIT_SHIFT; s.resolved = 0; s.passes = 0; s.cand_count = 0; s.cand_expected = 0; s.sample_count = 0;
     sel[b] = s;
 }
 
@@ -447,9 +741,9 @@ void run_select(const Src& src, long long pages, int B, const SelectBuffers& sb,
     for (int p = 0; p < max_passes; ++p)
         hist_kernel<Src><<<grid, 256, 0, st>>>(src, sb.sel, sb.hist, sb.done, k_evict, n_total, p == max_passes - 1,
                                                cand_target);
-    filter_kernel<Src><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, err);
-    resolve_kernel<<<B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, k_evict, cand_target,
-                                       sb.stats, cursor, err);
+    filter_kernel<Src, false><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, err);
+    resolve_kernel<true><<<B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, k_evict,
+                                             max(cand_target / 8u, 1u), sb.stats, cursor, err);
     count_launch(max_passes + 2);
 }
 
@@ -461,12 +755,22 @@ void launch_select_state_init(SelState* sel, int B, cudaStream_t st) {
 }
 
 void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
-                         long long k_evict, int32_t* compact_cursor, cudaStream_t st) {
+                         long long k_evict, int32_t* compact_cursor, int distrust_sample, cudaStream_t st) {
     CacheSrc src;
     src.cv = cv;
     src.t1 = t + 1;
-    run_select(src, cv.P_seq, cv.B, sb, n_total, k_evict, MAX_HIST_PASSES, 16384u, cv.evict_mask, cv.P_seq,
-               compact_cursor, cv.err, st);
+    uint32_t thresh = 0xffffffffu;                       // sample every key
+    if (n_total > SAMPLE_MEAN) thresh = (uint32_t)(4294967296.0 * (double)SAMPLE_MEAN / (double)n_total);
+    const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u;
+    dim3 gs((unsigned)((cv.P_seq + 255) / 256), cv.B);
+    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, thresh, seed);
+    bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample);
+    dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
+    filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
+    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
+                                                 sb.stats, compact_cursor, cv.err);
+    redo_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, cv.evict_mask, cv.P_seq, k_evict, cv.err);
+    count_launch(5);
 }
 
 void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,

@@ -30,10 +30,10 @@ struct SelState {
     long long n_below; // number of keys < cand_lo
     int shift;         // bin width = 2^shift keys
     int resolved;      // 1 once the candidate range is final for this call
-    int passes;        // histogram passes run in this call
+    int passes;        // histogram passes run in this call (sample-bracket path: keys sampled)
     unsigned int cand_count;   // candidates appended by the filter pass
     unsigned int cand_expected;
-    int pad;
+    unsigned int sample_count; // keys drawn by the sampling pass of this call
 };
 
 struct Cand {          // one candidate of the exact resolution stage
@@ -86,7 +86,7 @@ struct CacheView {
     float* lam;
     float* c;
     int32_t* pos;
-    int2* owner;           // [B][P_seq] {pool_local or -1, logical page index}
+    int4* owner;           // [B][P_seq] {pool_local or -1, logical page index, live entries in the page, 0}
     int32_t* block_table;  // [B*L*H][maxpp]
     int32_t* len;          // [B*L*H]
     int32_t* free_stack;   // [B][P_seq]
@@ -119,9 +119,14 @@ struct GateParams {
     const float* W2;  // [L][H][de][dg]
     const float* b2;  // [L][H][de]
     const float* w_g; // [de]
+    const float* v;   // [L][H][dg]  second layer folded with the shared readout: W2^T w_g
+    const float* s0;  // [L][H]      w_g . b2 + b_g
     float b_g;
     int D, dg, de, H, horizon;
 };
+
+// Recomputes v and s0 of layers [layer0, layer0 + nlayers) from W2, b2, w_g, b_g.
+void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, float* s0, cudaStream_t st);
 
 // rows_per_layer rows of x per layer, layers [layer0, layer0 + nlayers).
 void launch_gate(const GateParams& gp, const float* x, float* u_scratch, int layer0, int nlayers, int rows_per_layer,
@@ -137,11 +142,12 @@ struct SelectBuffers {
     Cand* cand;           // [B][cand_cap]
     long long cand_cap;
     long long* stats;     // [B][4]
+    u64* sample;          // [B][4096] sampled keys (cache path)
 };
 
 // compact_cursor [B]: zeroed by the selection for the compaction that follows.
 void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, long long k_evict,
-                         int32_t* compact_cursor, cudaStream_t st);
+                         int32_t* compact_cursor, int distrust_sample, cudaStream_t st);
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max, cudaStream_t st);
 
 void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,

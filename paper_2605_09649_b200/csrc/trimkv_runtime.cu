@@ -90,7 +90,7 @@ struct trimkv {
     SelectBuffers sb;
     AttnBuffers ab;
     int32_t *hole, *mover, *cursor;
-    float *W1, *b1, *W2, *b2, *w_g, *u, *g_lam, *g_c;
+    float *W1, *b1, *W2, *b2, *w_g, *gv, *gs0, *u, *g_lam, *g_c;
     float b_g;
     bool shared_set;
     std::vector<char> gate_set;
@@ -128,8 +128,8 @@ trimkv_status init_cache_state(trimkv* h) {
     CUDA_TRY(cudaMemcpy(h->cv.free_stack, stack.data(), stack.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
     std::vector<int32_t> cnt(h->B, (int32_t)h->P_seq);
     CUDA_TRY(cudaMemcpy(h->cv.free_count, cnt.data(), cnt.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
-    std::vector<int2> own((size_t)h->B * h->P_seq, make_int2(-1, 0));
-    CUDA_TRY(cudaMemcpy(h->cv.owner, own.data(), own.size() * sizeof(int2), cudaMemcpyHostToDevice));
+    std::vector<int4> own((size_t)h->B * h->P_seq, make_int4(-1, 0, 0, 0));
+    CUDA_TRY(cudaMemcpy(h->cv.owner, own.data(), own.size() * sizeof(int4), cudaMemcpyHostToDevice));
     CUDA_TRY(cudaMemset(h->cv.len, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->cv.err, 0, sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->sb.hist, 0, (size_t)h->B * NB * sizeof(uint32_t)));
@@ -156,7 +156,7 @@ trimkv_status device_status(trimkv* h) {
 
 GateParams gate_params(const trimkv* h) {
     GateParams gp;
-    gp.W1 = h->W1; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.b_g = h->b_g;
+    gp.W1 = h->W1; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.v = h->gv; gp.s0 = h->gs0; gp.b_g = h->b_g;
     gp.D = h->D; gp.dg = h->dg; gp.de = h->de; gp.H = h->H; gp.horizon = h->cfg.horizon;
     return gp;
 }
@@ -177,7 +177,7 @@ trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
     if (k <= 0) return TRIMKV_OK;
     PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
     if (pm) pm->mark(PH_SELECT, 0, st);
-    launch_select_cache(h->cv, h->sb, t, h->entries, k, h->cursor, st);
+    launch_select_cache(h->cv, h->sb, t, h->entries, k, h->cursor, h->cfg.reserved & 1, st);
     if (pm) { pm->mark(PH_SELECT, 1, st); pm->mark(PH_COMPACT, 0, st); }
     launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
     if (pm) pm->mark(PH_COMPACT, 1, st);
@@ -239,6 +239,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     if (cfg->horizon < 0 || cfg->horizon > 64) return fail(TRIMKV_E_ARG, "horizon must be in [0, 64]");
     if (cfg->hidden < 0 || (cfg->hidden > 0 && (cfg->hidden % 4 || cfg->gate_hidden < 4 || cfg->gate_hidden % 4 || cfg->gate_embed < 1)))
         return fail(TRIMKV_E_ARG, "hidden and gate_hidden must be multiples of 4, gate_embed positive");
+    if (cfg->hidden > 0 && cfg->gate_hidden > 1536) return fail(TRIMKV_E_UNSUPPORTED, "gate_hidden must be at most 1536");
     if ((long long)cfg->layers * cfg->kv_heads > 65536) return fail(TRIMKV_E_UNSUPPORTED, "layers * kv_heads too large");
 
     trimkv* h = new (std::nothrow) trimkv();
@@ -261,7 +262,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     h->shared_set = false;
     h->b_g = 0.f;
     h->entries = 0;
-    h->W1 = h->b1 = h->W2 = h->b2 = h->w_g = h->u = h->g_lam = h->g_c = nullptr;
+    h->W1 = h->b1 = h->W2 = h->b2 = h->w_g = h->gv = h->gs0 = h->u = h->g_lam = h->g_c = nullptr;
 
     CacheView& cv = h->cv;
     memset(&cv, 0, sizeof(cv));
@@ -291,6 +292,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     A(dev_alloc(h, &sb.done, (size_t)h->B, true));
     A(dev_alloc(h, &sb.cand, (size_t)h->B * sb.cand_cap, false));
     A(dev_alloc(h, &sb.stats, (size_t)h->B * 4, true));
+    A(dev_alloc(h, &sb.sample, (size_t)h->B * 4096, false));
     A(dev_alloc(h, &h->hole, (size_t)h->B * h->e_max, false));
     A(dev_alloc(h, &h->mover, (size_t)h->B * h->e_max, false));
     A(dev_alloc(h, &h->cursor, (size_t)h->B, true));
@@ -310,6 +312,8 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         A(dev_alloc(h, &h->W2, (size_t)h->L * h->H * h->de * h->dg, false));
         A(dev_alloc(h, &h->b2, (size_t)h->L * h->H * h->de, false));
         A(dev_alloc(h, &h->w_g, (size_t)h->de, false));
+        A(dev_alloc(h, &h->gv, (size_t)h->L * h->H * h->dg, false));
+        A(dev_alloc(h, &h->gs0, (size_t)h->L * h->H, false));
         A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg, false));
     }
     if (s == TRIMKV_OK) s = init_cache_state(h);
@@ -346,8 +350,9 @@ trimkv_status trimkv_set_gate(trimkv_t* h, int layer, const float* W1, const flo
     CUDA_TRY(cudaMemcpy(h->b1 + (size_t)layer * h->dg, b1, (size_t)h->dg * 4, cudaMemcpyDeviceToDevice));
     CUDA_TRY(cudaMemcpy(h->W2 + (size_t)layer * h->H * h->de * h->dg, W2, (size_t)h->H * h->de * h->dg * 4, cudaMemcpyDeviceToDevice));
     CUDA_TRY(cudaMemcpy(h->b2 + (size_t)layer * h->H * h->de, b2, (size_t)h->H * h->de * 4, cudaMemcpyDeviceToDevice));
-    CUDA_TRY(cudaDeviceSynchronize());
     h->gate_set[layer] = 1;
+    if (h->shared_set) launch_gate_fold(gate_params(h), layer, 1, h->gv, h->gs0, 0);
+    CUDA_TRY(cudaDeviceSynchronize());
     return TRIMKV_OK;
 }
 
@@ -357,9 +362,11 @@ trimkv_status trimkv_set_shared_projection(trimkv_t* h, const float* w_g, float 
     if (!w_g) return fail(TRIMKV_E_ARG, "NULL w_g");
     CUDA_TRY(cudaDeviceSynchronize());
     CUDA_TRY(cudaMemcpy(h->w_g, w_g, (size_t)h->de * 4, cudaMemcpyDeviceToDevice));
-    CUDA_TRY(cudaDeviceSynchronize());
     h->b_g = b_g;
     h->shared_set = true;
+    for (int l = 0; l < h->L; ++l)
+        if (h->gate_set[l]) launch_gate_fold(gate_params(h), l, 1, h->gv, h->gs0, 0);
+    CUDA_TRY(cudaDeviceSynchronize());
     return TRIMKV_OK;
 }
 
@@ -572,6 +579,7 @@ trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep,
     sb.hist = (uint32_t*)(ws + SEL_HDR);
     sb.cand = (Cand*)(ws + SEL_HDR + (size_t)NB * sizeof(uint32_t));
     sb.cand_cap = select_cand_cap(n);
+    sb.sample = nullptr;
     CUDA_TRY(cudaMemsetAsync(ws, 0, SEL_HDR + (size_t)NB * sizeof(uint32_t), st));
     launch_select_state_init(sb.sel, 1, st);
     launch_select_array(scores, n, k_evict, (u64*)keep_bits, sb, status_out, st);
