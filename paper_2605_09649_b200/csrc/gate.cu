@@ -15,7 +15,7 @@ namespace tkv {
 
 namespace {
 
-constexpr int GH_WARPS = 8;    // warps per CTA of the hidden-layer kernel; they split the input dimension
+constexpr int GH_WARPS = 4;    // warps per CTA of the hidden-layer kernel; they split the input dimension
 constexpr int GH_JW = 4;       // hidden units per CTA
 constexpr int GH_RW = 8;       // rows per CTA
 constexpr int GH_UNROLL = 4;   // 128-float slices of the input dimension in flight per warp
@@ -24,6 +24,23 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// Sums 32 per-lane values over the warp with 31 shuffles: afterwards lane i holds the warp total of v[i].
+__device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int s = 16, n = 32; s >= 1; s >>= 1, n >>= 1) {
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if (i < n / 2) {
+                const float send = upper ? v[i] : v[i + n / 2];
+                const float keep = upper ? v[i + n / 2] : v[i];
+                v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+            }
+        }
+    }
+    return v[0];
 }
 
 __device__ __forceinline__ float4 ld_stream(const float* p) {   // read-once data: do not keep it in L1
@@ -54,7 +71,7 @@ gate_fold_kernel(const float* __restrict__ W2, const float* __restrict__ b2, con
 
 // u[lb][r][j] = SiLU(x[lb][r][:] . W1[layer][j][:] + b1[layer][j]) for GH_RW rows and GH_JW hidden units per CTA.
 // grid = (row tiles, hidden-unit groups, layers): CTAs that share a slice of W1 are neighbours in launch order.
-__global__ void __launch_bounds__(GH_WARPS * 32, 2)
+__global__ void __launch_bounds__(GH_WARPS * 32, 4)
 gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, const float* __restrict__ b1,
                    float* __restrict__ u, int layer0, int R, int D, int dg) {
     __shared__ float red[GH_WARPS][GH_RW * GH_JW];
@@ -68,11 +85,9 @@ gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, co
     const float* Wb = W1 + ((size_t)layer * dg + j0) * D;
     const float* xb = x + ((size_t)lb * R + r0) * D;
 
-    float acc[GH_RW][GH_JW];
+    float acc[GH_RW * GH_JW];                     // [row][hidden unit]
 #pragma unroll
-    for (int a = 0; a < GH_RW; ++a)
-#pragma unroll
-        for (int b = 0; b < GH_JW; ++b) acc[a][b] = 0.f;
+    for (int a = 0; a < GH_RW * GH_JW; ++a) acc[a] = 0.f;
 
     const int nslice = (D + 127) / 128;
     for (int c0 = warp; c0 < nslice; c0 += GH_WARPS * GH_UNROLL) {
@@ -89,28 +104,29 @@ gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, co
             const int d0 = (c0 + un * GH_WARPS) * 128 + lane * 4;
             if (d0 < D) {
 #pragma unroll
-                for (int rr = 0; rr < GH_RW; ++rr) {
-                    if (rr < nr) {
-                        const float4 xv = __ldg(reinterpret_cast<const float4*>(xb + (size_t)rr * D + d0));
+                for (int rh = 0; rh < GH_RW; rh += 4) {          // rows in batches of four: loads first, then the FMAs
+                    float4 xv[4];
+#pragma unroll
+                    for (int r4 = 0; r4 < 4; ++r4)
+                        xv[r4] = (rh + r4 < nr) ? __ldg(reinterpret_cast<const float4*>(xb + (size_t)(rh + r4) * D + d0))
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int r4 = 0; r4 < 4; ++r4)
 #pragma unroll
                         for (int jj = 0; jj < GH_JW; ++jj) {
-                            acc[rr][jj] = fmaf(xv.x, w[un][jj].x, acc[rr][jj]);
-                            acc[rr][jj] = fmaf(xv.y, w[un][jj].y, acc[rr][jj]);
-                            acc[rr][jj] = fmaf(xv.z, w[un][jj].z, acc[rr][jj]);
-                            acc[rr][jj] = fmaf(xv.w, w[un][jj].w, acc[rr][jj]);
+                            float a = acc[(rh + r4) * GH_JW + jj];
+                            a = fmaf(xv[r4].x, w[un][jj].x, a);
+                            a = fmaf(xv[r4].y, w[un][jj].y, a);
+                            a = fmaf(xv[r4].z, w[un][jj].z, a);
+                            a = fmaf(xv[r4].w, w[un][jj].w, a);
+                            acc[(rh + r4) * GH_JW + jj] = a;
                         }
-                    }
                 }
             }
         }
     }
-#pragma unroll
-    for (int rr = 0; rr < GH_RW; ++rr)
-#pragma unroll
-        for (int jj = 0; jj < GH_JW; ++jj) {
-            const float s = warp_sum(acc[rr][jj]);
-            if (lane == 0) red[warp][rr * GH_JW + jj] = s;
-        }
+    static_assert(GH_RW * GH_JW == 32, "the warp reduction below sums exactly 32 values");
+    red[warp][lane] = warp_transpose_sum32(acc, lane);   // lane = row * GH_JW + hidden unit
     __syncthreads();
     if (threadIdx.x < GH_RW * GH_JW) {
         const int rr = threadIdx.x / GH_JW, jj = threadIdx.x % GH_JW;

@@ -390,9 +390,13 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: 
     return x;
 }
 
-// One thread per page: samples each live slot with probability thresh / 2^32.
+// One thread per page.  mode 0: every live slot is sampled (small sequences).  mode 1: every slot with probability
+// thresh / 2^32, decided per slot.  mode 2 (large sequences, 64 * p <= 1): at most one slot per page, the page being
+// chosen with probability 64 * p and the slot uniformly; slots beyond the page's fill are simply not sampled, so each
+// live slot still has probability p.
 __global__ void __launch_bounds__(256)
-sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, uint32_t thresh, uint32_t seed) {
+sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, int mode, uint32_t thresh,
+              uint32_t seed) {
     const int b = blockIdx.y;
     const long long page = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (page >= src.cv.P_seq) return;
@@ -401,59 +405,133 @@ sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample
     SelState* st = sel + b;
     const CacheView& cv = src.cv;
     const uint32_t base = (uint32_t)(page * PAGE) * 0x9E3779B1u + seed + (uint32_t)b * 0x85EBCA77u;
-    for (int off = 0; off < inf.z; ++off) {
-        if (thresh != 0xffffffffu && mix32(base + (uint32_t)off * 0x9E3779B1u) >= thresh) continue;
+    auto take = [&](int off) {
         const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
         const int pos = cv.pos[s];
         const float S = retention_score(cv.lam[s], cv.c[s], (float)(src.t1 - (long long)pos));
         const uint32_t tie = ((uint32_t)pos << cv.pool_bits) | (uint32_t)inf.x;
         const unsigned w = atomicAdd(&st->sample_count, 1u);
         if (w < SAMPLE_CAP) sample[(size_t)b * SAMPLE_CAP + w] = make_key(S, tie);
+    };
+    if (mode == 2) {
+        if (mix32(base) < thresh) {                         // thresh = 64 * p * 2^32
+            const int off = (int)(mix32(base ^ 0x68E31DA4u) & (PAGE - 1));
+            if (off < inf.z) take(off);
+        }
+    } else {
+        for (int off = 0; off < inf.z; ++off)
+            if (mode == 0 || mix32(base + (uint32_t)off * 0x9E3779B1u) < thresh) take(off);
     }
 }
 
-// One CTA per sequence: sorts the sample and sets the candidate range [cand_lo, cand_hi].
+// One CTA per sequence: ranks the sample by radix descent (each thread keeps its sample keys in registers) and
+// sets the candidate range [cand_lo, cand_hi].  The descent stops early once the bin that holds the wanted rank is
+// nearly empty and then takes the bin's outer edge, which only widens the range.
 __global__ void __launch_bounds__(1024)
 bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long long k_evict, long long n_total,
                int distrust) {
-    __shared__ u64 sk[SAMPLE_CAP];
-    const int b = blockIdx.x;
+    constexpr int DB = 11, NBIN = 1 << DB, PER = SAMPLE_CAP / 1024;
+    __shared__ unsigned hist[NBIN];
+    __shared__ unsigned wtot[32];
+    __shared__ u64 s_or[32], s_and[32];
+    __shared__ u64 s_prefix;
+    __shared__ long long s_r;
+    __shared__ unsigned s_cnt;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     SelState* st = sel + b;
     const unsigned raw = st->sample_count;
     const int ns = (int)min(raw, (unsigned)SAMPLE_CAP);
-    int n2 = 2;
-    while (n2 < ns) n2 <<= 1;
-    for (int i = threadIdx.x; i < n2; i += blockDim.x) sk[i] = i < ns ? sample[(size_t)b * SAMPLE_CAP + i] : ~0ull;
+    u64 key[PER];
+    u64 vor = 0ull, vand = ~0ull;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int idx = tid + i * 1024;
+        key[i] = idx < ns ? sample[(size_t)b * SAMPLE_CAP + idx] : ~0ull;
+        if (idx < ns) { vor |= key[i]; vand &= key[i]; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        vor |= __shfl_xor_sync(0xffffffffu, vor, o);
+        vand &= __shfl_xor_sync(0xffffffffu, vand, o);
+    }
+    if (lane == 0) { s_or[warp] = vor; s_and[warp] = vand; }
     __syncthreads();
-    for (int k2 = 2; k2 <= n2; k2 <<= 1) {
-        for (int j = k2 >> 1; j > 0; j >>= 1) {
-            for (int p = threadIdx.x; p < (n2 >> 1); p += blockDim.x) {
-                const int i = 2 * p - (p & (j - 1));          // lower index of the p-th compare-exchange pair
-                const int q = i + j;
-                const bool asc = (i & k2) == 0;
-                const u64 a = sk[i], c = sk[q];
-                if ((a > c) == asc) { sk[i] = c; sk[q] = a; }
+    vor = 0ull; vand = ~0ull;
+    for (int w = 0; w < 32; ++w) { vor |= s_or[w]; vand &= s_and[w]; }
+    const u64 diff = vor ^ vand;
+    const int top0 = (ns > 0 && diff) ? 64 - __clzll((long long)diff) : 0;   // low bits in which the sample keys differ
+
+    // Key bound for sample rank r (1-based, 1 <= r <= ns): the lower (upper = false) or upper edge of the finest
+    // bin the descent reaches; exact when the descent runs to the last bit.
+    auto bound_of_rank = [&](long long r, bool upper) -> u64 {
+        int top = top0;
+        u64 prefix = top >= 64 ? 0ull : (vor >> top);
+        while (top > 0) {
+            const int dbits = top < DB ? top : DB;
+            const int sh = top - dbits;
+            hist[tid] = 0u;
+            hist[tid + 1024] = 0u;
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                const bool live = tid + i * 1024 < ns;
+                const bool match = live && (top >= 64 ? true : ((key[i] >> top) == prefix));
+                if (match) atomicAdd(&hist[(unsigned)((key[i] >> sh) & ((1u << dbits) - 1u))], 1u);
             }
             __syncthreads();
-        }
-    }
-    if (threadIdx.x == 0) {
-        u64 lo = 0ull, hi = ~0ull;
-        if (ns > 0 && !distrust) {
-            long long r_lo, r_hi;
-            if ((long long)raw == n_total) {          // every key was sampled: the k-th smallest is known exactly
-                r_lo = r_hi = k_evict;
-            } else {
-                const double mu = (double)k_evict * (double)ns / (double)n_total;   // expected sample rank of the k-th key
-                const double dev = 7.0 * sqrt(mu) + 8.0;
-                r_lo = (long long)floor(mu - dev);
-                r_hi = (long long)ceil(mu + dev) + 1;
+            const unsigned h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+            unsigned incl = h0 + h1;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
             }
-            if (r_lo >= 1) lo = sk[min(r_lo, (long long)ns) - 1];
-            if (r_hi <= ns) hi = sk[max(r_hi, 1LL) - 1];
-        } else if (distrust) {
-            lo = hi = ~0ull;    // test hook: a range that cannot hold the k-th key, so that the exact redo runs
+            if (lane == 31) wtot[warp] = incl;
+            __syncthreads();
+            unsigned off = 0;
+            for (int w = 0; w < warp; ++w) off += wtot[w];
+            const long long excl = (long long)off + incl - (h0 + h1);
+            if (r > excl && r <= excl + h0) {
+                s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid);
+                s_r = r - excl;
+                s_cnt = h0;
+            } else if (r > excl + h0 && r <= excl + h0 + h1) {
+                s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid + 1);
+                s_r = r - excl - h0;
+                s_cnt = h1;
+            }
+            __syncthreads();
+            prefix = s_prefix;
+            r = s_r;
+            top = sh;
+            const unsigned cnt = s_cnt;
+            __syncthreads();
+            if (cnt <= 2u) break;
         }
+        if (top == 0) return prefix;
+        return upper ? ((prefix << top) | ((1ull << top) - 1ull)) : (prefix << top);
+    };
+
+    u64 lo = 0ull, hi = ~0ull;
+    if (ns > 0 && !distrust) {
+        long long r_lo, r_hi;
+        bool exact = false;
+        if ((long long)raw == n_total) {              // every key was sampled: the k-th smallest is known exactly
+            r_lo = r_hi = k_evict;
+            exact = true;
+        } else {
+            const double mu = (double)k_evict * (double)ns / (double)n_total;   // expected sample rank of the k-th key
+            const double dev = 7.0 * sqrt(mu) + 8.0;
+            r_lo = (long long)floor(mu - dev);
+            r_hi = (long long)ceil(mu + dev) + 1;
+        }
+        if (r_lo >= 1) lo = bound_of_rank(min(r_lo, (long long)ns), false);
+        if (r_hi <= ns) hi = bound_of_rank(max(r_hi, 1LL), true);
+        (void)exact;
+    } else if (distrust) {
+        lo = hi = ~0ull;        // test hook: a range that cannot hold the k-th key, so that the exact redo runs
+    }
+    if (tid == 0) {
         st->cand_lo = lo;
         st->cand_hi = hi;
         st->n_below = 0;
@@ -759,11 +837,16 @@ void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long
     CacheSrc src;
     src.cv = cv;
     src.t1 = t + 1;
-    uint32_t thresh = 0xffffffffu;                       // sample every key
-    if (n_total > SAMPLE_MEAN) thresh = (uint32_t)(4294967296.0 * (double)SAMPLE_MEAN / (double)n_total);
+    int mode = 0;                                        // sample every key
+    uint32_t thresh = 0xffffffffu;
+    if (n_total > SAMPLE_MEAN) {
+        const double p = (double)SAMPLE_MEAN / (double)n_total;
+        if (p * PAGE <= 0.5) { mode = 2; thresh = (uint32_t)(4294967296.0 * p * PAGE); }
+        else { mode = 1; thresh = (uint32_t)(4294967296.0 * p); }
+    }
     const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u;
     dim3 gs((unsigned)((cv.P_seq + 255) / 256), cv.B);
-    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, thresh, seed);
+    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, mode, thresh, seed);
     bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample);
     dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
     filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
