@@ -15,10 +15,11 @@ namespace tkv {
 
 namespace {
 
-constexpr int GH_WARPS = 4;    // warps per CTA of the hidden-layer kernel; they split the input dimension
-constexpr int GH_JW = 4;       // hidden units per CTA
+constexpr int GH_WARPS = 8;    // warps per CTA of the hidden-layer kernel
+constexpr int GH_DC = 512;     // floats of the input dimension per CTA (its x tile lives in shared memory)
 constexpr int GH_RW = 8;       // rows per CTA
-constexpr int GH_UNROLL = 4;   // 128-float slices of the input dimension in flight per warp
+constexpr int GH_JP = 2;       // hidden units per warp pass
+constexpr int GH_JSPLIT = 4;   // CTAs that share the hidden units of one (layer, input chunk)
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -26,13 +27,15 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Sums 32 per-lane values over the warp with 31 shuffles: afterwards lane i holds the warp total of v[i].
-__device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane) {
+// Sums 16 per-lane values over the warp with 20 shuffles: afterwards lanes 0..15 hold the warp totals of v[0..15].
+__device__ __forceinline__ float warp_transpose_sum16(float (&v)[16], int lane) {
 #pragma unroll
-    for (int s = 16, n = 32; s >= 1; s >>= 1, n >>= 1) {
+    for (int i = 0; i < 16; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], 16);   // fold the two half-warps
+#pragma unroll
+    for (int s = 8, n = 16; s >= 1; s >>= 1, n >>= 1) {
         const bool upper = (lane & s) != 0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
             if (i < n / 2) {
                 const float send = upper ? v[i] : v[i + n / 2];
                 const float keep = upper ? v[i + n / 2] : v[i];
@@ -69,73 +72,69 @@ gate_fold_kernel(const float* __restrict__ W2, const float* __restrict__ b2, con
     }
 }
 
-// u[lb][r][j] = SiLU(x[lb][r][:] . W1[layer][j][:] + b1[layer][j]) for GH_RW rows and GH_JW hidden units per CTA.
-// grid = (row tiles, hidden-unit groups, layers): CTAs that share a slice of W1 are neighbours in launch order.
-__global__ void __launch_bounds__(GH_WARPS * 32, 4)
-gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, const float* __restrict__ b1,
-                   float* __restrict__ u, int layer0, int R, int D, int dg) {
-    __shared__ float red[GH_WARPS][GH_RW * GH_JW];
+// Partial pre-activations: zpart[lb][chunk][r][j] = x[lb][r][chunk] . W1[layer][j][chunk] for GH_RW rows, one
+// GH_DC-float chunk of the input dimension and a quarter of the hidden units per CTA.  The x tile is staged in
+// shared memory once and W1 is streamed past it, two hidden units per warp pass with eight 16-byte loads in flight
+// per lane.  grid = (row tiles * chunks, GH_JSPLIT, layers): CTAs that share a slice of W1 are neighbours in launch
+// order (chunked-prefill calls re-read W1 from L2).
+__global__ void __launch_bounds__(GH_WARPS * 32, 2)
+gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, float* __restrict__ zpart, int layer0,
+                   int R, int D, int dg, int nchunk) {
+    __shared__ __align__(16) float xs[GH_RW][GH_DC];
     const int lb = blockIdx.z;
     const int layer = layer0 + lb;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int j0 = blockIdx.y * GH_JW;
-    const int r0 = blockIdx.x * GH_RW;
-    const int nj = min(GH_JW, dg - j0);
+    const int chunk = blockIdx.x % nchunk;
+    const int r0 = (blockIdx.x / nchunk) * GH_RW;
     const int nr = min(GH_RW, R - r0);
-    const float* Wb = W1 + ((size_t)layer * dg + j0) * D;
-    const float* xb = x + ((size_t)lb * R + r0) * D;
+    const int dbase = chunk * GH_DC;
+    const int jper = (dg + GH_JSPLIT - 1) / GH_JSPLIT;
+    const int jbeg = blockIdx.y * jper, jend = min(dg, jbeg + jper);
 
-    float acc[GH_RW * GH_JW];                     // [row][hidden unit]
-#pragma unroll
-    for (int a = 0; a < GH_RW * GH_JW; ++a) acc[a] = 0.f;
+    for (int i = threadIdx.x; i < GH_RW * (GH_DC / 4); i += blockDim.x) {
+        const int rr = i / (GH_DC / 4), dd = (i % (GH_DC / 4)) * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (rr < nr && dbase + dd < D) v = __ldg(reinterpret_cast<const float4*>(x + ((size_t)lb * R + r0 + rr) * D + dbase + dd));
+        *reinterpret_cast<float4*>(&xs[rr][dd]) = v;
+    }
+    __syncthreads();
 
-    const int nslice = (D + 127) / 128;
-    for (int c0 = warp; c0 < nslice; c0 += GH_WARPS * GH_UNROLL) {
-        float4 w[GH_UNROLL][GH_JW];
+    const float* Wl = W1 + (size_t)layer * dg * D + dbase;
+    float* zp = zpart + (((size_t)lb * nchunk + chunk) * R + r0) * dg;
+    for (int j0 = jbeg + warp * GH_JP; j0 < jend; j0 += GH_WARPS * GH_JP) {
+        float4 w[GH_JP][GH_DC / 128];
 #pragma unroll
-        for (int un = 0; un < GH_UNROLL; ++un) {
-            const int d0 = (c0 + un * GH_WARPS) * 128 + lane * 4;
+        for (int jj = 0; jj < GH_JP; ++jj)
 #pragma unroll
-            for (int jj = 0; jj < GH_JW; ++jj)
-                w[un][jj] = (d0 < D && jj < nj) ? ld_stream(Wb + (size_t)jj * D + d0) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+            for (int sl = 0; sl < GH_DC / 128; ++sl) {
+                const int dd = sl * 128 + lane * 4;
+                w[jj][sl] = (j0 + jj < jend && dbase + dd < D) ? ld_stream(Wl + (size_t)(j0 + jj) * D + dd)
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        float acc[GH_JP * GH_RW];
 #pragma unroll
-        for (int un = 0; un < GH_UNROLL; ++un) {
-            const int d0 = (c0 + un * GH_WARPS) * 128 + lane * 4;
-            if (d0 < D) {
+        for (int a = 0; a < GH_JP * GH_RW; ++a) acc[a] = 0.f;
 #pragma unroll
-                for (int rh = 0; rh < GH_RW; rh += 4) {          // rows in batches of four: loads first, then the FMAs
-                    float4 xv[4];
+        for (int sl = 0; sl < GH_DC / 128; ++sl) {
 #pragma unroll
-                    for (int r4 = 0; r4 < 4; ++r4)
-                        xv[r4] = (rh + r4 < nr) ? __ldg(reinterpret_cast<const float4*>(xb + (size_t)(rh + r4) * D + d0))
-                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int rr = 0; rr < GH_RW; ++rr) {
+                const float4 xv = *reinterpret_cast<const float4*>(&xs[rr][sl * 128 + lane * 4]);
 #pragma unroll
-                    for (int r4 = 0; r4 < 4; ++r4)
-#pragma unroll
-                        for (int jj = 0; jj < GH_JW; ++jj) {
-                            float a = acc[(rh + r4) * GH_JW + jj];
-                            a = fmaf(xv[r4].x, w[un][jj].x, a);
-                            a = fmaf(xv[r4].y, w[un][jj].y, a);
-                            a = fmaf(xv[r4].z, w[un][jj].z, a);
-                            a = fmaf(xv[r4].w, w[un][jj].w, a);
-                            acc[(rh + r4) * GH_JW + jj] = a;
-                        }
+                for (int jj = 0; jj < GH_JP; ++jj) {
+                    float a = acc[jj * GH_RW + rr];
+                    a = fmaf(xv.x, w[jj][sl].x, a);
+                    a = fmaf(xv.y, w[jj][sl].y, a);
+                    a = fmaf(xv.z, w[jj][sl].z, a);
+                    a = fmaf(xv.w, w[jj][sl].w, a);
+                    acc[jj * GH_RW + rr] = a;
                 }
             }
         }
-    }
-    static_assert(GH_RW * GH_JW == 32, "the warp reduction below sums exactly 32 values");
-    red[warp][lane] = warp_transpose_sum32(acc, lane);   // lane = row * GH_JW + hidden unit
-    __syncthreads();
-    if (threadIdx.x < GH_RW * GH_JW) {
-        const int rr = threadIdx.x / GH_JW, jj = threadIdx.x % GH_JW;
-        if (rr < nr && jj < nj) {
-            float z = 0.f;
-#pragma unroll
-            for (int w8 = 0; w8 < GH_WARPS; ++w8) z += red[w8][threadIdx.x];   // fixed order: deterministic
-            z += __ldg(b1 + (size_t)layer * dg + j0 + jj);
-            u[((size_t)lb * R + r0 + rr) * dg + j0 + jj] = z / (1.0f + expf(-z));
+        static_assert(GH_JP * GH_RW == 16, "the warp reduction below sums exactly 16 values");
+        const float tot = warp_transpose_sum16(acc, lane);      // lane = jj * GH_RW + rr
+        if (lane < 16) {
+            const int jj = lane / GH_RW, rr = lane % GH_RW;
+            if (rr < nr && j0 + jj < jend) zp[(size_t)rr * dg + j0 + jj] = tot;
         }
     }
 }
@@ -144,16 +143,25 @@ constexpr int GO_RT = 8;  // rows per CTA of the output kernel
 
 // s[lb][r][h] = v[layer][h] . u[lb][r] + s0[layer][h]; then beta / lambda / c.   grid = (row tiles, layers).
 __global__ void __launch_bounds__(256)
-gate_out_kernel(const float* __restrict__ u, const float* __restrict__ v, const float* __restrict__ s0, int layer0, int R,
-                int dg, int H, int horizon, float* __restrict__ beta, float* __restrict__ lam, float* __restrict__ cterm) {
-    extern __shared__ float su[];           // [GO_RT][dg] rows of u
+gate_out_kernel(const float* __restrict__ zpart, const float* __restrict__ b1, const float* __restrict__ v,
+                const float* __restrict__ s0, int layer0, int R, int dg, int nchunk, int H, int horizon,
+                float* __restrict__ beta, float* __restrict__ lam, float* __restrict__ cterm) {
+    extern __shared__ float su[];           // [GO_RT][dg] rows of u = SiLU(sum of the chunk partials + b1)
     const int lb = blockIdx.y;
     const int layer = layer0 + lb;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r0 = blockIdx.x * GO_RT;
     const int nr = min(GO_RT, R - r0);
-    for (int i = threadIdx.x * 4; i < nr * dg; i += blockDim.x * 4)
-        *reinterpret_cast<float4*>(su + i) = *reinterpret_cast<const float4*>(u + ((size_t)lb * R + r0) * dg + i);
+    for (int i = threadIdx.x * 4; i < nr * dg; i += blockDim.x * 4) {
+        float4 z = __ldg(reinterpret_cast<const float4*>(b1 + (size_t)layer * dg + i % dg));
+        for (int ch = 0; ch < nchunk; ++ch) {           // fixed order: deterministic
+            const float4 p = *reinterpret_cast<const float4*>(zpart + (((size_t)lb * nchunk + ch) * R + r0) * dg + i);
+            z.x += p.x; z.y += p.y; z.z += p.z; z.w += p.w;
+        }
+        z.x = z.x / (1.0f + expf(-z.x)); z.y = z.y / (1.0f + expf(-z.y));
+        z.z = z.z / (1.0f + expf(-z.z)); z.w = z.w / (1.0f + expf(-z.w));
+        *reinterpret_cast<float4*>(su + i) = z;
+    }
     __syncthreads();
     for (int h = warp; h < H; h += 8) {
         const float* vh = v + ((size_t)layer * H + h) * dg;
@@ -201,14 +209,17 @@ void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, f
     count_launch();
 }
 
-void launch_gate(const GateParams& gp, const float* x, float* u_scratch, int layer0, int nlayers, int rows_per_layer,
+int gate_chunks(int D) { return (D + GH_DC - 1) / GH_DC; }
+
+void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st) {
-    dim3 g1((rows_per_layer + GH_RW - 1) / GH_RW, (gp.dg + GH_JW - 1) / GH_JW, nlayers);
-    gate_hidden_kernel<<<g1, GH_WARPS * 32, 0, st>>>(x, gp.W1, gp.b1, u_scratch, layer0, rows_per_layer, gp.D, gp.dg);
+    const int nchunk = gate_chunks(gp.D);
+    dim3 g1(((rows_per_layer + GH_RW - 1) / GH_RW) * nchunk, GH_JSPLIT, nlayers);
+    gate_hidden_kernel<<<g1, GH_WARPS * 32, 0, st>>>(x, gp.W1, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
     dim3 g2((rows_per_layer + GO_RT - 1) / GO_RT, nlayers);
     const size_t smem = (size_t)GO_RT * gp.dg * sizeof(float);
-    gate_out_kernel<<<g2, 256, smem, st>>>(u_scratch, gp.v, gp.s0, layer0, rows_per_layer, gp.dg, gp.H, gp.horizon, beta,
-                                           lam, c);
+    gate_out_kernel<<<g2, 256, smem, st>>>(z_scratch, gp.b1, gp.v, gp.s0, layer0, rows_per_layer, gp.dg, nchunk, gp.H,
+                                           gp.horizon, beta, lam, c);
     count_launch(2);
 }
 

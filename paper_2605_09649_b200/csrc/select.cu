@@ -23,8 +23,8 @@ struct CacheSrc {
     __device__ long long pages() const { return cv.P_seq; }
     // {pool, logical page, live entries, -}; pool < 0: the page is free
     __device__ int4 info(int b, long long p) const { return __ldg(cv.owner + (size_t)b * cv.P_seq + p); }
-    // returns the valid-entry bits (4) of this lane
-    __device__ unsigned load4(int b, long long p, int e0, const int4& inf, u64 (&key)[4]) const {
+    // returns the valid-entry bits (4) of this lane; sc = orderable score (high key word), tie = ~low key word
+    __device__ unsigned load4(int b, long long p, int e0, const int4& inf, uint32_t (&sc)[4], uint32_t (&tie)[4]) const {
         if (inf.x < 0 || e0 >= inf.z) return 0u;
         const size_t s = ((size_t)b * cv.P_seq + p) * PAGE + e0;
         const float4 lm = *reinterpret_cast<const float4*>(cv.lam + s);
@@ -33,18 +33,18 @@ struct CacheSrc {
         const float l4[4] = {lm.x, lm.y, lm.z, lm.w};
         const float c4[4] = {cc.x, cc.y, cc.z, cc.w};
         const int p4[4] = {ps.x, ps.y, ps.z, ps.w};
+        const int t1i = (int)t1;
         unsigned vm = 0;
+        bool bad = false;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (e0 + j < inf.z) {
-                const float age = (float)(t1 - (long long)p4[j]);
-                const float S = retention_score(l4[j], c4[j], age);
-                if (S != S) latch_error(cv.err, TRIMKV_E_NONFINITE);
-                const uint32_t tie = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)inf.x;
-                key[j] = make_key(S, tie);
-                vm |= 1u << j;
-            }
+            const float S = retention_score(l4[j], c4[j], (float)(t1i - p4[j]));
+            bad |= (S != S) && (e0 + j < inf.z);
+            sc[j] = orderable_key(S);
+            tie[j] = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)inf.x;
+            if (e0 + j < inf.z) vm |= 1u << j;
         }
+        if (bad) latch_error(cv.err, TRIMKV_E_NONFINITE);
         return vm;
     }
 };
@@ -55,9 +55,9 @@ struct ArraySrc {
     int32_t* err;
     __device__ long long pages() const { return (n + PAGE - 1) / PAGE; }
     __device__ int4 info(int, long long) const { return make_int4(0, 0, PAGE, 0); }
-    __device__ unsigned load4(int, long long p, int e0, const int4&, u64 (&key)[4]) const {
+    __device__ unsigned load4(int, long long p, int e0, const int4&, uint32_t (&sc)[4], uint32_t (&tie)[4]) const {
         const long long i0 = p * PAGE + e0;
-        float v[4];
+        float v[4] = {0.f, 0.f, 0.f, 0.f};
         unsigned vm = 0;
         if (i0 + 3 < n) {
             const float4 f = *reinterpret_cast<const float4*>(s + i0);
@@ -68,16 +68,19 @@ struct ArraySrc {
             for (int j = 0; j < 4; ++j)
                 if (i0 + j < n) { v[j] = s[i0 + j]; vm |= 1u << j; }
         }
+        bool bad = false;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (vm & (1u << j)) {
-                if (v[j] != v[j]) latch_error(err, TRIMKV_E_NONFINITE);
-                key[j] = make_key(v[j], (uint32_t)(i0 + j));
-            }
+            bad |= (v[j] != v[j]) && (vm & (1u << j));
+            sc[j] = orderable_key(v[j]);
+            tie[j] = (uint32_t)(i0 + j);
         }
+        if (bad) latch_error(err, TRIMKV_E_NONFINITE);
         return vm;
     }
 };
+
+__device__ __forceinline__ u64 compose_key(uint32_t sc, uint32_t tie) { return ((u64)sc << 32) | (u64)(~tie); }
 
 // ------------------------------------------------------------------ threshold search (one CTA, 256 threads)
 __device__ void threshold_scan(SelState* st, uint32_t* hist_b, long long k, long long n_total, bool last_pass,
@@ -188,13 +191,14 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
     unsigned under = 0;
     int cur_bin = -1;
     unsigned cur_cnt = 0;
-    auto tally = [&](const u64 (&key)[4], unsigned vm) {
+    auto tally = [&](const uint32_t (&sc)[4], const uint32_t (&tie)[4], unsigned vm) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (vm & (1u << j)) {
-                kmin = key[j] < kmin ? key[j] : kmin;
-                kmax = key[j] > kmax ? key[j] : kmax;
-                const int bin = bin_of(key[j], lo, shift);
+                const u64 key = compose_key(sc[j], tie[j]);
+                kmin = key < kmin ? key : kmin;
+                kmax = key > kmax ? key : kmax;
+                const int bin = bin_of(key, lo, shift);
                 if (bin == 0) {
                     ++under;
                 } else if (bin < NB - 1) {
@@ -221,12 +225,12 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
         int4 nA = make_int4(-1, 0, 0, 0), nB = nA;
         if (nx + sub < p1) nA = src.info(b, nx + sub);
         if (nx + 2 + sub < p1) nB = src.info(b, nx + 2 + sub);
-        u64 keyA[4], keyB[4];
+        uint32_t scA[4], scB[4], tiA[4], tiB[4];
         unsigned vmA = 0, vmB = 0;
-        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, keyA);
-        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, keyB);
-        tally(keyA, vmA);
-        tally(keyB, vmB);
+        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, scA, tiA);
+        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, scB, tiB);
+        tally(scA, tiA, vmA);
+        tally(scB, tiB, vmB);
         infA = nA;
         infB = nB;
     }
@@ -293,14 +297,25 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
     const long long p1 = min(P, p0 + chunk);
     Cand* cb = cand + (size_t)b * cand_cap;
 
-    auto emit = [&](long long page, const int4& inf, const u64 (&key)[4], unsigned vm) {   // called by all lanes
+    const uint32_t lo32 = (uint32_t)(c_lo >> 32), hi32 = (uint32_t)(c_hi >> 32);
+    auto emit = [&](long long page, const int4& inf, const uint32_t (&sc)[4], const uint32_t (&tie)[4], unsigned vm) {
+        // called by all lanes.  Most entries score above the range: one 32-bit compare settles them.
         unsigned ev = 0, cd = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (vm & (1u << j)) {
-                if (key[j] < c_lo) ev |= 1u << j;
-                else if (key[j] <= c_hi) cd |= 1u << j;
+            if ((vm & (1u << j)) && sc[j] <= hi32) {
+                if (sc[j] < lo32) {
+                    ev |= 1u << j;
+                } else {
+                    const u64 key = compose_key(sc[j], tie[j]);
+                    if (key < c_lo) ev |= 1u << j;
+                    else if (key <= c_hi) cd |= 1u << j;
+                }
             }
+        }
+        if (__ballot_sync(0xffffffffu, (ev | cd) != 0u) == 0u) {      // nothing evicted, no candidate: clear masks
+            if (l16 == 0 && page < p1 && inf.x >= 0) evict_mask[(size_t)b * mask_stride + page] = 0ull;
+            return;
         }
         if (COUNT_BELOW) below += __popc(ev);
         // candidates: warp-aggregated append
@@ -323,7 +338,7 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
                 if (cd & (1u << j)) {
                     if (w < cand_cap) {
                         Cand cnd;
-                        cnd.key = key[j];
+                        cnd.key = compose_key(sc[j], tie[j]);
                         cnd.slot = (u64)(page * PAGE + e0 + j);
                         cb[w] = cnd;
                     } else {
@@ -358,12 +373,12 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
         if (nx + sub < p1) nA = src.info(b, page_of(nx + sub));
         if (nx + 2 + sub < p1) nB = src.info(b, page_of(nx + 2 + sub));
         const long long pgA = qA < p1 ? page_of(qA) : p1, pgB = qB < p1 ? page_of(qB) : p1;
-        u64 keyA[4], keyB[4];
+        uint32_t scA[4], scB[4], tiA[4], tiB[4];
         unsigned vmA = 0, vmB = 0;
-        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, keyA);
-        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, keyB);
-        emit(pgA, infA, keyA, vmA);
-        emit(pgB, infB, keyB, vmB);
+        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, scA, tiA);
+        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, scB, tiB);
+        emit(pgA, infA, scA, tiA, vmA);
+        emit(pgB, infB, scB, tiB, vmB);
         infA = nA;
         infB = nB;
     }
@@ -582,12 +597,29 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
     }
     u64 tau = 0ull;
     if (r > 0) {
+        // Candidate keys are kept in registers when they fit (the usual case); otherwise each sweep re-reads them.
+        constexpr int PER = 8;
+        const bool inreg = C <= (long long)PER * 1024;
+        u64 kr[PER];
+        if (inreg) {
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                const long long idx = tid + (long long)i * 1024;
+                kr[i] = idx < C ? cb[idx].key : 0ull;
+            }
+        }
         // bits in which the candidate keys differ
         u64 vor = 0ull, vand = ~0ull;
-        for (long long i = tid; i < C; i += blockDim.x) {
-            const u64 key = cb[i].key;
-            vor |= key;
-            vand &= key;
+        if (inreg) {
+#pragma unroll
+            for (int i = 0; i < PER; ++i)
+                if (tid + (long long)i * 1024 < C) { vor |= kr[i]; vand &= kr[i]; }
+        } else {
+            for (long long i = tid; i < C; i += blockDim.x) {
+                const u64 key = cb[i].key;
+                vor |= key;
+                vand &= key;
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -608,10 +640,16 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
             hist[tid + 1024] = 0u;
             if (tid == 0) s_found = 0;
             __syncthreads();
-            for (long long i = tid; i < C; i += blockDim.x) {
-                const u64 key = cb[i].key;
+            auto count = [&](u64 key) {
                 const bool match = top >= 64 ? true : ((key >> top) == prefix);
                 if (match) atomicAdd(&hist[(unsigned)((key >> sh) & ((1u << dbits) - 1u))], 1u);
+            };
+            if (inreg) {
+#pragma unroll
+                for (int i = 0; i < PER; ++i)
+                    if (tid + (long long)i * 1024 < C) count(kr[i]);
+            } else {
+                for (long long i = tid; i < C; i += blockDim.x) count(cb[i].key);
             }
             __syncthreads();
             const unsigned h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
@@ -629,14 +667,15 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
             if (r > excl && r <= excl + h0) {
                 s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid);
                 s_r = r - excl;
-                s_found = 1;
+                s_found = (int)h0;
             } else if (r > excl + h0 && r <= excl + h0 + h1) {
                 s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid + 1);
                 s_r = r - excl - h0;
-                s_found = 1;
+                s_found = (int)h1;
             }
             __syncthreads();
-            if (!s_found) {                          // cannot happen with consistent counts
+            const int found = s_found;
+            if (!found) {                            // cannot happen with consistent counts
                 if (tid == 0) latch_error(err, TRIMKV_E_STATE);
                 break;
             }
@@ -644,6 +683,19 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
             r = s_r;
             top = sh;
             __syncthreads();
+            if (found == 1 && top > 0) {             // one key left under this prefix: it is the r-th smallest
+                auto pick = [&](u64 key) { if ((key >> top) == prefix) s_prefix = key; };
+                if (inreg) {
+#pragma unroll
+                    for (int i = 0; i < PER; ++i)
+                        if (tid + (long long)i * 1024 < C) pick(kr[i]);
+                } else {
+                    for (long long i = tid; i < C; i += blockDim.x) pick(cb[i].key);
+                }
+                __syncthreads();
+                prefix = s_prefix;
+                top = 0;
+            }
         }
         tau = prefix;   // the r-th smallest candidate key: everything <= tau is evicted
         for (long long i = tid; i < C; i += blockDim.x) {
@@ -715,13 +767,14 @@ redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_ma
             const long long page = pp + sub;
             if (page < P) {
                 const int4 inf = src.info(b, page);
-                u64 key[4];
-                const unsigned vm = src.load4(b, page, e0, inf, key);
+                uint32_t sc[4], tie[4];
+                const unsigned vm = src.load4(b, page, e0, inf, sc, tie);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     if (vm & (1u << j)) {
-                        const bool match = top >= 64 ? true : ((key[j] >> top) == prefix);
-                        if (match) atomicAdd(&hist[(unsigned)((key[j] >> sh) & ((1u << dbits) - 1u))], 1u);
+                        const u64 key = compose_key(sc[j], tie[j]);
+                        const bool match = top >= 64 ? true : ((key >> top) == prefix);
+                        if (match) atomicAdd(&hist[(unsigned)((key >> sh) & ((1u << dbits) - 1u))], 1u);
                     }
                 }
             }
@@ -762,16 +815,16 @@ redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_ma
     for (long long pp = warp * 2; pp < P; pp += 64) {          // warp-uniform trip count
         const long long page = pp + sub;
         int4 inf = make_int4(-1, 0, 0, 0);
-        u64 key[4];
+        uint32_t sc[4], tie[4];
         unsigned vm = 0;
         if (page < P) {
             inf = src.info(b, page);
-            vm = src.load4(b, page, e0, inf, key);
+            vm = src.load4(b, page, e0, inf, sc, tie);
         }
         unsigned ev = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if ((vm & (1u << j)) && key[j] <= tau) ev |= 1u << j;
+            if ((vm & (1u << j)) && compose_key(sc[j], tie[j]) <= tau) ev |= 1u << j;
         const unsigned nib = ev << (4 * (l16 & 7));
         unsigned wlo = (l16 < 8) ? nib : 0u, whi = (l16 >= 8) ? nib : 0u;
 #pragma unroll

@@ -128,8 +128,12 @@ struct GateParams {
 // Recomputes v and s0 of layers [layer0, layer0 + nlayers) from W2, b2, w_g, b_g.
 void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, float* s0, cudaStream_t st);
 
+// Number of input-dimension chunks the hidden layer is split into; the scratch of launch_gate holds
+// gate_chunks(D) * rows * dg floats per layer.
+int gate_chunks(int D);
+
 // rows_per_layer rows of x per layer, layers [layer0, layer0 + nlayers).
-void launch_gate(const GateParams& gp, const float* x, float* u_scratch, int layer0, int nlayers, int rows_per_layer,
+void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st);
 
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,

@@ -314,7 +314,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         A(dev_alloc(h, &h->w_g, (size_t)h->de, false));
         A(dev_alloc(h, &h->gv, (size_t)h->L * h->H * h->dg, false));
         A(dev_alloc(h, &h->gs0, (size_t)h->L * h->H, false));
-        A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg, false));
+        A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg * gate_chunks(h->D), false));
     }
     if (s == TRIMKV_OK) s = init_cache_state(h);
     if (s != TRIMKV_OK) {
