@@ -9,10 +9,13 @@ namespace {
 
 // One CTA per pool: take pages from the sequence's free stack if the pool grows past its last page,
 // then copy the new rows (K, V, retention metadata) to their slots.
+// mode bit 0 (APPEND_KV): allocate pages, write K/V rows, positions, page records and the new length.
+// mode bit 1 (APPEND_META): write the retention terms (lambda, c).  Alone, it completes an earlier APPEND_KV call
+// with the same arguments: the length then already counts the new tokens.
 __global__ void __launch_bounds__(256)
 append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* __restrict__ lam_in,
               const float* __restrict__ c_in, int horizon, const char* __restrict__ k_in,
-              const char* __restrict__ v_in) {
+              const char* __restrict__ v_in, int mode) {
     __shared__ int s_old;
     __shared__ int s_fail;
     const int h = blockIdx.x % cv.H;
@@ -23,6 +26,23 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
     const long long pool = (long long)b * cv.L * cv.H + pool_local;
     int32_t* bt = cv.block_table + pool * cv.maxpp;
 
+    if (!(mode & APPEND_KV)) {
+        const int old = cv.len[pool] - n_new;
+        if (old < 0) return;                           // the K/V half of this append failed (its error is latched)
+        const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
+        for (int j = threadIdx.x; j < n_new; j += blockDim.x) {
+            const int idx = old + j;
+            const int page = bt[idx / PAGE];
+            const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + idx % PAGE;
+            const size_t mi = (in_row0 + (size_t)j * cv.H);
+            const float lm = lam_in[mi];
+            const float cc = c_in ? c_in[mi] : horizon_term_f32(lm, horizon);
+            if (lm != lm || cc != cc) latch_error(cv.err, TRIMKV_E_NONFINITE);
+            cv.lam[slot] = lm;
+            cv.c[slot] = cc;
+        }
+        return;
+    }
     if (threadIdx.x == 0) {
         const int old = cv.len[pool];
         const long long nw = (long long)old + n_new;
@@ -71,12 +91,14 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
         const int idx = old + j;
         const int page = bt[idx / PAGE];
         const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + idx % PAGE;
-        const size_t mi = (in_row0 + (size_t)j * cv.H);
-        const float lm = lam_in[mi];
-        const float cc = c_in ? c_in[mi] : horizon_term_f32(lm, horizon);
-        if (lm != lm || cc != cc) latch_error(cv.err, TRIMKV_E_NONFINITE);
-        cv.lam[slot] = lm;
-        cv.c[slot] = cc;
+        if (mode & APPEND_META) {
+            const size_t mi = (in_row0 + (size_t)j * cv.H);
+            const float lm = lam_in[mi];
+            const float cc = c_in ? c_in[mi] : horizon_term_f32(lm, horizon);
+            if (lm != lm || cc != cc) latch_error(cv.err, TRIMKV_E_NONFINITE);
+            cv.lam[slot] = lm;
+            cv.c[slot] = cc;
+        }
         cv.pos[slot] = (int32_t)(pos0 + j + 1);
     }
     // page records of every page that received entries: owner pool, logical index, live entries
@@ -259,9 +281,9 @@ __global__ void gather_pool_kernel(CacheView cv, int b, long long pool, int n, i
 }  // namespace
 
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
-                   const float* c, int horizon, const void* k, const void* v, cudaStream_t st) {
+                   const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st) {
     const int grid = nlayers * cv.B * cv.H;
-    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v);
+    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v, mode);
     count_launch();
 }
 

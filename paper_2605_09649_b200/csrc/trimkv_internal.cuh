@@ -136,8 +136,9 @@ int gate_chunks(int D);
 void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st);
 
+constexpr int APPEND_KV = 1, APPEND_META = 2;   // halves of an append; see append_kernel
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
-                   const float* c, int horizon, const void* k, const void* v, cudaStream_t st);
+                   const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st);
 
 struct SelectBuffers {
     SelState* sel;        // [B]

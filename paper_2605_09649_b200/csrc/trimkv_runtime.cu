@@ -98,6 +98,10 @@ struct trimkv {
     long long entries;               // per sequence (all sequences advance together)
     long long rows_max;
     std::vector<void*> allocs;
+    // decode_step_all runs on two streams of its own: `fast` (highest priority) carries K/V append, attention and
+    // compaction; `side` (lowest priority) carries the gate and the selection beside the attention kernels
+    cudaStream_t fast = nullptr, side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr;
 };
 
 namespace {
@@ -169,21 +173,33 @@ trimkv_status gate_ready(const trimkv* h, int layer0, int nlayers) {
     return TRIMKV_OK;
 }
 
+// Selection on `sel_st`, compaction on `st`; when the two differ the caller orders them with events.
+trimkv_status select_impl(trimkv* h, long long k, cudaStream_t sel_st) {
+    PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
+    if (pm) pm->mark(PH_SELECT, 0, sel_st);
+    launch_select_cache(h->cv, h->sb, h->tokens[0], h->entries, k, h->cursor, h->cfg.reserved & 1, sel_st);
+    if (pm) pm->mark(PH_SELECT, 1, sel_st);
+    return TRIMKV_OK;
+}
+
+trimkv_status compact_impl(trimkv* h, cudaStream_t st) {
+    PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
+    if (pm) pm->mark(PH_COMPACT, 0, st);
+    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
+    if (pm) pm->mark(PH_COMPACT, 1, st);
+    h->entries = h->M;
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
 trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
     const long long t = h->tokens[0];
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layer %d holds %lld tokens, layer 0 holds %lld", l, h->tokens[l], t);
     const long long k = h->entries - h->M;
     if (k <= 0) return TRIMKV_OK;
-    PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
-    if (pm) pm->mark(PH_SELECT, 0, st);
-    launch_select_cache(h->cv, h->sb, t, h->entries, k, h->cursor, h->cfg.reserved & 1, st);
-    if (pm) { pm->mark(PH_SELECT, 1, st); pm->mark(PH_COMPACT, 0, st); }
-    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
-    if (pm) pm->mark(PH_COMPACT, 1, st);
-    h->entries = h->M;
-    CUDA_TRY(cudaGetLastError());
-    return TRIMKV_OK;
+    select_impl(h, k, st);
+    return compact_impl(h, st);
 }
 
 trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, void* out, cudaStream_t st) {
@@ -316,6 +332,17 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         A(dev_alloc(h, &h->gs0, (size_t)h->L * h->H, false));
         A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg * gate_chunks(h->D), false));
     }
+    if (s == TRIMKV_OK) {
+        int prio_lo = 0, prio_hi = 0;
+        cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);     // numerically lower = higher priority
+        if (cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_lo) != cudaSuccess ||
+            cudaStreamCreateWithPriority(&h->fast, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_done, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_append, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_side, cudaEventDisableTiming) != cudaSuccess)
+            s = fail(TRIMKV_E_CUDA, "stream or event creation failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
     if (s == TRIMKV_OK) s = init_cache_state(h);
     if (s != TRIMKV_OK) {
         char keep[sizeof(g_err)];
@@ -331,6 +358,12 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
 void trimkv_destroy(trimkv_t* h) {
     if (!h) return;
     cudaDeviceSynchronize();
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_append) cudaEventDestroy(h->ev_append);
+    if (h->ev_side) cudaEventDestroy(h->ev_side);
+    if (h->ev_done) cudaEventDestroy(h->ev_done);
+    if (h->side) cudaStreamDestroy(h->side);
+    if (h->fast) cudaStreamDestroy(h->fast);
     for (void* p : h->allocs) cudaFree(p);
     delete h;
 }
@@ -402,7 +435,7 @@ trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, c
         cc = h->g_c;
     }
     if (h->prof.on) h->prof.mark(PH_APPEND, 0, st);
-    launch_append(h->cv, layer, 1, n_new, h->tokens[layer], lam, cc, h->cfg.horizon, k, v, st);
+    launch_append(h->cv, layer, 1, n_new, h->tokens[layer], lam, cc, h->cfg.horizon, k, v, APPEND_KV | APPEND_META, st);
     if (h->prof.on) h->prof.mark(PH_APPEND, 1, st);
     CUDA_TRY(cudaGetLastError());
     h->tokens[layer] += n_new;
@@ -431,23 +464,49 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layers hold different token counts");
     if (t + 1 > h->max_pos) return fail(TRIMKV_E_UNSUPPORTED, "position limit %lld reached", h->max_pos);
     cudaStream_t st = (cudaStream_t)stream;
+    if (x) {
+        if (trimkv_status s = gate_ready(h, 0, h->L)) return s;
+    }
+    // Two internal streams, forked from and joined back to the caller's stream.  `fast`: K/V append -> attention ->
+    // (wait for side) -> compaction.  `side`: gate -> retention terms of the new entries -> score + selection.
+    // Attention never reads the retention terms and the selection never reads K/V, so the weight streaming of the gate
+    // and the metadata scans run beside the attention kernel, which keeps the memory system busy throughout; compaction
+    // moves K/V rows and therefore waits for both.  `fast` has the higher priority so that its few, large CTAs are
+    // placed ahead of the many small ones of the side kernels.
+    cudaStream_t sd = h->side, fs = h->fast;
+    CUDA_TRY(cudaEventRecord(h->ev_fork, st));
+    CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
+    CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_fork, 0));
+    if (h->prof.on) h->prof.mark(PH_APPEND, 0, fs);
+    launch_append(h->cv, 0, h->L, 1, t, nullptr, nullptr, h->cfg.horizon, k, v, APPEND_KV, fs);
+    if (h->prof.on) h->prof.mark(PH_APPEND, 1, fs);
+    CUDA_TRY(cudaEventRecord(h->ev_append, fs));
+    for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
+    h->entries += (long long)h->L * h->H;
+    const long long kev = h->entries - h->M;
+    trimkv_status s = attention_impl(h, 0, h->L, q, out, fs);
+
     const float* lam = lambda;
     const float* cc = nullptr;
     if (x) {
-        if (trimkv_status s = gate_ready(h, 0, h->L)) return s;
-        if (h->prof.on) h->prof.mark(PH_GATE, 0, st);
-        launch_gate(gate_params(h), x, h->u, 0, h->L, h->B, nullptr, h->g_lam, h->g_c, st);
-        if (h->prof.on) h->prof.mark(PH_GATE, 1, st);
+        if (h->prof.on) h->prof.mark(PH_GATE, 0, sd);
+        launch_gate(gate_params(h), x, h->u, 0, h->L, h->B, nullptr, h->g_lam, h->g_c, sd);
+        if (h->prof.on) h->prof.mark(PH_GATE, 1, sd);
         lam = h->g_lam;
         cc = h->g_c;
     }
-    if (h->prof.on) h->prof.mark(PH_APPEND, 0, st);
-    launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, st);
-    if (h->prof.on) h->prof.mark(PH_APPEND, 1, st);
-    for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
-    h->entries += (long long)h->L * h->H;
-    if (trimkv_status s = attention_impl(h, 0, h->L, q, out, st)) return s;
-    return evict_impl(h, st);
+    CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
+    launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, APPEND_META, sd);
+    if (kev > 0) select_impl(h, kev, sd);
+    CUDA_TRY(cudaEventRecord(h->ev_side, sd));
+
+    CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
+    if (s == TRIMKV_OK && kev > 0) s = compact_impl(h, fs);
+    CUDA_TRY(cudaEventRecord(h->ev_done, fs));
+    CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
+    if (s != TRIMKV_OK) return s;
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
 }
 
 trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host) {
