@@ -136,6 +136,12 @@ TRIMKV_API trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const v
 TRIMKV_API trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
                                      const void* q, void* out, void* stream);
 
+/* trimkv_decode_step_all runs on two internal streams by default: K/V append, attention and compaction on one, the
+ * gate and the selection beside them on the other (attention never reads retention terms, the selection never reads
+ * K/V); both are forked from and joined back to the caller's stream.  enable = 0 runs every phase back to back on the
+ * caller's stream instead (same results; for per-kernel timing).  Synchronises. */
+TRIMKV_API trimkv_status trimkv_set_overlap(trimkv_t* h, int enable);
+
 /* Pool lengths to host memory, int32 [B, L, H].  Synchronises; reports latched device errors. */
 TRIMKV_API trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host);
 
@@ -161,8 +167,9 @@ TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);
  * decode_attention, decode_step_all and score_and_evict).  trimkv_profile(h, 1) starts recording,
  * trimkv_profile(h, 0) stops; both synchronise and discard earlier records.  trimkv_profile_read
  * synchronises, writes to host ms[8] the summed milliseconds and to count[8] the number of recorded
- * intervals per phase {0 gate, 1 append, 2 attention plan, 3 attention main kernel, 4 attention merge,
- * 5 score+select, 6 compact, 7 unused}, and clears the records. */
+ * intervals per phase {0 gate, 1 append, 2 unused, 3 attention kernel, 4 unused, 5 score+select, 6 compact,
+ * 7 unused}, and clears the records.  Phases that run on different internal streams overlap in time. */
+/* enable = 2 records the attention main kernel alone (two events per call: cheap enough for a timed run). */
 TRIMKV_API trimkv_status trimkv_profile(trimkv_t* h, int enable);
 TRIMKV_API trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host);
 

@@ -6,8 +6,9 @@
 // to shared memory with bulk asynchronous copies (cp.async.bulk + mbarrier, 3 stages of 16 KB per warp),
 // the warp computes S^T = K Q^T and O^T += V^T P^T with mma.sync m16n8k16 (the GQA group is the N
 // dimension, so no tensor-core work is spent on padding rows), keeps an online softmax in registers with
-// warp-shuffle reductions over the entries, and writes (m, l, O) partials.  A second kernel merges the
-// partials of each pool.  The kernel is bound by HBM bandwidth: every K/V byte is read once.
+// warp-shuffle reductions over the entries, and writes (m, l, O) partials.  The warp that finishes the last item
+// of a pool (a per-pool ticket) merges that pool's partials and writes the output, so no second kernel is needed.
+// The kernel is bound by HBM bandwidth: every K/V byte is read once.
 //
 // Any other shape / fp32 uses a plain one-warp-per-query-head kernel.
 #include <algorithm>
@@ -23,7 +24,10 @@ constexpr int ATT_WARPS = 4;
 constexpr int ATT_STAGES = 3;
 constexpr int ROWB = 256;                      // bytes per K or V row (d = 128, bf16)
 constexpr int STAGE_BYTES = 2 * TILE * ROWB;   // K tile + V tile
-constexpr int ATT_SMEM = ATT_WARPS * ATT_STAGES * STAGE_BYTES + 256;
+constexpr int ATT_GROUPS = 1024;               // pool groups of the in-kernel item table
+constexpr int ATT_BAR_OFF = ATT_WARPS * ATT_STAGES * STAGE_BYTES;
+constexpr int ATT_GRP_OFF = ATT_BAR_OFF + 256;
+constexpr int ATT_SMEM = ATT_GRP_OFF + (ATT_GROUPS + 1) * 4 + 12;
 constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -92,50 +96,6 @@ __device__ __forceinline__ long long scope_pool(const CacheView& cv, int layer0,
     return ((long long)b * cv.L + layer0 + lb) * cv.H + h;
 }
 
-// One CTA of 1024 threads: items per pool = ceil(ceil(len / TILE) / tpi); exclusive prefix over the scope;
-// item table {scope index, first tile}.
-__global__ void __launch_bounds__(1024)
-attn_plan_kernel(CacheView cv, int layer0, int n_scope, int tpi, int32_t* __restrict__ item_prefix,
-                 int2* __restrict__ item_desc, long long max_items) {
-    __shared__ int wsum[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (n_scope + 1023) / 1024;
-    const int s0 = tid * per, s1 = min(n_scope, s0 + per);
-    int local = 0;
-    for (int si = s0; si < s1; ++si) {
-        const int len = cv.len[scope_pool(cv, layer0, si)];
-        const int tiles = (len + TILE - 1) / TILE;
-        local += (tiles + tpi - 1) / tpi;
-    }
-    int incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) wsum[warp] = incl;
-    __syncthreads();
-    int off = 0, total = 0;
-    for (int w = 0; w < 32; ++w) {
-        if (w < warp) off += wsum[w];
-        total += wsum[w];
-    }
-    int run = off + incl - local;
-    for (int si = s0; si < s1; ++si) {
-        const int len = cv.len[scope_pool(cv, layer0, si)];
-        const int tiles = (len + TILE - 1) / TILE;
-        const int items = (tiles + tpi - 1) / tpi;
-        item_prefix[si] = run;
-        for (int c = 0; c < items; ++c)
-            if (run + c < max_items) item_desc[run + c] = make_int2(si, c * tpi);
-        run += items;
-    }
-    if (tid == 0) {
-        item_prefix[n_scope] = total;
-        if (total > max_items) latch_error(cv.err, TRIMKV_E_NOMEM);
-    }
-}
-
 // ------------------------------------------------------------------ bf16 / d = 128 worker kernel
 struct ItemCtx {
     int item;        // global item index, -1 = none
@@ -144,19 +104,47 @@ struct ItemCtx {
     int first_tile;  // first tile of the item inside its pool
     int ntile;       // tiles in the item
     int len;         // pool length
+    int pool_items;  // items of this pool
+    int pool_base;   // global index of the pool's first item
     int page_id;     // lane i holds the physical page of the item's i-th page
 };
 
+// A pool of `len` entries is cut into items_of_len() items of tiles_per_item() tiles each (the last one shorter):
+// as few items as the cap of tpi tiles per item allows, of equal size, each starting on a page boundary.
+__device__ __forceinline__ int items_of_len(int len, int tpi) {
+    const int tiles = (len + TILE - 1) / TILE;
+    return (tiles + tpi - 1) / tpi;
+}
+__device__ __forceinline__ int tiles_per_item(int len, int items) {
+    const int tiles = (len + TILE - 1) / TILE;
+    return (((tiles + items - 1) / items) + 1) & ~1;
+}
+
 template <int NT>   // NT = ceil(g / 8): column tiles of 8 query heads
 __global__ void __launch_bounds__(ATT_WARPS * 32, 1)
-attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, const int32_t* __restrict__ item_prefix,
-                const int2* __restrict__ item_desc, const __nv_bfloat16* __restrict__ q, float* __restrict__ part_o,
+attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, int Hq, int32_t* __restrict__ pool_done,
+                const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ part_o,
                 float* __restrict__ part_ml, float scale_log2, long long max_items) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     unsigned char* wbuf = smem_raw + (size_t)warp * ATT_STAGES * STAGE_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + (size_t)ATT_WARPS * ATT_STAGES * STAGE_BYTES) + warp * ATT_STAGES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + ATT_BAR_OFF) + warp * ATT_STAGES;
+    int* grp = reinterpret_cast<int*>(smem_raw + ATT_GRP_OFF);     // grp[i] = items before pool group i
 
+    // ---- item table: items per group of gsz pools, then an exclusive scan (every CTA computes the same table)
+    const int ngrp = (n_scope + gsz - 1) / gsz;
+    for (int gi = threadIdx.x; gi <= ngrp; gi += blockDim.x) grp[gi] = 0;
+    __syncthreads();
+#pragma unroll 4
+    for (int si = threadIdx.x; si < n_scope; si += blockDim.x) {        // independent, coalesced length loads
+        const int len = cv.len[scope_pool(cv, layer0, si)];
+        const int it = items_of_len(len, tpi);
+        if (it) atomicAdd(&grp[si / gsz + 1], it);
+        if (len == 0 && blockIdx.x == 0) {              // an empty pool has no item: its outputs are zero
+            __nv_bfloat16* op = out + ((size_t)(si / cv.H) * Hq + (size_t)(si % cv.H) * g) * 128;
+            for (int e = 0; e < g * 128; ++e) op[e] = __float2bfloat16_rn(0.f);
+        }
+    }
     // stale shared memory must hold finite values: masked entries still multiply V rows by zero
     for (int i = lane * 16; i < ATT_STAGES * STAGE_BYTES; i += 32 * 16)
         *reinterpret_cast<uint4*>(wbuf + i) = make_uint4(0u, 0u, 0u, 0u);
@@ -164,25 +152,63 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, c
         for (int s = 0; s < ATT_STAGES; ++s) mbar_init(bars + s, 1);
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-
-    const int total_items = min((long long)item_prefix[n_scope], max_items);
+    __syncthreads();
+    if (warp == 0) {                                      // exclusive scan of the group sums by one warp
+        const int per = (ngrp + 31) / 32;
+        const int g0 = lane * per, g1 = min(ngrp, g0 + per);
+        int local = 0;
+        for (int gi = g0; gi < g1; ++gi) local += grp[gi + 1];
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        int run = incl - local;
+        for (int gi = g0; gi < g1; ++gi) {
+            const int v = grp[gi + 1];
+            grp[gi + 1] = run + v;                        // inclusive: grp[gi + 1] = items before group gi + 1
+            run += v;
+        }
+        if (lane == 0) grp[0] = 0;
+    }
+    __syncthreads();
+    const int all_items = grp[ngrp];
+    if (all_items > max_items && threadIdx.x == 0 && blockIdx.x == 0) latch_error(cv.err, TRIMKV_E_NOMEM);
+    const int total_items = (int)min((long long)all_items, max_items);
     const int gw = blockIdx.x * ATT_WARPS + warp;
     const int GW = gridDim.x * ATT_WARPS;
 
     auto load_item = [&](int item) -> ItemCtx {
         ItemCtx c;
-        c.item = -1; c.si = 0; c.b = 0; c.first_tile = 0; c.ntile = 0; c.len = 0; c.page_id = 0;
+        c.item = -1; c.si = 0; c.b = 0; c.first_tile = 0; c.ntile = 0; c.len = 0; c.pool_items = 0; c.pool_base = 0; c.page_id = 0;
         if (item >= total_items) return c;
-        const int2 dsc = item_desc[item];
+        int lo = 0, hi = ngrp - 1;                       // last group whose first item is <= item
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (grp[mid] <= item) lo = mid; else hi = mid - 1;
+        }
+        int base = grp[lo], si = lo * gsz, len = 0, cnt = 0;
+        const int si_end = min(n_scope, (lo + 1) * gsz);
+        bool found = false;
+        for (; si < si_end; ++si) {                       // ends inside the group: item < grp[lo + 1]
+            len = cv.len[scope_pool(cv, layer0, si)];
+            cnt = items_of_len(len, tpi);
+            if (item < base + cnt) { found = true; break; }
+            base += cnt;
+        }
+        if (!found) return c;
         c.item = item;
-        c.si = dsc.x;
-        c.first_tile = dsc.y;
-        const long long pool = scope_pool(cv, layer0, c.si);
-        c.b = (c.si / cv.H) % cv.B;
-        c.len = cv.len[pool];
-        const int tiles = (c.len + TILE - 1) / TILE;
-        c.ntile = min(tpi, tiles - c.first_tile);
+        c.si = si;
+        c.len = len;
+        c.pool_items = cnt;
+        c.pool_base = base;
+        const int per = tiles_per_item(len, cnt);
+        c.first_tile = (item - base) * per;
+        const long long pool = scope_pool(cv, layer0, si);
+        c.b = (si / cv.H) % cv.B;
+        const int tiles = (len + TILE - 1) / TILE;
+        c.ntile = max(0, min(per, tiles - c.first_tile));
         const int npage_item = (c.ntile + 1) / 2;
         c.page_id = (lane < npage_item) ? cv.block_table[pool * cv.maxpp + c.first_tile / 2 + lane] : 0;
         return c;
@@ -334,7 +360,10 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, c
         }
         if (failed) break;
 
-        // ---- item epilogue: partial (m, l, O)
+        // ---- item epilogue.  A pool with a single item is finished here; otherwise the partial (m, l, O) is stored
+        // and the warp that completes the pool's last item merges all of them.
+        const bool single = cons.pool_items == 1;
+        __nv_bfloat16* outp = out + ((size_t)lbb * Hq + (size_t)h * g) * 128;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             float l0 = l_run[nt][0], l1 = l_run[nt][1];
@@ -344,6 +373,22 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, c
                 l1 += __shfl_xor_sync(0xffffffffu, l1, off);
             }
             const int head0 = nt * 8 + 2 * (lane & 3);
+            if (single) {
+                const float r0 = l0 > 0.f ? 1.0f / l0 : 0.f, r1 = l1 > 0.f ? 1.0f / l1 : 0.f;
+#pragma unroll
+                for (int dt = 0; dt < 8; ++dt) {
+                    const int dr = dt * 16 + (lane >> 2);
+                    if (head0 < g) {
+                        outp[(size_t)head0 * 128 + dr] = __float2bfloat16_rn(o[nt][dt][0] * r0);
+                        outp[(size_t)head0 * 128 + dr + 8] = __float2bfloat16_rn(o[nt][dt][2] * r0);
+                    }
+                    if (head0 + 1 < g) {
+                        outp[(size_t)(head0 + 1) * 128 + dr] = __float2bfloat16_rn(o[nt][dt][1] * r1);
+                        outp[(size_t)(head0 + 1) * 128 + dr + 8] = __float2bfloat16_rn(o[nt][dt][3] * r1);
+                    }
+                }
+                continue;
+            }
             if ((lane >> 2) == 0) {
                 if (head0 < g) {
                     part_ml[((size_t)cons.item * g + head0) * 2 + 0] = m_run[nt][0];
@@ -369,6 +414,95 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, c
                 }
             }
         }
+        if (!single) {
+            __threadfence();                              // partials visible before the ticket
+            __syncwarp();
+            int ticket = 0;
+            if (lane == 0) ticket = atomicAdd(pool_done + cons.si, 1);
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket == cons.pool_items - 1) {          // this warp completed the pool: merge
+                __threadfence();
+                if (lane == 0) pool_done[cons.si] = 0;    // ready for the next call
+                const int i0 = cons.pool_base, i1 = min(cons.pool_base + cons.pool_items, total_items);
+                const int n = i1 - i0;
+                constexpr int GM = NT * 8;
+                // (m, l) of every item and head: lane t holds item t0 + t; running max and denominator per head
+                float Mj[GM], Dj[GM];
+#pragma unroll
+                for (int j = 0; j < GM; ++j) { Mj[j] = -INFINITY; Dj[j] = 0.f; }
+                for (int t0 = 0; t0 < n; t0 += 32) {
+                    const int t = t0 + lane;
+                    float mj[GM], lj[GM];
+#pragma unroll
+                    for (int j = 0; j < GM; ++j) {
+                        mj[j] = -INFINITY; lj[j] = 0.f;
+                        if (j < g && t < n) {
+                            const float2 v = __ldcg(reinterpret_cast<const float2*>(part_ml + ((size_t)(i0 + t) * g + j) * 2));
+                            mj[j] = v.x; lj[j] = v.y;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < GM; ++j) {
+                        if (j < g) {
+                            float mx = mj[j];
+#pragma unroll
+                            for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+                            const float Mn = fmaxf(Mj[j], mx);
+                            float d = exp2f(mj[j] - Mn) * lj[j];
+#pragma unroll
+                            for (int off = 16; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+                            Dj[j] = Dj[j] * exp2f(Mj[j] - Mn) + d;
+                            Mj[j] = Mn;
+                        }
+                    }
+                }
+                // O: four heads at a time, two items per batch (8 independent 16-byte loads per lane in flight)
+#pragma unroll
+                for (int jq = 0; jq < GM; jq += 4) {
+                    if (jq < g) {
+                        float4 num[4];
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj) num[jj] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int t = 0; t < n; t += 2) {
+                            float4 po[2][4];
+                            float mm[2][4];
+#pragma unroll
+                            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                for (int jj = 0; jj < 4; ++jj) {
+                                    po[u][jj] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    mm[u][jj] = -INFINITY;
+                                    if (t + u < n && jq + jj < g) {
+                                        const size_t row = (size_t)(i0 + t + u) * g + jq + jj;
+                                        po[u][jj] = __ldcg(reinterpret_cast<const float4*>(part_o + row * 128) + lane);
+                                        mm[u][jj] = __ldcg(part_ml + row * 2);
+                                    }
+                                }
+#pragma unroll
+                            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                for (int jj = 0; jj < 4; ++jj) {
+                                    const float w = exp2f(mm[u][jj] - Mj[jq + jj]);     // 0 for the padded slots
+                                    num[jj].x += w * po[u][jj].x; num[jj].y += w * po[u][jj].y;
+                                    num[jj].z += w * po[u][jj].z; num[jj].w += w * po[u][jj].w;
+                                }
+                        }
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj) {
+                            if (jq + jj < g) {
+                                const float r = Dj[jq + jj] > 0.f ? 1.0f / Dj[jq + jj] : 0.f;
+                                __nv_bfloat162 a = __floats2bfloat162_rn(num[jj].x * r, num[jj].y * r);
+                                __nv_bfloat162 c2 = __floats2bfloat162_rn(num[jj].z * r, num[jj].w * r);
+                                uint2 pk;
+                                pk.x = *reinterpret_cast<uint32_t*>(&a);
+                                pk.y = *reinterpret_cast<uint32_t*>(&c2);
+                                *reinterpret_cast<uint2*>(outp + (size_t)(jq + jj) * 128 + lane * 4) = pk;
+                            }
+                        }
+                    }
+                }
+            }
+        }
         cons = load_item(cons.item + GW);
     }
 
@@ -380,29 +514,6 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int g, int Hq, c
             mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u);
             ++consumed;
         }
-    }
-}
-
-// Merge the partials of every pool in scope: out = sum_i 2^(m_i - M) O_i / sum_i 2^(m_i - M) l_i.
-__global__ void __launch_bounds__(128)
-attn_merge_kernel(CacheView cv, int g, int Hq, const int32_t* __restrict__ item_prefix, const float* __restrict__ part_o,
-                  const float* __restrict__ part_ml, __nv_bfloat16* __restrict__ out) {
-    const int si = blockIdx.x;
-    const int h = si % cv.H;
-    const int lbb = si / cv.H;
-    const int i0 = item_prefix[si], i1 = item_prefix[si + 1];
-    const int d = threadIdx.x;   // 128 threads = one per output column
-    for (int j = 0; j < g; ++j) {
-        float M = -INFINITY;
-        for (int it = i0; it < i1; ++it) M = fmaxf(M, part_ml[((size_t)it * g + j) * 2]);
-        float num = 0.f, den = 0.f;
-        for (int it = i0; it < i1; ++it) {
-            const float w = exp2f(part_ml[((size_t)it * g + j) * 2] - M);
-            den += w * part_ml[((size_t)it * g + j) * 2 + 1];
-            num += w * part_o[((size_t)it * g + j) * 128 + d];
-        }
-        const float r = (i1 > i0 && den > 0.f) ? num / den : 0.f;
-        out[((size_t)lbb * Hq + (size_t)h * g + j) * 128 + d] = __float2bfloat16_rn(r);
     }
 }
 
@@ -496,28 +607,26 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const long long workers = (long long)sms * ATT_WARPS;
-        long long tpi = tiles_estimate / (workers * 24);       // ~24 items per worker for balance
+        long long tpi = tiles_estimate / (workers * 6);        // ~6 items per worker: few partials, enough slack
         const long long room = ab.max_items - n_scope;          // items <= tiles / tpi + n_scope must fit
         if (room > 0) tpi = std::max(tpi, (tiles_upper + room - 1) / room);
         tpi = (tpi + 1) & ~1LL;
         if (tpi < 2) tpi = 2;
         if (tpi > 64) tpi = 64;
-        if (pm) pm->mark(PH_ATTN_PLAN, 0, st);
-        attn_plan_kernel<<<1, 1024, 0, st>>>(cv, layer0, n_scope, (int)tpi, ab.item_prefix, ab.item_desc, ab.max_items);
-        if (pm) { pm->mark(PH_ATTN_PLAN, 1, st); pm->mark(PH_ATTN_MAIN, 0, st); }
+        int gsz = 1;
+        while ((n_scope + gsz - 1) / gsz > ATT_GROUPS) gsz <<= 1;
+        if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
         const float scale_log2 = scale * 1.4426950408889634f;
         if (g <= 8)
-            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, g, Hq, ab.item_prefix,
-                                                                      ab.item_desc, (const __nv_bfloat16*)q, ab.part_o,
-                                                                      ab.part_ml, scale_log2, ab.max_items);
+            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done,
+                                                                      (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
+                                                                      ab.part_o, ab.part_ml, scale_log2, ab.max_items);
         else
-            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, g, Hq, ab.item_prefix,
-                                                                      ab.item_desc, (const __nv_bfloat16*)q, ab.part_o,
-                                                                      ab.part_ml, scale_log2, ab.max_items);
-        if (pm) { pm->mark(PH_ATTN_MAIN, 1, st); pm->mark(PH_ATTN_MERGE, 0, st); }
-        attn_merge_kernel<<<n_scope, 128, 0, st>>>(cv, g, Hq, ab.item_prefix, ab.part_o, ab.part_ml, (__nv_bfloat16*)out);
-        if (pm) pm->mark(PH_ATTN_MERGE, 1, st);
-        count_launch(3);
+            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done,
+                                                                      (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
+                                                                      ab.part_o, ab.part_ml, scale_log2, ab.max_items);
+        if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
+        count_launch(1);
     } else {
         const int warps = n_scope * g;
         const int grid = (warps + 3) / 4;

@@ -161,8 +161,7 @@ void launch_invert_mask(const u64* evict_mask, u64* keep_bits, long long n, cuda
 void launch_select_state_init(SelState* sel, int B, cudaStream_t st);
 
 struct AttnBuffers {
-    int32_t* item_prefix;  // [pools_in_scope + 1]
-    int2* item_desc;       // [max_items] {scope index, first tile}
+    int32_t* pool_done;    // [pools] items of the pool finished so far in the running call; zero between calls
     float* part_o;         // [max_items][g][d]
     float* part_ml;        // [max_items][g][2]
     long long max_items;

@@ -55,6 +55,7 @@ void set_last_error(const char* fmt, ...) {
 
 struct Profiler : public tkv::PhaseMarker {
     bool on = false;
+    int only = -1;                                 // >= 0: record this phase alone
     std::vector<cudaEvent_t> pool;                 // reusable events
     size_t used = 0;
     std::vector<std::pair<int, std::pair<cudaEvent_t, cudaEvent_t>>> recs;
@@ -68,7 +69,7 @@ struct Profiler : public tkv::PhaseMarker {
         return pool[used++];
     }
     void mark(int phase, int end, cudaStream_t st) override {
-        if (!on || recs.size() >= (1u << 18)) return;
+        if (!on || recs.size() >= (1u << 18) || (only >= 0 && phase != only)) return;
         cudaEvent_t e = get();
         if (!e) return;
         cudaEventRecord(e, st);
@@ -101,6 +102,7 @@ struct trimkv {
     // decode_step_all runs on two streams of its own: `fast` (highest priority) carries K/V append, attention and
     // compaction; `side` (lowest priority) carries the gate and the selection beside the attention kernels
     cudaStream_t fast = nullptr, side = nullptr;
+    bool overlap = true;
     cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr;
 };
 
@@ -140,6 +142,7 @@ trimkv_status init_cache_state(trimkv* h) {
     CUDA_TRY(cudaMemset(h->sb.done, 0, (size_t)h->B * sizeof(unsigned)));
     CUDA_TRY(cudaMemset(h->sb.stats, 0, (size_t)h->B * 4 * sizeof(long long)));
     CUDA_TRY(cudaMemset(h->cursor, 0, (size_t)h->B * sizeof(int32_t)));
+    CUDA_TRY(cudaMemset(h->ab.pool_done, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
     launch_select_state_init(h->sb.sel, h->B, 0);
     CUDA_TRY(cudaDeviceSynchronize());
     std::fill(h->tokens.begin(), h->tokens.end(), 0LL);
@@ -315,8 +318,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     AttnBuffers& ab = h->ab;
     const long long tiles_max = (long long)h->B * (h->n_max / 32 + 2 * LH);
     ab.max_items = std::max<long long>(592LL * 32, tiles_max / 32) + 2 * (long long)pools;
-    A(dev_alloc(h, &ab.item_prefix, pools + 1, true));
-    A(dev_alloc(h, &ab.item_desc, (size_t)ab.max_items, false));
+    A(dev_alloc(h, &ab.pool_done, pools, true));
     A(dev_alloc(h, &ab.part_o, (size_t)ab.max_items * h->g * h->d, false));
     A(dev_alloc(h, &ab.part_ml, (size_t)ab.max_items * h->g * 2, false));
     h->rows_max = std::max<long long>((long long)h->B * cfg->max_chunk, (long long)h->L * h->B);
@@ -473,14 +475,17 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
     // and the metadata scans run beside the attention kernel, which keeps the memory system busy throughout; compaction
     // moves K/V rows and therefore waits for both.  `fast` has the higher priority so that its few, large CTAs are
     // placed ahead of the many small ones of the side kernels.
-    cudaStream_t sd = h->side, fs = h->fast;
-    CUDA_TRY(cudaEventRecord(h->ev_fork, st));
-    CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
-    CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_fork, 0));
+    const bool two = h->overlap;                 // off: every phase back to back on the caller's stream
+    cudaStream_t sd = two ? h->side : st, fs = two ? h->fast : st;
+    if (two) {
+        CUDA_TRY(cudaEventRecord(h->ev_fork, st));
+        CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
+        CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_fork, 0));
+    }
     if (h->prof.on) h->prof.mark(PH_APPEND, 0, fs);
     launch_append(h->cv, 0, h->L, 1, t, nullptr, nullptr, h->cfg.horizon, k, v, APPEND_KV, fs);
     if (h->prof.on) h->prof.mark(PH_APPEND, 1, fs);
-    CUDA_TRY(cudaEventRecord(h->ev_append, fs));
+    if (two) CUDA_TRY(cudaEventRecord(h->ev_append, fs));
     for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
     h->entries += (long long)h->L * h->H;
     const long long kev = h->entries - h->M;
@@ -495,15 +500,18 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
         lam = h->g_lam;
         cc = h->g_c;
     }
-    CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
+    if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
     launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, APPEND_META, sd);
     if (kev > 0) select_impl(h, kev, sd);
-    CUDA_TRY(cudaEventRecord(h->ev_side, sd));
-
-    CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
+    if (two) {
+        CUDA_TRY(cudaEventRecord(h->ev_side, sd));
+        CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
+    }
     if (s == TRIMKV_OK && kev > 0) s = compact_impl(h, fs);
-    CUDA_TRY(cudaEventRecord(h->ev_done, fs));
-    CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
+    if (two) {
+        CUDA_TRY(cudaEventRecord(h->ev_done, fs));
+        CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
+    }
     if (s != TRIMKV_OK) return s;
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
@@ -577,6 +585,14 @@ trimkv_status trimkv_profile(trimkv_t* h, int enable) {
     CUDA_TRY(cudaDeviceSynchronize());
     h->prof.clear();
     h->prof.on = enable != 0;
+    h->prof.only = enable == 2 ? (int)PH_ATTN_MAIN : -1;
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_set_overlap(trimkv_t* h, int enable) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    h->overlap = enable != 0;
     return TRIMKV_OK;
 }
 
