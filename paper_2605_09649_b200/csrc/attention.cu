@@ -24,6 +24,7 @@ constexpr int ATT_WARPS = 4;
 constexpr int ATT_STAGES = 3;
 constexpr int ROWB = 256;                      // bytes per K or V row (d = 128, bf16)
 constexpr int STAGE_BYTES = 2 * TILE * ROWB;   // K tile + V tile
+constexpr int ATT_MAX_TPI = 512;               // tiles per work item, at most (page ids are fetched 32 at a time)
 constexpr int ATT_GROUPS = 1024;               // pool groups of the in-kernel item table
 constexpr int ATT_BAR_OFF = ATT_WARPS * ATT_STAGES * STAGE_BYTES;
 constexpr int ATT_GRP_OFF = ATT_BAR_OFF + 256;
@@ -222,7 +223,12 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
     auto issue_one = [&]() {   // issue the producer cursor's tile into stage (issued % STAGES), advance
         if (prod.item < 0) return;
         const int tt = prod_tile;
-        const int page = __shfl_sync(0xffffffffu, prod.page_id, tt >> 1);
+        if (tt > 0 && (tt & 63) == 0) {                  // next 32 pages of a long item
+            const long long pool = scope_pool(cv, layer0, prod.si);
+            const int left = (prod.ntile - tt + 1) / 2;
+            prod.page_id = (lane < left) ? cv.block_table[pool * cv.maxpp + (prod.first_tile + tt) / 2 + lane] : 0;
+        }
+        const int page = __shfl_sync(0xffffffffu, prod.page_id, (tt >> 1) & 31);
         const int half = (prod.first_tile + tt) & 1;
         if (lane == 0) {
             const unsigned s = issued % ATT_STAGES;
@@ -503,7 +509,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
                 }
             }
         }
-        cons = load_item(cons.item + GW);
+        cons = (prod.item == cons.item + GW) ? prod : load_item(cons.item + GW);   // usually fetched by the producer already
     }
 
     if (failed) {
@@ -607,12 +613,15 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const long long workers = (long long)sms * ATT_WARPS;
-        long long tpi = tiles_estimate / (workers * 6);        // ~6 items per worker: few partials, enough slack
+        // Items of about half a worker's share: most pools are then one item and need no merge, while a pool that
+        // dominates the cache is still cut up.  (Few warps suffice to saturate HBM, so coarse items cost no bandwidth.)
+        // (A cross-warp merge costs a device-scope fence per item, which drains the warp's copy pipeline.)
+        long long tpi = tiles_estimate / (workers * 2);
         const long long room = ab.max_items - n_scope;          // items <= tiles / tpi + n_scope must fit
         if (room > 0) tpi = std::max(tpi, (tiles_upper + room - 1) / room);
         tpi = (tpi + 1) & ~1LL;
         if (tpi < 2) tpi = 2;
-        if (tpi > 64) tpi = 64;
+        if (tpi > ATT_MAX_TPI) tpi = ATT_MAX_TPI;
         int gsz = 1;
         while ((n_scope + gsz - 1) / gsz > ATT_GROUPS) gsz <<= 1;
         if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
