@@ -189,6 +189,12 @@ def run_ours(args, w):
 
     cache = binding.TrimKV.from_workload(w)
     per_layer, w_g = workloads.gate_params(w, seed, device=dev)
+    if args.skew > 0:
+        # per-(layer, head) logit offsets through b2 (b2 . w_g shifts s): retention then differs strongly between heads and
+        # the pools become ragged, as the paper reports for trained gates; the default run keeps the plain random init
+        off = workloads.head_logit_offsets(w, seed, args.skew, device=dev)
+        wn = w_g / (w_g * w_g).sum()
+        per_layer = [(W1, b1, W2, (b2 + off[l][:, None] * wn[None, :]).contiguous()) for l, (W1, b1, W2, b2) in enumerate(per_layer)]
     for l, p in enumerate(per_layer):
         cache.set_gate(l, *p)
     cache.set_shared_projection(w_g, w.b_g)
@@ -312,7 +318,8 @@ def run_ours(args, w):
         "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
                    "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
                    "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk,
-                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g,
+                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew,
+                   "pool_len_min_max": [int(lens[0].min()), int(lens[0].max())],
                    "parallelism": f"sequences sharded over {world} rank(s), no collective",
                    "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1)},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -342,6 +349,7 @@ def main():
     ap.add_argument("--context", type=int, default=None, help="override the prompt length (development only)")
     ap.add_argument("--b-g", type=float, default=None, help="override the shared gate bias")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--skew", type=float, default=0.0, help="std of per-(layer, head) gate-logit offsets (ragged pools)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -28,7 +28,9 @@ constexpr int ATT_MAX_TPI = 512;               // tiles per work item, at most (
 constexpr int ATT_GROUPS = 1024;               // pool groups of the in-kernel item table
 constexpr int ATT_BAR_OFF = ATT_WARPS * ATT_STAGES * STAGE_BYTES;
 constexpr int ATT_GRP_OFF = ATT_BAR_OFF + 256;
-constexpr int ATT_SMEM = ATT_GRP_OFF + (ATT_GROUPS + 1) * 4 + 12;
+constexpr int ATT_RING = 8;                    // per-warp queue of item ids fetched by the producer, read by the consumer
+constexpr int ATT_RING_OFF = ATT_GRP_OFF + (ATT_GROUPS + 1) * 4 + 12;
+constexpr int ATT_SMEM = ATT_RING_OFF + ATT_WARPS * ATT_RING * 4;
 constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -124,6 +126,7 @@ __device__ __forceinline__ int tiles_per_item(int len, int items) {
 template <int NT>   // NT = ceil(g / 8): column tiles of 8 query heads
 __global__ void __launch_bounds__(ATT_WARPS * 32, 1)
 attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, int Hq, int32_t* __restrict__ pool_done,
+                int32_t* __restrict__ sched,
                 const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ part_o,
                 float* __restrict__ part_ml, float scale_log2, long long max_items) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -131,6 +134,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
     unsigned char* wbuf = smem_raw + (size_t)warp * ATT_STAGES * STAGE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + ATT_BAR_OFF) + warp * ATT_STAGES;
     int* grp = reinterpret_cast<int*>(smem_raw + ATT_GRP_OFF);     // grp[i] = items before pool group i
+    volatile int* ring = reinterpret_cast<volatile int*>(smem_raw + ATT_RING_OFF) + warp * ATT_RING;
 
     // ---- item table: items per group of gsz pools, then an exclusive scan (every CTA computes the same table)
     const int ngrp = (n_scope + gsz - 1) / gsz;
@@ -215,9 +219,15 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
         return c;
     };
 
+    // Items are handed out dynamically (ragged pools make a static split uneven): a warp starts with item gw and then
+    // takes GW + (a global counter), one item at a time.  The producer runs ahead of the consumer by at most the
+    // pipeline depth, so a short per-warp ring of item ids links the two.
     ItemCtx prod = load_item(gw), cons = prod;
     int prod_tile = 0;
     unsigned issued = 0, consumed = 0;
+    unsigned prod_seq = prod.item >= 0 ? 1u : 0u, cons_seq = 0;
+    if (lane == 0) ring[0] = gw;
+    __syncwarp();
     bool failed = false;
 
     auto issue_one = [&]() {   // issue the producer cursor's tile into stage (issued % STAGES), advance
@@ -242,8 +252,16 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
         }
         ++issued;
         if (++prod_tile == prod.ntile) {
-            prod = load_item(prod.item + GW);
+            int nxt = 0;
+            if (lane == 0) nxt = GW + atomicAdd(sched, 1);
+            nxt = __shfl_sync(0xffffffffu, nxt, 0);
+            prod = load_item(nxt);                        // item = -1 past the end: the producer then stays idle
             prod_tile = 0;
+            if (prod.item >= 0) {
+                if (lane == 0) ring[prod_seq % ATT_RING] = nxt;
+                ++prod_seq;
+                __syncwarp();
+            }
         }
     };
 
@@ -509,7 +527,14 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
                 }
             }
         }
-        cons = (prod.item == cons.item + GW) ? prod : load_item(cons.item + GW);   // usually fetched by the producer already
+        // next item of this warp: the producer has already moved past the one just finished
+        ++cons_seq;
+        if (cons_seq < prod_seq) {
+            const int id = ring[cons_seq % ATT_RING];
+            cons = (prod.item == id) ? prod : load_item(id);
+        } else {
+            cons.item = -1;
+        }
     }
 
     if (failed) {
@@ -520,6 +545,11 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
             mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u);
             ++consumed;
         }
+    }
+    // the last warp of the grid to finish rearms the item counter for the next launch
+    if (lane == 0) {
+        const int d = atomicAdd(sched + 1, 1);
+        if (d == GW - 1) { sched[0] = 0; sched[1] = 0; }
     }
 }
 
@@ -627,11 +657,11 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
         const float scale_log2 = scale * 1.4426950408889634f;
         if (g <= 8)
-            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done,
+            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done, ab.sched,
                                                                       (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
                                                                       ab.part_o, ab.part_ml, scale_log2, ab.max_items);
         else
-            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done,
+            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done, ab.sched,
                                                                       (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
                                                                       ab.part_o, ab.part_ml, scale_log2, ab.max_items);
         if (pm) pm->mark(PH_ATTN_MAIN, 1, st);

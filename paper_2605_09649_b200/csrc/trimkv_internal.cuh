@@ -162,6 +162,7 @@ void launch_select_state_init(SelState* sel, int B, cudaStream_t st);
 
 struct AttnBuffers {
     int32_t* pool_done;    // [pools] items of the pool finished so far in the running call; zero between calls
+    int32_t* sched;        // [2] {items handed out beyond the first per warp, warps finished}; zero between calls
     float* part_o;         // [max_items][g][d]
     float* part_ml;        // [max_items][g][2]
     long long max_items;

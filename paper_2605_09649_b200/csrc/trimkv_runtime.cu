@@ -143,6 +143,7 @@ trimkv_status init_cache_state(trimkv* h) {
     CUDA_TRY(cudaMemset(h->sb.stats, 0, (size_t)h->B * 4 * sizeof(long long)));
     CUDA_TRY(cudaMemset(h->cursor, 0, (size_t)h->B * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->ab.pool_done, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
+    CUDA_TRY(cudaMemset(h->ab.sched, 0, 2 * sizeof(int32_t)));
     launch_select_state_init(h->sb.sel, h->B, 0);
     CUDA_TRY(cudaDeviceSynchronize());
     std::fill(h->tokens.begin(), h->tokens.end(), 0LL);
@@ -319,6 +320,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     const long long tiles_max = (long long)h->B * (h->n_max / 32 + 2 * LH);
     ab.max_items = std::max<long long>(592LL * 32, tiles_max / 32) + 2 * (long long)pools;
     A(dev_alloc(h, &ab.pool_done, pools, true));
+    A(dev_alloc(h, &ab.sched, 2, true));
     A(dev_alloc(h, &ab.part_o, (size_t)ab.max_items * h->g * h->d, false));
     A(dev_alloc(h, &ab.part_ml, (size_t)ab.max_items * h->g * 2, false));
     h->rows_max = std::max<long long>((long long)h->B * cfg->max_chunk, (long long)h->L * h->B);
