@@ -339,6 +339,54 @@ def run_ours(args, w):
     cache.close()
 
 
+# ------------------------------------------------------------------------------------------------- selection sweep
+def run_select_sweep(args):
+    """Standalone global selection over flat fp32 score arrays (uniform in [-8, 0]), N = 2^20 .. 2^28, timed alone.
+    Reported per (N, k): milliseconds per call and GB/s of score bytes (4 N) per call.  One JSON line."""
+    import numpy as np
+    import torch
+    from paper_2605_09649_b200 import binding, workloads
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the selection has no CPU fallback")
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    peak, peak_kind = load_peaks()
+    K, W = max(args.steps, 1), max(args.warmup, 3)
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev)            # larger than L2
+    rows = []
+    for p in range(args.sweep_min, args.sweep_max + 1):
+        n = 1 << p
+        s = workloads.selection_scores(n, seed=args.seed, device=dev)
+        bits = torch.empty((n + 63) // 64, dtype=torch.int64, device=dev)
+        ws = torch.empty(binding.select_workspace_bytes(n), dtype=torch.uint8, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        for k in (n // 8, n // 2, n - 512):
+            for _ in range(W):
+                binding.select_topk(s, k, bits, ws, status)
+            ms = []
+            for _ in range(K):
+                flush.zero_()                                                 # L2 flush between timed calls
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                binding.select_topk(s, k, bits, ws, status)
+                e1.record()
+                torch.cuda.synchronize()
+                ms.append(e0.elapsed_time(e1))
+            assert int(status.item()) == 0
+            m = float(np.median(ms))
+            rows.append({"n": n, "k_keep": k, "ms": m, "gbs": 4.0 * n / (m * 1e-3) / 1e9})
+        del s, bits, ws
+    best = max(r["gbs"] for r in rows if r["n"] == rows[-1]["n"])
+    line = {"metric": "standalone global selection, GB/s of score bytes per call", "unit": "GB/s", "value": best, "n_gpus": 1,
+            "steps": K, "warmup": W, "higher_is_better": True, "dtype": "f32", "data": "synthetic (uniform log-retention in [-8, 0])",
+            "config": {"workload": "select_sweep", "n": [1 << args.sweep_min, 1 << args.sweep_max], "l2": "flushed between timed calls"},
+            "roofline": {"bound": "hbm", "kernel": "hist_kernel + filter_kernel", "achieved": best, "peak": peak, "unit": "GB/s",
+                         "frac": best / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "note": "achieved counts ONE pass of 4 N bytes per call; the method reads the scores 2-3 times"},
+            "sweep": rows}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,7 +399,12 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--skew", type=float, default=0.0, help="std of per-(layer, head) gate-logit offsets (ragged pools)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
+    ap.add_argument("--sweep-max", type=int, default=28)
+    ap.add_argument("--sweep-min", type=int, default=20)
     args = ap.parse_args()
+    if args.select_sweep:
+        return run_select_sweep(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2605_09649_b200 import workloads
     w = workloads.WORKLOADS[args.workload]

@@ -18,6 +18,7 @@ namespace {
 // ------------------------------------------------------------------ key sources
 // A source presents its entries as pages of 64; a half-warp reads one page, 4 consecutive entries per lane.
 struct CacheSrc {
+    static constexpr bool FLAT = false;
     CacheView cv;
     long long t1;   // t + 1
     __device__ long long pages() const { return cv.P_seq; }
@@ -50,6 +51,7 @@ struct CacheSrc {
 };
 
 struct ArraySrc {
+    static constexpr bool FLAT = true;
     const float* s;
     long long n;
     int32_t* err;
@@ -154,10 +156,16 @@ __device__ void threshold_scan(SelState* st, uint32_t* hist_b, long long k, long
         if (cnt <= (u64)cand_target || c_lo >= c_hi || last_pass) {
             st->resolved = 1;
         } else {
-            const u64 span = c_hi - c_lo;
-            const int bits = 64 - __clzll((long long)span);
-            st->lo = c_lo;
-            st->shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
+            u64 nlo = c_lo;
+            int bits = 64 - __clzll((long long)(c_hi - nlo));
+            int nshift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
+            if (nshift >= 32) {                 // bins then depend on the score word alone: start them on a score boundary
+                nlo &= ~0xffffffffull;
+                bits = 64 - __clzll((long long)(c_hi - nlo));
+                nshift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
+            }
+            st->lo = nlo;
+            st->shift = nshift;
         }
         st->kmin = ~0ull;
         st->kmax = 0ull;
@@ -213,10 +221,52 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
             }
         }
     };
+    bool fast_done = false;
+    if constexpr (Src::FLAT) {
+        // Flat arrays, bins at least one score step wide and starting on a score boundary: the bin of a key depends on
+        // its 32-bit score word alone.  Grid-stride over 16-byte groups, four groups in flight per thread.
+        if (shift >= 32 && (lo & 0xffffffffull) == 0ull) {
+            const uint32_t lo32 = (uint32_t)(lo >> 32);
+            const int sh32 = shift - 32;
+            uint32_t smin = 0xffffffffu, smax = 0u;
+            bool bad = false;
+            auto one = [&](float x) {
+                bad |= (x != x);
+                const uint32_t sc = orderable_key(x);
+                smin = min(smin, sc);
+                smax = max(smax, sc);
+                if (sc < lo32) {
+                    ++under;
+                } else {
+                    const uint32_t bi = (sc - lo32) >> sh32;
+                    if (bi < (uint32_t)REG_BINS) atomicAdd(&sh[bi + 1], 1u);
+                }
+            };
+            const long long n4 = src.n >> 2;
+            const float4* s4 = reinterpret_cast<const float4*>(src.s);
+            const long long T = (long long)gridDim.x * blockDim.x;
+            for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += 4 * T) {
+                float4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (i + u * T < n4) v[u] = __ldg(s4 + i + u * T);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (i + u * T < n4) { one(v[u].x); one(v[u].y); one(v[u].z); one(v[u].w); }
+            }
+            if (blockIdx.x == 0 && threadIdx.x < (int)(src.n & 3)) one(src.s[(n4 << 2) + threadIdx.x]);
+            if (bad) latch_error(src.err, TRIMKV_E_NONFINITE);
+            if (smin <= smax) {
+                kmin = (u64)smin << 32;
+                kmax = ((u64)smax << 32) | 0xffffffffull;
+            }
+            fast_done = true;
+        }
+    }
     // Each half-warp takes two pages per trip; the page records of the next trip are fetched one trip ahead,
     // so the metadata loads of a trip depend on nothing that is still in flight.
     const long long stride = (long long)(blockDim.x >> 5) * 4;
-    long long pp = p0 + warp * 4;
+    long long pp = fast_done ? p1 : p0 + warp * 4;
     int4 infA = make_int4(-1, 0, 0, 0), infB = infA;
     if (pp + sub < p1) infA = src.info(b, pp + sub);
     if (pp + 2 + sub < p1) infB = src.info(b, pp + 2 + sub);
@@ -391,6 +441,90 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
 
 
 
+// Filter pass for flat arrays.  A warp takes 512 consecutive scores per trip; lane l reads elements 32 j + l, so the
+// ballot over the lanes for a given j is already 32 consecutive bits of the eviction mask.
+__global__ void __launch_bounds__(256)
+flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, Cand* __restrict__ cb,
+                   long long cand_cap, u64* __restrict__ evict_mask, int32_t* err) {
+    constexpr int J = 16;
+    const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
+    const uint32_t lo32 = (uint32_t)(c_lo >> 32), hi32 = (uint32_t)(c_hi >> 32);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long words = (n + 63) / 64;
+    const long long nchunk = (n + 32 * J - 1) / (32 * J);
+    const long long W = (long long)gridDim.x * (blockDim.x >> 5);
+    // Candidates go through a per-warp buffer so that the single global counter sees one atomic per ~50 candidates
+    // (a quarter of a million same-address atomics would serialise the whole pass).
+    constexpr int FBUF = 64;
+    __shared__ Cand sbuf[8][FBUF];
+    Cand* wb = sbuf[warp];
+    int nbuf = 0;                                        // warp-uniform
+    auto flush = [&]() {
+        unsigned wbase = 0;
+        if (lane == 0) wbase = atomicAdd(&st->cand_count, (unsigned)nbuf);
+        wbase = __shfl_sync(0xffffffffu, wbase, 0);
+        for (int i = lane; i < nbuf; i += 32) {
+            if ((long long)wbase + i < cand_cap) cb[(long long)wbase + i] = wb[i];
+            else latch_error(err, TRIMKV_E_NOMEM);
+        }
+        __syncwarp();
+        nbuf = 0;
+    };
+    const unsigned below_lane = (1u << lane) - 1u;
+    for (long long c = (long long)blockIdx.x * (blockDim.x >> 5) + warp; c < nchunk; c += W) {
+        const long long base = c * (32 * J);
+        const long long rem = n - base;                  // elements left from the start of this chunk
+        const float* p = s + base + lane;
+        float x[J];
+        if (rem >= 32 * J) {
+#pragma unroll
+            for (int j = 0; j < J; ++j) x[j] = __ldg(p + 32 * j);
+        } else {
+#pragma unroll
+            for (int j = 0; j < J; ++j) x[j] = (32 * j + lane < rem) ? __ldg(p + 32 * j) : __int_as_float(0x7f800000);
+        }
+        unsigned evb[J];
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+            const uint32_t sc = orderable_key(x[j]);
+            // one 32-bit compare settles an entry unless its score word equals that of a range end
+            bool ev = sc < lo32;
+            bool cd = !ev && sc <= hi32;
+            if (cd && (sc == lo32 || sc == hi32)) {
+                const u64 key = compose_key(sc, (uint32_t)(base + 32 * j + lane));
+                ev = key < c_lo;
+                cd = !ev && key <= c_hi;
+            }
+            if (rem < 32 * J && 32 * j + lane >= rem) { ev = false; cd = false; }
+            evb[j] = __ballot_sync(0xffffffffu, ev);
+            const unsigned cdb = __ballot_sync(0xffffffffu, cd);
+            if (cdb) {                                   // stage the candidates in this warp's shared-memory buffer
+                const int cnt = __popc(cdb);
+                if (nbuf + cnt > FBUF) { flush(); }
+                if (cd) {
+                    const long long idx = base + 32 * j + lane;
+                    Cand cnd;
+                    cnd.key = compose_key(sc, (uint32_t)idx);
+                    cnd.slot = (u64)idx;
+                    wb[nbuf + __popc(cdb & below_lane)] = cnd;
+                }
+                nbuf += cnt;
+                __syncwarp();
+            }
+        }
+        if (lane < J / 2) {
+            // word `lane` of this chunk = ballots 2 * lane (low half) and 2 * lane + 1 (high half)
+            u64 wv = 0ull;
+#pragma unroll
+            for (int j = 0; j < J / 2; ++j)
+                if (lane == j) wv = (u64)evb[2 * j] | ((u64)evb[2 * j + 1] << 32);
+            const long long wi = c * (J / 2) + lane;
+            if (wi < words) evict_mask[wi] = wv;
+        }
+    }
+    if (nbuf > 0) flush();
+}
+
 // ------------------------------------------------------------------ sample bracket (cache path)
 // One full pass suffices when a candidate range that surely holds the k-th smallest key is known beforehand.
 // A Bernoulli sample of the sequence's keys (a hash of the slot decides, about SAMPLE_MEAN keys) is sorted by one
@@ -530,10 +664,8 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
     u64 lo = 0ull, hi = ~0ull;
     if (ns > 0 && !distrust) {
         long long r_lo, r_hi;
-        bool exact = false;
         if ((long long)raw == n_total) {              // every key was sampled: the k-th smallest is known exactly
             r_lo = r_hi = k_evict;
-            exact = true;
         } else {
             const double mu = (double)k_evict * (double)ns / (double)n_total;   // expected sample rank of the k-th key
             const double dev = 7.0 * sqrt(mu) + 8.0;
@@ -542,7 +674,6 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
         }
         if (r_lo >= 1) lo = bound_of_rank(min(r_lo, (long long)ns), false);
         if (r_hi <= ns) hi = bound_of_rank(max(r_hi, 1LL), true);
-        (void)exact;
     } else if (distrust) {
         lo = hi = ~0ull;        // test hook: a range that cannot hold the k-th key, so that the exact redo runs
     }
@@ -837,6 +968,47 @@ redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_ma
     if (tid == 0) st->resolved = 1;
 }
 
+// Flat arrays: centres the first histogram pass on the data.  1024 threads read 4096 evenly spaced scores; the bins
+// then span the sampled score range widened by an eighth on both sides (any range is correct: keys outside it fall
+// into the catch-all bins and cost a further pass at worst; a fitting one settles the selection in one pass).
+__global__ void __launch_bounds__(1024)
+seed_range_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st) {
+    __shared__ uint32_t wmin[32], wmax[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t smin = 0xffffffffu, smax = 0u;
+    const long long step = n / 4096 > 0 ? n / 4096 : 1;
+    for (int i = 0; i < 4; ++i) {
+        const long long idx = (long long)(tid * 4 + i) * step;
+        if (idx < n) {
+            const float x = s[idx];
+            if (x == x) {
+                const uint32_t sc = orderable_key(x);
+                smin = min(smin, sc);
+                smax = max(smax, sc);
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        smin = min(smin, __shfl_xor_sync(0xffffffffu, smin, o));
+        smax = max(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+    }
+    if (lane == 0) { wmin[warp] = smin; wmax[warp] = smax; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 0; w < 32; ++w) { smin = min(smin, wmin[w]); smax = max(smax, wmax[w]); }
+        if (smin < smax) {
+            const uint32_t pad = (smax - smin) / 8u + 1u;
+            const uint32_t a = smin > pad ? smin - pad : 0u;
+            const uint32_t b = smax < 0xffffffffu - pad ? smax + pad : 0xffffffffu;
+            const u64 lo = (u64)a << 32, hi = ((u64)b << 32) | 0xffffffffull;
+            const int bits = 64 - __clzll((long long)(hi - lo));
+            const int shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
+            if (shift >= 32) { st->lo = lo; st->shift = shift; }
+        }
+    }
+}
+
 __global__ void state_init_kernel(SelState* sel, int B) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
@@ -864,17 +1036,17 @@ int grid_x_for(long long pages, int B) {
     return (int)g;
 }
 
-template <class Src>
-void run_select(const Src& src, long long pages, int B, const SelectBuffers& sb, long long n_total, long long k_evict,
-                int max_passes, unsigned cand_target, u64* evict_mask, long long mask_stride, int32_t* cursor,
-                int32_t* err, cudaStream_t st) {
-    dim3 grid(grid_x_for(pages, B), B);
+// Histogram path (flat arrays): up to max_passes histogram passes, filter, exact resolve.
+void run_select_flat(const ArraySrc& src, const SelectBuffers& sb, long long k_evict, int max_passes, unsigned cand_target,
+                     u64* evict_mask, int32_t* err, cudaStream_t st) {
+    const long long pages = (src.n + PAGE - 1) / PAGE;
+    dim3 grid(grid_x_for(pages, 1), 1);
     for (int p = 0; p < max_passes; ++p)
-        hist_kernel<Src><<<grid, 256, 0, st>>>(src, sb.sel, sb.hist, sb.done, k_evict, n_total, p == max_passes - 1,
-                                               cand_target);
-    filter_kernel<Src, false><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, err);
-    resolve_kernel<true><<<B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, evict_mask, mask_stride, k_evict,
-                                             max(cand_target / 8u, 1u), sb.stats, cursor, err);
+        hist_kernel<ArraySrc><<<grid, 256, 0, st>>>(src, sb.sel, sb.hist, sb.done, k_evict, src.n, p == max_passes - 1,
+                                                    cand_target);
+    flat_filter_kernel<<<grid, 256, 0, st>>>(src.s, src.n, sb.sel, sb.cand, sb.cand_cap, evict_mask, err);
+    resolve_kernel<true><<<1, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, evict_mask, pages, k_evict,
+                                             max(cand_target / 8u, 1u), sb.stats, nullptr, err);
     count_launch(max_passes + 2);
 }
 
@@ -915,8 +1087,9 @@ void launch_select_array(const float* scores, long long n, long long k_evict, u6
     src.s = scores;
     src.n = n;
     src.err = err;
-    const long long pages = (n + PAGE - 1) / PAGE;
-    run_select(src, pages, 1, sb, n, k_evict, 7, (unsigned)sb.cand_cap, evict_mask, pages, nullptr, err, st);
+    seed_range_kernel<<<1, 1024, 0, st>>>(scores, n, sb.sel);
+    count_launch();
+    run_select_flat(src, sb, k_evict, 7, (unsigned)sb.cand_cap, evict_mask, err, st);
 }
 
 void launch_invert_mask(const u64* evict_mask, u64* keep_bits, long long n, cudaStream_t st) {
