@@ -25,6 +25,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_mma_kernel launch, from the ncu capture summarised in
+# profiles/attn_mma_kernel_llama8b_cache_at_budget.md (same kernel source as now; set to None when the kernel changes).
+NCU_TRAFFIC_BYTES = {"llama8b_32k": None}
+
 METRIC = "decode tokens/s at fixed global KV budget (step time in ms_per_step, % of HBM peak in roofline)"
 UNIT = "tokens/s"
 
@@ -323,7 +327,8 @@ def run_ours(args, w):
                    "parallelism": f"sequences sharded over {world} rank(s), no collective",
                    "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1)},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if args.skew == 0 and args.context is None else None,
                      "algorithmic_bytes_per_launch": ab["kv"], "avg_launch_ms": attn_ms_per,
                      "note": "timed region: the kernel shares HBM with the gate and selection kernels running beside it",
                      "alone": {"avg_launch_ms": iso_ms, "achieved": iso_gbs, "frac": iso_gbs / peak},

@@ -211,16 +211,22 @@ void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, f
 
 int gate_chunks(int D) { return (D + GH_DC - 1) / GH_DC; }
 
+void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, int layer0, int nlayers, int rows_per_layer,
+                     float* beta, float* lam, float* c, cudaStream_t st) {
+    dim3 g2((rows_per_layer + GO_RT - 1) / GO_RT, nlayers);
+    const size_t smem = (size_t)GO_RT * gp.dg * sizeof(float);
+    gate_out_kernel<<<g2, 256, smem, st>>>(z_scratch, gp.b1, gp.v, gp.s0, layer0, rows_per_layer, gp.dg, nchunk, gp.H,
+                                           gp.horizon, beta, lam, c);
+    count_launch();
+}
+
 void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st) {
     const int nchunk = gate_chunks(gp.D);
     dim3 g1(((rows_per_layer + GH_RW - 1) / GH_RW) * nchunk, GH_JSPLIT, nlayers);
     gate_hidden_kernel<<<g1, GH_WARPS * 32, 0, st>>>(x, gp.W1, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
-    dim3 g2((rows_per_layer + GO_RT - 1) / GO_RT, nlayers);
-    const size_t smem = (size_t)GO_RT * gp.dg * sizeof(float);
-    gate_out_kernel<<<g2, 256, smem, st>>>(z_scratch, gp.b1, gp.v, gp.s0, layer0, rows_per_layer, gp.dg, nchunk, gp.H,
-                                           gp.horizon, beta, lam, c);
-    count_launch(2);
+    count_launch();
+    launch_gate_out(gp, z_scratch, nchunk, layer0, nlayers, rows_per_layer, beta, lam, c, st);
 }
 
 }  // namespace tkv

@@ -140,6 +140,18 @@ constexpr int APPEND_KV = 1, APPEND_META = 2;   // halves of an append; see appe
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st);
 
+// Second half of the gate alone: z_scratch holds nchunk partial pre-activations per (row, hidden unit).
+void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, int layer0, int nlayers, int rows_per_layer,
+                     float* beta, float* lam, float* c, cudaStream_t st);
+
+// Tensor-core (tcgen05, 3xTF32) form of the hidden layer for calls with many rows of one layer.
+struct GateTcState;
+bool gate_tc_supported(int D, int dg);
+GateTcState* gate_tc_create(float* xhi, float* xlo, long long rows_alloc, float* whi, float* wlo, int L, int dg, int D);
+void gate_tc_destroy(GateTcState* s);
+void launch_split_tf32(const float* in, float* hi, float* lo, long long n, cudaStream_t st);
+void launch_gate_gemm_tc(GateTcState* s, const float* x, int R, int layer, float* z, int32_t* err, cudaStream_t st);
+
 struct SelectBuffers {
     SelState* sel;        // [B]
     uint32_t* hist;       // [B][NB]

@@ -36,6 +36,8 @@ trimkv_status fail(trimkv_status s, const char* fmt, ...) {
                         cudaGetErrorString(e__));                                                          \
     } while (0)
 
+constexpr int TC_MIN_ROWS = 256;   // rows of one layer from which the gate's hidden layer runs on tensor cores
+
 int ceil_log2(long long v) {
     int b = 0;
     while ((1LL << b) < v) ++b;
@@ -92,6 +94,8 @@ struct trimkv {
     AttnBuffers ab;
     int32_t *hole, *mover, *cursor;
     float *W1, *b1, *W2, *b2, *w_g, *gv, *gs0, *u, *g_lam, *g_c;
+    float *W1hi = nullptr, *W1lo = nullptr, *xhi = nullptr, *xlo = nullptr;   // 3xTF32 operands of the tensor-core gate
+    GateTcState* tc = nullptr;
     float b_g;
     bool shared_set;
     std::vector<char> gate_set;
@@ -167,6 +171,16 @@ GateParams gate_params(const trimkv* h) {
     gp.W1 = h->W1; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.v = h->gv; gp.s0 = h->gs0; gp.b_g = h->b_g;
     gp.D = h->D; gp.dg = h->dg; gp.de = h->de; gp.H = h->H; gp.horizon = h->cfg.horizon;
     return gp;
+}
+
+// Gate of one layer for `rows` rows: tensor cores when the call is a dense contraction, else the weight-streaming kernels.
+void gate_one_layer(trimkv* h, const float* x, int layer, int rows, float* beta, float* lam, float* c, cudaStream_t st) {
+    if (h->tc && rows >= TC_MIN_ROWS) {
+        launch_gate_gemm_tc(h->tc, x, rows, layer, h->u, h->cv.err, st);
+        launch_gate_out(gate_params(h), h->u, 1, layer, 1, rows, beta, lam, c, st);
+    } else {
+        launch_gate(gate_params(h), x, h->u, layer, 1, rows, beta, lam, c, st);
+    }
 }
 
 trimkv_status gate_ready(const trimkv* h, int layer0, int nlayers) {
@@ -335,6 +349,13 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         A(dev_alloc(h, &h->gv, (size_t)h->L * h->H * h->dg, false));
         A(dev_alloc(h, &h->gs0, (size_t)h->L * h->H, false));
         A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg * gate_chunks(h->D), false));
+        if (s == TRIMKV_OK && gate_tc_supported(h->D, h->dg) && (long long)h->B * cfg->max_chunk >= TC_MIN_ROWS) {
+            A(dev_alloc(h, &h->W1hi, (size_t)h->L * h->dg * h->D, true));
+            A(dev_alloc(h, &h->W1lo, (size_t)h->L * h->dg * h->D, true));
+            A(dev_alloc(h, &h->xhi, (size_t)h->rows_max * h->D, true));
+            A(dev_alloc(h, &h->xlo, (size_t)h->rows_max * h->D, true));
+            if (s == TRIMKV_OK) h->tc = gate_tc_create(h->xhi, h->xlo, h->rows_max, h->W1hi, h->W1lo, h->L, h->dg, h->D);
+        }
     }
     if (s == TRIMKV_OK) {
         int prio_lo = 0, prio_hi = 0;
@@ -369,6 +390,7 @@ void trimkv_destroy(trimkv_t* h) {
     if (h->side) cudaStreamDestroy(h->side);
     if (h->fast) cudaStreamDestroy(h->fast);
     for (void* p : h->allocs) cudaFree(p);
+    gate_tc_destroy(h->tc);
     delete h;
 }
 
@@ -388,6 +410,8 @@ trimkv_status trimkv_set_gate(trimkv_t* h, int layer, const float* W1, const flo
     CUDA_TRY(cudaMemcpy(h->W2 + (size_t)layer * h->H * h->de * h->dg, W2, (size_t)h->H * h->de * h->dg * 4, cudaMemcpyDeviceToDevice));
     CUDA_TRY(cudaMemcpy(h->b2 + (size_t)layer * h->H * h->de, b2, (size_t)h->H * h->de * 4, cudaMemcpyDeviceToDevice));
     h->gate_set[layer] = 1;
+    if (h->tc) launch_split_tf32(h->W1 + (size_t)layer * h->dg * h->D, h->W1hi + (size_t)layer * h->dg * h->D,
+                                 h->W1lo + (size_t)layer * h->dg * h->D, (long long)h->dg * h->D, 0);
     if (h->shared_set) launch_gate_fold(gate_params(h), layer, 1, h->gv, h->gs0, 0);
     CUDA_TRY(cudaDeviceSynchronize());
     return TRIMKV_OK;
@@ -413,7 +437,7 @@ trimkv_status trimkv_gate(trimkv_t* h, int layer, int n_new, const float* x, flo
     if (layer < 0 || layer >= h->L || n_new < 1 || !x || !aligned16(x)) return fail(TRIMKV_E_ARG, "bad layer, n_new or x (x must be 16-byte aligned)");
     if ((long long)h->B * n_new > h->rows_max) return fail(TRIMKV_E_ARG, "n_new exceeds max_chunk");
     if (trimkv_status s = gate_ready(h, layer, 1)) return s;
-    launch_gate(gate_params(h), x, h->u, layer, 1, h->B * n_new, beta, lambda, c, (cudaStream_t)stream);
+    gate_one_layer(h, x, layer, h->B * n_new, beta, lambda, c, (cudaStream_t)stream);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
 }
@@ -433,7 +457,7 @@ trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, c
         if (!aligned16(x)) return fail(TRIMKV_E_ARG, "x must be 16-byte aligned");
         if (trimkv_status s = gate_ready(h, layer, 1)) return s;
         if (h->prof.on) h->prof.mark(PH_GATE, 0, st);
-        launch_gate(gate_params(h), x, h->u, layer, 1, h->B * n_new, nullptr, h->g_lam, h->g_c, st);
+        gate_one_layer(h, x, layer, h->B * n_new, nullptr, h->g_lam, h->g_c, st);
         if (h->prof.on) h->prof.mark(PH_GATE, 1, st);
         lam = h->g_lam;
         cc = h->g_c;

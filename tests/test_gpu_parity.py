@@ -85,6 +85,29 @@ def test_gate_matches_oracle_llama_shape(b_g, std):
     cache.close()
 
 
+@pytest.mark.parametrize("name,b_g,std,n", [("llama8b_32k", 18.0, 0.02, 64), ("llama8b_32k", 4.0, 0.05, 40),
+                                             ("qwen_vl_16k", 4.0, 0.02, 100), ("stress_128k", 0.5, 0.02, 300)])
+def test_gate_chunk_sized_calls_use_tensor_cores_and_match_oracle(name, b_g, std, n):
+    """Hundreds of rows of one layer per call: the hidden layer runs as the split-precision tensor-core GEMM (row counts
+    that do not fill the last 128-row tile, three hidden sizes); outputs within 1e-5 of the fp64 oracle."""
+    w = workloads.WORKLOADS[name].replace(layers=2, budget_entries=4096, chunk=max(n, 320 // workloads.WORKLOADS[name].batch + 1))
+    assert w.batch * w.chunk >= 256 and w.batch * n >= 256
+    per_layer, w_g = workloads.gate_params(w, 1, device=DEV, std=std)
+    cache = binding.TrimKV.from_workload(w)
+    for l, p in enumerate(per_layer):
+        cache.set_gate(l, *p)
+    cache.set_shared_projection(w_g, b_g)
+    for layer in range(w.layers):
+        x = workloads.hidden_states(w, 5, layer, 0, n, device=DEV)
+        beta, lam, c = cache.gate(layer, x)
+        ob, ol, oc = _oracle_gate(per_layer, w_g, b_g, layer, x, w.horizon)
+        _rel_close(to_np(beta), ob, GATE_RTOL, "beta")
+        _rel_close(to_np(lam), ol, GATE_RTOL, "lambda")
+        _rel_close(to_np(c), oc, GATE_RTOL, "c")
+    cache.sync_status()
+    cache.close()
+
+
 def test_gate_zero_readout_gives_sigmoid_of_bias():
     w = workloads.WORKLOADS["tiny"].replace(batch=2)
     cache, per_layer, w_g = _gate_setup(w, 0, 18.0)
