@@ -1,4 +1,4 @@
-"""Full-size parity: the named workloads at their BASELINE shapes, cache at its budget, stepped with
+"""Full-size parity: the named workloads at their full shapes, cache at its budget, stepped with
 trimkv_decode_step_all exactly as bench.py does (all layers per call, gate on x, two internal streams).
 
 The oracle cannot run a whole step at these sizes in seconds, so one sequence is sampled and checked in full for

@@ -1,6 +1,6 @@
 """GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs.
 
-Tolerances (the benchmark spec's): kept/evicted sets bit-exact given identical fp32 retention values; gate
+Tolerances: kept/evicted sets bit-exact given identical fp32 retention values; gate
 outputs within 1e-5 relative; attention within 2e-2 max-abs in bf16 and 1e-4 in fp32.
 """
 import numpy as np
