@@ -36,7 +36,7 @@ class Workload:
     decode_steps: int
     chunk: int                   # prefill chunk (tokens per append before an eviction)
     gate_hidden: int = 512       # d_g (Sec. 5.1)
-XX
+    gate_embed: int = 64         # d_e (width of Proj's output; the paper does not state it)
     horizon: int = 2             # T - t at inference (Sec. 5.1)
     b_g: float = 18.0            # shared bias (its initial value, Sec. 5.1)
     visual_period: int = 0       # >0: every `visual_period` tokens end with `visual_len` visual tokens
