@@ -204,17 +204,56 @@ def run_ours(args, w):
     cache.set_shared_projection(w_g, w.b_g)
     bank = workloads.ProjectionBank(w, seed, device=dev)
 
-    # ---- untimed: chunked prefill with eviction after every chunk
+    # ---- untimed: chunked prefill with eviction after every chunk (library time measured with events on the side)
+    def prefill(start, count):
+        """Appends tokens [start, start + count) in chunks with an eviction after each; returns (ms of library work, chunks)."""
+        ms, chunks, done = 0.0, 0, 0
+        while done < count:
+            n = min(w.chunk, count - done)
+            evs = []
+            for l in range(w.layers):
+                x = workloads.hidden_states(w, seed, l, start + done, n, device=dev)
+                _, k, v = workloads.project_qkv(w, bank, l, x)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                cache.append(l, k, v, x=x)
+                if l == w.layers - 1:
+                    cache.score_and_evict()
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            ms += sum(a.elapsed_time(b) for a, b in evs)
+            chunks += 1
+            done += n
+        return ms, chunks
+
     t_setup = time.time()
-    done = 0
-    while done < w.context:
-        n = min(w.chunk, w.context - done)
-        for l in range(w.layers):
-            x = workloads.hidden_states(w, seed, l, done, n, device=dev)
-            _, k, v = workloads.project_qkv(w, bank, l, x)
-            cache.append(l, k, v, x=x)
-        cache.score_and_evict()
-        done += n
+    tokens_seen = 0
+    prefill_ms, prefill_chunks, early_decode_ms, early_decode_steps = 0.0, 0, 0.0, 0
+    for turn in range(w.turns):
+        ms, ch = prefill(tokens_seen, w.context)
+        prefill_ms += ms; prefill_chunks += ch
+        tokens_seen += w.context
+        if turn < w.turns - 1:
+            # earlier turns of a dialogue: their decode steps run here (timed coarsely); the last turn's are the timed region
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            sets = []
+            for i in range(4):
+                xs, ks, vs, qs = [], [], [], []
+                for l in range(w.layers):
+                    x = workloads.hidden_states(w, seed, l, tokens_seen + i, 1, device=dev)
+                    q, k, v = workloads.project_qkv(w, bank, l, x)
+                    xs.append(x[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0]); qs.append(q[:, 0])
+                sets.append([torch.stack(t).contiguous() for t in (xs, ks, vs, qs)])
+            o = torch.empty_like(sets[0][3])
+            a.record()
+            for i in range(w.decode_steps):
+                X, Kt, Vt, Q = sets[i % 4]
+                cache.decode_step_all(Kt, Vt, Q, o, x=X)
+            b.record()
+            torch.cuda.synchronize()
+            early_decode_ms += a.elapsed_time(b); early_decode_steps += w.decode_steps
+            tokens_seen += w.decode_steps
     cache.sync_status()
     entries = int(cache.lengths()[0].sum())
     t_setup = time.time() - t_setup
@@ -223,7 +262,7 @@ def run_ours(args, w):
     def step_inputs(i):
         xs, ks, vs, qs = [], [], [], []
         for l in range(w.layers):
-            x = workloads.hidden_states(w, seed, l, w.context + i, 1, device=dev)
+            x = workloads.hidden_states(w, seed, l, tokens_seen + i, 1, device=dev)
             q, k, v = workloads.project_qkv(w, bank, l, x)
             xs.append(x[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0]); qs.append(q[:, 0])
         return [torch.stack(t).contiguous() for t in (xs, ks, vs, qs)]
@@ -325,7 +364,12 @@ def run_ours(args, w):
                    "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew,
                    "pool_len_min_max": [int(lens[0].min()), int(lens[0].max())],
                    "parallelism": f"sequences sharded over {world} rank(s), no collective",
-                   "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1)},
+                   "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1),
+                   "turns": w.turns, "tokens_before_timed_region": tokens_seen,
+                   "prefill": {"chunks": prefill_chunks, "ms_per_chunk": prefill_ms / max(prefill_chunks, 1),
+                               "tokens_per_s": w.batch * w.chunk / (prefill_ms / max(prefill_chunks, 1) * 1e-3) if prefill_ms > 0 else None,
+                               "what": "gate + append of every layer and one eviction per chunk (no chunk attention)"},
+                   "earlier_turn_decode_ms_per_step": early_decode_ms / early_decode_steps if early_decode_steps else None},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": NCU_TRAFFIC_BYTES.get(w.name) if args.skew == 0 and args.context is None else None,

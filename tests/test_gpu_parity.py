@@ -313,6 +313,37 @@ def test_bf16_multi_page_long_pool():
     _run_bf16_case(w, 21, [512] * 11 + [300], 3, lam_fn, check_rows=False)
 
 
+def test_multi_turn_dialogue_flow_matches_oracle():
+    """Several turns of (chunked prompt with an eviction per chunk, then decode steps) under one persistent budget:
+    positions keep counting across turns; kept sets bit-exact after every eviction, attention within tolerance."""
+    w = BF16_SMALL.replace(budget_entries=520, batch=2, chunk=64)
+    pair = Pair(w)
+    r = np.random.default_rng(17)
+    g = torch.Generator(device=DEV); g.manual_seed(17)
+    dt = torch.bfloat16
+    for turn in range(3):
+        for n in (64, 64, 31):                                   # the turn's user tokens, in chunks
+            for l in range(w.layers):
+                k = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                v = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), scale=0.02 * (1 + turn))
+                pair.append(l, k, v, lam, oracle_retention(lam, w.horizon))
+            pair.evict()
+            pair.check_sets()
+        for step in range(5):                                    # the turn's decoded tokens
+            for l in range(w.layers):
+                k = torch.randn(w.batch, 1, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                v = torch.randn(w.batch, 1, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                lam = random_lambda((w.batch, 1, w.kv_heads), int(r.integers(1 << 30)), scale=0.02)
+                pair.append(l, k, v, lam, oracle_retention(lam, w.horizon))
+                q = torch.randn(w.batch, w.q_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                pair.check_attention(l, q, ATT_ATOL_BF16)
+            pair.evict()
+            pair.check_sets()
+            assert int(pair.gpu.lengths().sum()) == w.batch * w.budget_entries
+    pair.close()
+
+
 def test_step_all_matches_layerwise_oracle():
     w = BF16_SMALL.replace(budget_entries=400)
     lam_fn = lambda r, shape, l: random_lambda(shape, int(r.integers(1 << 30)))
