@@ -16,6 +16,8 @@ What each function follows:
   largest scores over all layers and heads (full sort = the plain definition).
 * `attention`, `attention_weights` -- Sec. 2.1 softmax attention restricted to the
   retained set (Eq. (1) with r in {0,1}).
+* `retention_attention`, `retention_attention_weights` -- Sec. 2.2 retention-gated attention
+  (weights beta_i^(t-i) e^{z_i}), an option of the decode attention.
 * `OracleCache`                    -- the per-step loop: append, score, evict, attend.
 
 Parity pins: every function here is pinned by tests/test_oracle_pins.py except the
@@ -147,6 +149,30 @@ def attention(q, K, V):
     return attention_weights(q, K) @ V
 
 
+def retention_attention_weights(q, K, lam32, pos, t):
+    """alpha~_i = beta_i^(t-i) e^{z_i} / sum_j beta_j^(t-j) e^{z_j}  (Sec. 2.2, retention-gated attention), fp64.
+
+    z_i = q . k_i / sqrt(d); beta_i^(t-i) = exp((t - i) * lambda_i) with the entry's stored fp32 lambda_i = ln beta_i and
+    its 1-based position i; t = number of tokens seen.  The newest token (i = t) has weight beta^0 = 1; lambda = 0
+    everywhere gives back plain softmax attention.
+    """
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    z = (K @ q) / np.sqrt(F64(q.shape[-1]))
+    z = z + (F64(t) - np.asarray(pos, F64)) * np.asarray(lam32, F32).astype(F64)
+    z = z - z.max()
+    w = np.exp(z)
+    return w / w.sum()
+
+
+def retention_attention(q, K, V, lam32, pos, t):
+    """o~ = sum_i alpha~_i v_i over the retained entries (Sec. 2.2); zeros for an empty set."""
+    V = np.asarray(V, F64)
+    if V.shape[0] == 0:
+        return np.zeros(V.shape[-1], F64)
+    return retention_attention_weights(q, K, lam32, pos, t) @ V
+
+
 # ------------------------------------------------------------------ the step loop
 class OracleCache:
     """One sequence's budgeted cache: per-(layer, head) sets of entries, ordered by position.
@@ -254,11 +280,19 @@ class OracleCache:
     def kept_positions(self, layer, head):
         return self.pos[layer][head].copy()
 
-    def decode_attention(self, layer, q):
-        """q [Hq, d] -> o [Hq, d] fp64; query head j reads the pool of KV head j // g."""
+    def decode_attention(self, layer, q, retention_bias=False):
+        """q [Hq, d] -> o [Hq, d] fp64; query head j reads the pool of KV head j // g.
+
+        retention_bias: use the retention-gated weights of Sec. 2.2 (beta_i^(t-i) e^{z_i}) instead of the plain softmax
+        over the retained set (Eq. (1)); t = tokens appended to this layer so far.
+        """
         q = np.asarray(q, F64)
         out = np.zeros((self.Hq, self.d), F64)
         for j in range(self.Hq):
             h = j // self.g
-            out[j] = attention(q[j], self.K[layer][h], self.V[layer][h])
+            if retention_bias:
+                out[j] = retention_attention(q[j], self.K[layer][h], self.V[layer][h], self.lam[layer][h],
+                                             self.pos[layer][h], self.tokens[layer])
+            else:
+                out[j] = attention(q[j], self.K[layer][h], self.V[layer][h])
         return out

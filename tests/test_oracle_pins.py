@@ -335,3 +335,50 @@ def test_corollary_3_2_identity():
     alpha_r = orc.attention_weights(q, K[keep])        # attention over the retained set
     delta_r = 1.0 - alpha_r[useful[keep]].sum()
     assert math.isclose(delta_r, predicted, rel_tol=1e-10, abs_tol=1e-14)
+
+
+# ----------------------------------------------------------------- retention-gated attention: Sec. 2.2
+def test_retention_attention_closed_forms():
+    """alpha~_i = beta_i^(t-i) e^{z_i} / sum_j ...: hand-checkable cases.
+
+    * beta = 1 everywhere (lambda = 0) recovers standard attention (stated in Sec. 2.2);
+    * q = 0 (all z equal): weights are beta_i^(t-i) normalised, here with dyadic beta so the values are exact rationals;
+    * the newest token (i = t) carries weight beta^0 = 1 whatever its beta;
+    * a uniform shift of all ages (same beta) cancels in the normalisation.
+    """
+    d = 8
+    K = rng.normal(size=(5, d)); V = rng.normal(size=(5, d)); q = rng.normal(size=d)
+    pos = np.array([1, 2, 4, 7, 9]); t = 9
+    np.testing.assert_allclose(orc.retention_attention(q, K, V, np.zeros(5, np.float32), pos, t), orc.attention(q, K, V), rtol=1e-13)
+    # q = 0, beta = 1/2: weights 2^-(t-i) normalised: ages 8, 7, 5, 2, 0
+    lam = np.full(5, math.log(0.5), np.float32)
+    w = orc.retention_attention_weights(np.zeros(d), K, lam, pos, t)
+    raw = np.array([2.0 ** -8, 2.0 ** -7, 2.0 ** -5, 2.0 ** -2, 1.0])
+    np.testing.assert_allclose(w, raw / raw.sum(), rtol=1e-6)           # lambda is stored in fp32
+    # two entries, worked by hand: beta_1 = 1/4 at age 1, beta_2 = anything at age 0, z_1 = z_2 + ln 8
+    K2 = np.array([[math.log(8.0) * math.sqrt(2.0), 0.0], [0.0, 0.0]]); q2 = np.array([1.0, 0.0])
+    w2 = orc.retention_attention_weights(q2, K2, np.array([math.log(0.25), -3.0], np.float32), np.array([4, 5]), 5)
+    np.testing.assert_allclose(w2, [2.0 / 3.0, 1.0 / 3.0], rtol=1e-6)   # (1/4 * 8) : 1
+    # same beta everywhere: adding a constant to every age changes nothing
+    lam3 = np.full(5, -0.3, np.float32)
+    a = orc.retention_attention(q, K, V, lam3, pos, t)
+    b = orc.retention_attention(q, K, V, lam3, pos, t + 11)
+    np.testing.assert_allclose(a, b, rtol=1e-9)
+    # smaller beta on an old entry lowers its weight (monotone in beta)
+    lo = orc.retention_attention_weights(q, K, np.array([-2.0, 0, 0, 0, 0], np.float32), pos, t)
+    hi = orc.retention_attention_weights(q, K, np.array([-0.1, 0, 0, 0, 0], np.float32), pos, t)
+    assert lo[0] < hi[0] and abs(lo.sum() - 1) < 1e-12
+
+
+def test_cache_retention_attention_uses_layer_time_and_gqa():
+    c = orc.OracleCache(100, 1, 2, 4, 8)
+    k = rng.normal(size=(6, 2, 8)); v = rng.normal(size=(6, 2, 8))
+    lam = (-rng.uniform(0.01, 0.5, size=(6, 2))).astype(np.float32)
+    c.append(0, k, v, lam=lam)
+    q = rng.normal(size=(4, 8))
+    out = c.decode_attention(0, q, retention_bias=True)
+    for j in range(4):
+        h = j // 2
+        want = orc.retention_attention(q[j], k[:, h], v[:, h], lam[:, h], np.arange(1, 7), 6)
+        np.testing.assert_allclose(out[j], want, rtol=1e-12)
+    assert np.abs(out - c.decode_attention(0, q)).max() > 1e-3
