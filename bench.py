@@ -191,7 +191,7 @@ def run_ours(args, w):
     seed = args.seed + 1000 * rank                      # every rank owns different sequences
     K, W = args.steps, args.warmup
 
-    cache = binding.TrimKV.from_workload(w)
+    cache = binding.TrimKV.from_workload(w, retention_bias=args.retention_bias)
     per_layer, w_g = workloads.gate_params(w, seed, device=dev)
     if args.skew > 0:
         # per-(layer, head) logit offsets through b2 (b2 . w_g shifts s): retention then differs strongly between heads and
@@ -345,6 +345,9 @@ def run_ours(args, w):
         return
     peak, peak_kind = load_peaks()
     ab = algorithmic_bytes(w, entries + w.layers * w.kv_heads)
+    if args.retention_bias:                                        # lambda and position of every entry ride along
+        extra_b = w.batch * (entries + w.layers * w.kv_heads) * 8
+        ab["kv"] += extra_b; ab["total"] += extra_b
     attn_ms_per = live[0] / max(live[1], 1)                       # timed region: beside the gate and the selection
     achieved = ab["kv"] / (attn_ms_per * 1e-3) / 1e9 if attn_ms_per > 0 else 0.0
     iso_ms = phases["attn_main"][0] / max(phases["attn_main"][1], 1)
@@ -361,7 +364,7 @@ def run_ours(args, w):
         "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
                    "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
                    "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk,
-                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew,
+                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew, "retention_bias": bool(args.retention_bias),
                    "pool_len_min_max": [int(lens[0].min()), int(lens[0].max())],
                    "parallelism": f"sequences sharded over {world} rank(s), no collective",
                    "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1),
@@ -447,6 +450,8 @@ def main():
     ap.add_argument("--b-g", type=float, default=None, help="override the shared gate bias")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--skew", type=float, default=0.0, help="std of per-(layer, head) gate-logit offsets (ragged pools)")
+    ap.add_argument("--retention-bias", action="store_true",
+                    help="decode attention with the retention-gated weights of Sec. 2.2 (reads 8 more bytes per entry)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
     ap.add_argument("--sweep-max", type=int, default=28)

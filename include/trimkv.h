@@ -75,6 +75,9 @@ typedef struct trimkv_config {
     int32_t reserved;       /* 0; bit 0 = testing aid: distrust the selection's key sample, so that the
                                exact single-CTA redo of the selection runs in every eviction round  */
     int64_t max_pool_pages; /* cap on pages of one (layer, head) pool; 0 = a pool may take all */
+    int32_t retention_bias; /* 0: decode attention is the plain softmax over the retained set (Eq. (1));
+                               1: retention-gated weights beta_i^(t-i) e^{z_i} of Sec. 2.2 (t = tokens seen) */
+    int32_t reserved2;      /* set to 0                                                        */
 } trimkv_config;
 
 /* Fill *cfg with defaults (batch 1, q_heads = kv_heads, bf16, no gate, page 64, d_g 512,

@@ -40,6 +40,7 @@ class Config(C.Structure):
         ("head_dim", C.c_int32), ("hidden", C.c_int32), ("max_batch", C.c_int32), ("page_size", C.c_int32),
         ("gate_hidden", C.c_int32), ("gate_embed", C.c_int32), ("horizon", C.c_int32), ("kv_dtype", C.c_int32),
         ("max_chunk", C.c_int32), ("reserved", C.c_int32), ("max_pool_pages", C.c_int64),
+        ("retention_bias", C.c_int32), ("reserved2", C.c_int32),
     ]
 
 
@@ -131,7 +132,8 @@ class TrimKV:
 
     def __init__(self, budget_entries: int, layers: int, kv_heads: int, head_dim: int, *, q_heads: Optional[int] = None,
                  hidden: int = 0, batch: int = 1, gate_hidden: int = 512, gate_embed: int = 64, horizon: int = 2,
-                 kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0, distrust_sample: bool = False):
+                 kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0, distrust_sample: bool = False,
+                 retention_bias: bool = False):
         L = lib()
         cfg = Config()
         L.trimkv_default_config(C.byref(cfg), budget_entries, layers, kv_heads, head_dim)
@@ -144,6 +146,7 @@ class TrimKV:
         cfg.kv_dtype = {"bf16": DTYPE_BF16, "f32": DTYPE_F32}[kv_dtype]
         cfg.max_chunk = max_chunk
         cfg.max_pool_pages = max_pool_pages
+        cfg.retention_bias = 1 if retention_bias else 0
         cfg.reserved = 1 if distrust_sample else 0     # testing aid: forces the selection's exact redo path
         self.cfg = cfg
         self.torch_dtype = torch.bfloat16 if kv_dtype == "bf16" else torch.float32

@@ -30,7 +30,9 @@ constexpr int ATT_BAR_OFF = ATT_WARPS * ATT_STAGES * STAGE_BYTES;
 constexpr int ATT_GRP_OFF = ATT_BAR_OFF + 256;
 constexpr int ATT_RING = 8;                    // per-warp queue of item ids fetched by the producer, read by the consumer
 constexpr int ATT_RING_OFF = ATT_GRP_OFF + (ATT_GROUPS + 1) * 4 + 12;
-constexpr int ATT_SMEM = ATT_RING_OFF + ATT_WARPS * ATT_RING * 4;
+constexpr int ATT_META_OFF = (ATT_RING_OFF + ATT_WARPS * ATT_RING * 4 + 127) & ~127;   // per warp and stage: lambda[32], pos[32]
+constexpr int ATT_META_BYTES = 2 * TILE * 4;
+constexpr int ATT_SMEM = ATT_META_OFF + ATT_WARPS * ATT_STAGES * ATT_META_BYTES;
 constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -123,9 +125,11 @@ __device__ __forceinline__ int tiles_per_item(int len, int items) {
     return (((tiles + items - 1) / items) + 1) & ~1;
 }
 
-template <int NT>   // NT = ceil(g / 8): column tiles of 8 query heads
+// NT = ceil(g / 8): column tiles of 8 query heads.  BIAS: retention-gated weights beta_i^(t-i) e^{z_i} (Sec. 2.2): the
+// entries' lambda and position travel with each tile and (t_now - pos) * lambda is added to the logit.
+template <int NT, bool BIAS>
 __global__ void __launch_bounds__(ATT_WARPS * 32, 1)
-attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, int Hq, int32_t* __restrict__ pool_done,
+attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, int Hq, int t_now, int32_t* __restrict__ pool_done,
                 int32_t* __restrict__ sched,
                 const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ part_o,
                 float* __restrict__ part_ml, float scale_log2, long long max_items) {
@@ -135,6 +139,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + ATT_BAR_OFF) + warp * ATT_STAGES;
     int* grp = reinterpret_cast<int*>(smem_raw + ATT_GRP_OFF);     // grp[i] = items before pool group i
     volatile int* ring = reinterpret_cast<volatile int*>(smem_raw + ATT_RING_OFF) + warp * ATT_RING;
+    unsigned char* meta = smem_raw + ATT_META_OFF + (size_t)warp * ATT_STAGES * ATT_META_BYTES;
 
     // ---- item table: items per group of gsz pools, then an exclusive scan (every CTA computes the same table)
     const int ngrp = (n_scope + gsz - 1) / gsz;
@@ -246,9 +251,14 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
             const char* ksrc = cv.kv + kv_row_offset(cv, prod.b, page, 0, half * TILE);
             const char* vsrc = cv.kv + kv_row_offset(cv, prod.b, page, 1, half * TILE);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_expect_tx(bars + s, STAGE_BYTES);
+            mbar_expect_tx(bars + s, STAGE_BYTES + (BIAS ? ATT_META_BYTES : 0));
             bulk_g2s(dst, ksrc, TILE * ROWB, bars + s);
             bulk_g2s(dst + TILE * ROWB, vsrc, TILE * ROWB, bars + s);
+            if (BIAS) {
+                const size_t slot0 = ((size_t)prod.b * cv.P_seq + page) * PAGE + half * TILE;
+                bulk_g2s(meta + s * ATT_META_BYTES, cv.lam + slot0, TILE * 4, bars + s);
+                bulk_g2s(meta + s * ATT_META_BYTES + TILE * 4, cv.pos + slot0, TILE * 4, bars + s);
+            }
         }
         ++issued;
         if (++prod_tile == prod.ntile) {
@@ -305,6 +315,18 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
             const uint32_t kbase = smem_u32(wbuf + (size_t)s * STAGE_BYTES);
             const uint32_t vbase = kbase + TILE * ROWB;
             const int valid = min(TILE, cons.len - (cons.first_tile + tt) * TILE);
+            float rb[2][2] = {{0.f, 0.f}, {0.f, 0.f}};           // log2-domain retention bias of this thread's four rows
+            if (BIAS) {
+                const float* mlam = reinterpret_cast<const float*>(meta + s * ATT_META_BYTES);
+                const int* mpos = reinterpret_cast<const int*>(meta + s * ATT_META_BYTES + TILE * 4);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int r = mt * 16 + hh * 8 + (lane >> 2);
+                        rb[mt][hh] = (float)(t_now - mpos[r]) * mlam[r] * 1.4426950408889634f;
+                    }
+            }
 
             // ---- S^T[entry][head] = K Q^T
             float sacc[2][NT][4];
@@ -333,10 +355,10 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
                 for (int mt = 0; mt < 2; ++mt) {
                     const int r0 = mt * 16 + (lane >> 2);
                     float* sc = sacc[mt][nt];
-                    sc[0] = (r0 < valid) ? sc[0] * scale_log2 : -INFINITY;
-                    sc[1] = (r0 < valid) ? sc[1] * scale_log2 : -INFINITY;
-                    sc[2] = (r0 + 8 < valid) ? sc[2] * scale_log2 : -INFINITY;
-                    sc[3] = (r0 + 8 < valid) ? sc[3] * scale_log2 : -INFINITY;
+                    sc[0] = (r0 < valid) ? sc[0] * scale_log2 + rb[mt][0] : -INFINITY;
+                    sc[1] = (r0 < valid) ? sc[1] * scale_log2 + rb[mt][0] : -INFINITY;
+                    sc[2] = (r0 + 8 < valid) ? sc[2] * scale_log2 + rb[mt][1] : -INFINITY;
+                    sc[3] = (r0 + 8 < valid) ? sc[3] * scale_log2 + rb[mt][1] : -INFINITY;
                     mx0 = fmaxf(mx0, fmaxf(sc[0], sc[2]));
                     mx1 = fmaxf(mx1, fmaxf(sc[1], sc[3]));
                 }
@@ -571,7 +593,7 @@ __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { retu
 template <typename T, int MAXD>
 __global__ void __launch_bounds__(128)
 attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T* __restrict__ q, T* __restrict__ out,
-                  float scale) {
+                  float scale, int bias, int t_now) {
     const int wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (wid >= n_scope * g) return;
@@ -606,6 +628,10 @@ attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T*
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (bias) {                                       // retention-gated weights: + (t - i) * lambda_i
+            const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + off;
+            s += (float)(t_now - cv.pos[slot]) * cv.lam[slot];
+        }
         const float mn = fmaxf(m, s);
         const float f = __expf(m - mn), p = __expf(s - mn);
         l = l * f + p;
@@ -627,16 +653,18 @@ attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T*
 }  // namespace
 
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
-                      long long tiles_estimate, long long tiles_upper, const void* q, void* out, cudaStream_t st,
-                      PhaseMarker* pm) {
+                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, const void* q,
+                      void* out, cudaStream_t st, PhaseMarker* pm) {
     const int n_scope = nlayers * cv.B * cv.H;
     const int g = Hq / cv.H;
     const float scale = 1.0f / sqrtf((float)cv.d);
     if (is_bf16 && cv.d == 128 && g <= 16) {
         static bool attr_set = false;
         if (!attr_set) {
-            cudaFuncSetAttribute(attn_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
-            cudaFuncSetAttribute(attn_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            cudaFuncSetAttribute(attn_mma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            cudaFuncSetAttribute(attn_mma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            cudaFuncSetAttribute(attn_mma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
+            cudaFuncSetAttribute(attn_mma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
             attr_set = true;
         }
         int dev = 0, sms = 148;
@@ -656,14 +684,13 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         while ((n_scope + gsz - 1) / gsz > ATT_GROUPS) gsz <<= 1;
         if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
         const float scale_log2 = scale * 1.4426950408889634f;
-        if (g <= 8)
-            attn_mma_kernel<1><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done, ab.sched,
-                                                                      (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
-                                                                      ab.part_o, ab.part_ml, scale_log2, ab.max_items);
-        else
-            attn_mma_kernel<2><<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, ab.pool_done, ab.sched,
-                                                                      (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
-                                                                      ab.part_o, ab.part_ml, scale_log2, ab.max_items);
+        auto launch = [&](auto kernel) {
+            kernel<<<sms, ATT_WARPS * 32, ATT_SMEM, st>>>(cv, layer0, n_scope, (int)tpi, gsz, g, Hq, (int)t_now, ab.pool_done, ab.sched,
+                                                          (const __nv_bfloat16*)q, (__nv_bfloat16*)out, ab.part_o, ab.part_ml,
+                                                          scale_log2, ab.max_items);
+        };
+        if (g <= 8) { if (retention_bias) launch(attn_mma_kernel<1, true>); else launch(attn_mma_kernel<1, false>); }
+        else        { if (retention_bias) launch(attn_mma_kernel<2, true>); else launch(attn_mma_kernel<2, false>); }
         if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
         count_launch(1);
     } else {
@@ -672,10 +699,10 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
         if (is_bf16)
             attn_plain_kernel<__nv_bfloat16, 256><<<grid, 128, 0, st>>>(cv, layer0, n_scope, g, Hq, (const __nv_bfloat16*)q,
-                                                                         (__nv_bfloat16*)out, scale);
+                                                                         (__nv_bfloat16*)out, scale, retention_bias, (int)t_now);
         else
             attn_plain_kernel<float, 256><<<grid, 128, 0, st>>>(cv, layer0, n_scope, g, Hq, (const float*)q, (float*)out,
-                                                                scale);
+                                                                scale, retention_bias, (int)t_now);
         if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
         count_launch();
     }

@@ -188,9 +188,10 @@ struct PhaseMarker {
     virtual ~PhaseMarker() {}
 };
 
+// retention_bias != 0: retention-gated weights beta_i^(t_now - i) e^{z_i} instead of the plain softmax.
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
-                      long long tiles_estimate, long long tiles_upper, const void* q, void* out, cudaStream_t st,
-                      PhaseMarker* pm);
+                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, const void* q,
+                      void* out, cudaStream_t st, PhaseMarker* pm);
 
 void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
                         void* v, int n, cudaStream_t st);

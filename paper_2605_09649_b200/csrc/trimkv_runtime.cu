@@ -223,8 +223,8 @@ trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
 trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, void* out, cudaStream_t st) {
     const long long tiles = (h->entries * h->B / 32) * nlayers / h->L + (long long)nlayers * h->B * h->H;
     const long long tiles_upper = h->entries * h->B / 32 + (long long)nlayers * h->B * h->H;
-    launch_attention(h->cv, h->ab, layer0, nlayers, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, tiles, tiles_upper, q,
-                     out, st, h->prof.on ? &h->prof : nullptr);
+    launch_attention(h->cv, h->ab, layer0, nlayers, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, tiles, tiles_upper,
+                     h->cfg.retention_bias, h->tokens[layer0], q, out, st, h->prof.on ? &h->prof : nullptr);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
 }

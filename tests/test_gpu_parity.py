@@ -344,6 +344,45 @@ def test_multi_turn_dialogue_flow_matches_oracle():
     pair.close()
 
 
+@pytest.mark.parametrize("kv_dtype,atol", [("bf16", ATT_ATOL_BF16), ("f32", ATT_ATOL_F32)])
+def test_retention_gated_attention_option(kv_dtype, atol):
+    """retention_bias: weights beta_i^(t-i) e^{z_i} (Sec. 2.2) instead of the plain softmax; strong decay so that the bias
+    matters; chunks, evictions and decode steps as in the plain case; and lambda = 0 gives the plain result."""
+    d = 128 if kv_dtype == "bf16" else 64
+    w = workloads.Workload("soft", 2, 2, 8, d, 0, 2, 333, kv_dtype, 0, 0, 160)
+    dt = workloads.torch_dtype(kv_dtype)
+    pair = Pair(w, retention_bias=True)
+    plain = binding.TrimKV.from_workload(w)
+    r = np.random.default_rng(23)
+    g = torch.Generator(device=DEV); g.manual_seed(23)
+    worst_gap = 0.0
+    for n in (150, 97, 1, 1, 1, 40):
+        for l in range(w.layers):
+            k = torch.randn(w.batch, n, w.kv_heads, d, generator=g, device=DEV).to(dt)
+            v = torch.randn(w.batch, n, w.kv_heads, d, generator=g, device=DEV).to(dt)
+            lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), scale=0.05)
+            c = oracle_retention(lam, w.horizon)
+            pair.append(l, k, v, lam, c)
+            plain.append(l, k, v, lam=torch.from_numpy(lam).to(DEV), c=torch.from_numpy(c).to(DEV))
+            q = torch.randn(w.batch, w.q_heads, d, generator=g, device=DEV).to(dt)
+            out = pair.check_attention(l, q, atol)
+            worst_gap = max(worst_gap, float((out.float() - plain.decode_attention(l, q).float()).abs().max()))
+        pair.evict(); plain.score_and_evict()
+        pair.check_sets()
+    assert worst_gap > 0.05                       # the option really changes the result
+    pair.close(); plain.close()
+    # lambda = 0: identical to the plain softmax
+    a = binding.TrimKV.from_workload(w, retention_bias=True)
+    b = binding.TrimKV.from_workload(w)
+    k = torch.randn(w.batch, 70, w.kv_heads, d, generator=g, device=DEV).to(dt)
+    z = torch.zeros(w.batch, 70, w.kv_heads, device=DEV)
+    q = torch.randn(w.batch, w.q_heads, d, generator=g, device=DEV).to(dt)
+    for cch in (a, b):
+        cch.append(0, k, k, lam=z)
+    assert torch.equal(a.decode_attention(0, q), b.decode_attention(0, q))
+    a.close(); b.close()
+
+
 def test_step_all_matches_layerwise_oracle():
     w = BF16_SMALL.replace(budget_entries=400)
     lam_fn = lambda r, shape, l: random_lambda(shape, int(r.integers(1 << 30)))

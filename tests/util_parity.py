@@ -18,6 +18,7 @@ class Pair:
     def __init__(self, w: workloads.Workload, device="cuda", oracle_seqs=None, oracle_kv=True, **overrides):
         self.w = w
         self.dev = device
+        self.retention_bias = bool(overrides.get("retention_bias", False))
         self.gpu = binding.TrimKV.from_workload(w, **overrides)
         self.seqs = list(range(w.batch)) if oracle_seqs is None else list(oracle_seqs)
         self.oracle_kv = oracle_kv
@@ -64,7 +65,7 @@ class Pair:
         out = self.gpu.decode_attention(layer, q)
         got = to_np(out)
         for b in self.seqs:
-            want = self.orc[b].decode_attention(layer, to_np(q[b]))
+            want = self.orc[b].decode_attention(layer, to_np(q[b]), retention_bias=self.retention_bias)
             err = np.abs(got[b] - want).max()
             assert err <= atol, f"attention error {err} > {atol} in sequence {b}, layer {layer}"
         return out
