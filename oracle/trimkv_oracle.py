@@ -183,8 +183,11 @@ class OracleCache:
     never return (monotone r, Eq. (1)).
     """
 
-    def __init__(self, budget, layers, kv_heads, q_heads, head_dim, horizon=2):
+    def __init__(self, budget, layers, kv_heads, q_heads, head_dim, horizon=2, per_pool_budget=0):
         self.budget = int(budget)
+        # > 0: the fixed-budget variant the paper compares with (TrimKV, Sec. 2.2 / 5.2: a budget of M entries for
+        # each attention head instead of one global budget): every pool keeps its own M best entries
+        self.per_pool_budget = int(per_pool_budget)
         self.L, self.H, self.Hq, self.d = int(layers), int(kv_heads), int(q_heads), int(head_dim)
         assert self.Hq % self.H == 0
         self.g = self.Hq // self.H
@@ -253,6 +256,21 @@ class OracleCache:
         t = self.tokens[0]
         if any(tt != t for tt in self.tokens):
             raise RuntimeError("layers hold different token counts")
+        if self.per_pool_budget > 0:
+            evicted = 0
+            for l in range(self.L):
+                for h in range(self.H):
+                    m = len(self.pos[l][h])
+                    if m <= self.per_pool_budget:
+                        continue
+                    S = score(self.lam[l][h], self.c[l][h], self.pos[l][h], t)
+                    z = np.zeros(m, np.int64)
+                    keep = select_keep(S, self.pos[l][h], z, z, self.per_pool_budget)
+                    for name in ("pos", "lam", "c", "K", "V"):
+                        arr = getattr(self, name)
+                        arr[l][h] = arr[l][h][keep]
+                    evicted += m - self.per_pool_budget
+            return evicted
         n = self.total_entries()
         if n <= self.budget:
             return 0

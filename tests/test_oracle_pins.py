@@ -382,3 +382,29 @@ def test_cache_retention_attention_uses_layer_time_and_gqa():
         want = orc.retention_attention(q[j], k[:, h], v[:, h], lam[:, h], np.arange(1, 7), 6)
         np.testing.assert_allclose(out[j], want, rtol=1e-12)
     assert np.abs(out - c.decode_attention(0, q)).max() > 1e-3
+
+
+def test_per_pool_budget_variant():
+    """Fixed per-head budget (the TrimKV arm): each pool keeps its own M best entries, independently of the others.
+    Equal retention in a pool => that pool keeps its last M positions; a pool with slowly decaying old entries keeps
+    them; brute force per pool; pools never exceed M while the global variant moves capacity between them."""
+    L, H, M = 2, 2, 5
+    c = orc.OracleCache(10 ** 9, L, H, H, 0, horizon=1, per_pool_budget=M)
+    g = orc.OracleCache(M * L * H, L, H, H, 0, horizon=1)
+    n = 12
+    lam = np.full((n, H), -0.1, np.float32)
+    lam[:, 1] = -2.0                                   # head 1 forgets fast
+    lam[0:3, 1] = -1e-4                                # ... except its three oldest tokens
+    kv = np.zeros((n, H, 0))
+    for cache in (c, g):
+        for l in range(L):
+            cache.append(l, kv, kv, lam=lam)
+        cache.score_and_evict()
+    for l in range(L):
+        assert c.kept_positions(l, 0).tolist() == [8, 9, 10, 11, 12]          # sliding window
+        assert c.kept_positions(l, 1).tolist() == [1, 2, 3, 11, 12]           # durable old tokens + the newest
+        S = orc.score(lam[:, 1], orc.horizon_term_from_lambda32(lam[:, 1], 1), np.arange(1, n + 1), n)
+        want = sorted(np.argsort(-S.astype(np.float64), kind="stable")[:M] + 1)
+        assert c.kept_positions(l, 1).tolist() == want
+    assert (c.lengths() == M).all()
+    assert g.lengths().sum() == M * L * H and (g.lengths() != M).any()        # the global budget reallocates
