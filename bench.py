@@ -191,7 +191,8 @@ def run_ours(args, w):
     seed = args.seed + 1000 * rank                      # every rank owns different sequences
     K, W = args.steps, args.warmup
 
-    cache = binding.TrimKV.from_workload(w, retention_bias=args.retention_bias)
+    per_pool = w.budget_entries // (w.layers * w.kv_heads) if args.fixed_budget else 0
+    cache = binding.TrimKV.from_workload(w, retention_bias=args.retention_bias, per_pool_budget=per_pool)
     per_layer, w_g = workloads.gate_params(w, seed, device=dev)
     if args.skew > 0:
         # per-(layer, head) logit offsets through b2 (b2 . w_g shifts s): retention then differs strongly between heads and
@@ -339,6 +340,7 @@ def run_ours(args, w):
     cache.sync_status()
     lens = cache.lengths()
     assert int(lens[0].sum()) == min(w.budget_entries, entries), "budget invariant violated"
+    assert per_pool == 0 or int(lens.max()) <= per_pool
 
     if rank != 0:
         cache.close()
@@ -364,7 +366,7 @@ def run_ours(args, w):
         "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
                    "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
                    "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk,
-                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew, "retention_bias": bool(args.retention_bias),
+                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew, "retention_bias": bool(args.retention_bias), "fixed_per_pool_budget": per_pool,
                    "pool_len_min_max": [int(lens[0].min()), int(lens[0].max())],
                    "parallelism": f"sequences sharded over {world} rank(s), no collective",
                    "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1),
@@ -452,6 +454,8 @@ def main():
     ap.add_argument("--skew", type=float, default=0.0, help="std of per-(layer, head) gate-logit offsets (ragged pools)")
     ap.add_argument("--retention-bias", action="store_true",
                     help="decode attention with the retention-gated weights of Sec. 2.2 (reads 8 more bytes per entry)")
+    ap.add_argument("--fixed-budget", action="store_true",
+                    help="the fixed per-head budget variant (every pool keeps budget / (layers * kv_heads) entries)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
     ap.add_argument("--sweep-max", type=int, default=28)

@@ -77,7 +77,9 @@ typedef struct trimkv_config {
     int64_t max_pool_pages; /* cap on pages of one (layer, head) pool; 0 = a pool may take all */
     int32_t retention_bias; /* 0: decode attention is the plain softmax over the retained set (Eq. (1));
                                1: retention-gated weights beta_i^(t-i) e^{z_i} of Sec. 2.2 (t = tokens seen) */
-    int32_t reserved2;      /* set to 0                                                        */
+    int32_t per_pool_budget; /* 0: one global budget per sequence (the paper's method).  > 0: the fixed-budget variant it is
+                               compared with (TrimKV): every (layer, head) pool keeps its own per_pool_budget best
+                               entries; budget_entries (>= per_pool_budget x layers x kv_heads) then only sizes the cache */
 } trimkv_config;
 
 /* Fill *cfg with defaults (batch 1, q_heads = kv_heads, bf16, no gate, page 64, d_g 512,

@@ -40,7 +40,7 @@ class Config(C.Structure):
         ("head_dim", C.c_int32), ("hidden", C.c_int32), ("max_batch", C.c_int32), ("page_size", C.c_int32),
         ("gate_hidden", C.c_int32), ("gate_embed", C.c_int32), ("horizon", C.c_int32), ("kv_dtype", C.c_int32),
         ("max_chunk", C.c_int32), ("reserved", C.c_int32), ("max_pool_pages", C.c_int64),
-        ("retention_bias", C.c_int32), ("reserved2", C.c_int32),
+        ("retention_bias", C.c_int32), ("per_pool_budget", C.c_int32),
     ]
 
 
@@ -133,7 +133,7 @@ class TrimKV:
     def __init__(self, budget_entries: int, layers: int, kv_heads: int, head_dim: int, *, q_heads: Optional[int] = None,
                  hidden: int = 0, batch: int = 1, gate_hidden: int = 512, gate_embed: int = 64, horizon: int = 2,
                  kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0, distrust_sample: bool = False,
-                 retention_bias: bool = False):
+                 retention_bias: bool = False, per_pool_budget: int = 0):
         L = lib()
         cfg = Config()
         L.trimkv_default_config(C.byref(cfg), budget_entries, layers, kv_heads, head_dim)
@@ -147,6 +147,7 @@ class TrimKV:
         cfg.max_chunk = max_chunk
         cfg.max_pool_pages = max_pool_pages
         cfg.retention_bias = 1 if retention_bias else 0
+        cfg.per_pool_budget = per_pool_budget
         cfg.reserved = 1 if distrust_sample else 0     # testing aid: forces the selection's exact redo path
         self.cfg = cfg
         self.torch_dtype = torch.bfloat16 if kv_dtype == "bf16" else torch.float32

@@ -1009,6 +1009,126 @@ seed_range_kernel(const float* __restrict__ s, long long n, SelState* __restrict
     }
 }
 
+// ------------------------------------------------------------------ fixed per-pool budget (TrimKV arm)
+// One CTA per pool: the pool keeps its `keep` best entries on its own.  The keys of the pool (up to 8192; longer pools
+// re-read their metadata every sweep) sit in registers; a radix descent over the bits in which they differ finds the
+// k-th smallest key exactly, then every entry with a key up to it is flagged in its page's eviction mask.
+__global__ void __launch_bounds__(256)
+pool_select_kernel(CacheView cv, long long t1, int keep) {
+    constexpr int DB = 9, NBIN = 1 << DB, PER = 32;
+    __shared__ unsigned hist[NBIN];
+    __shared__ unsigned wtot[8];
+    __shared__ u64 s_or[8], s_and[8];
+    __shared__ u64 s_prefix;
+    __shared__ long long s_r;
+    __shared__ int s_found;
+    const long long pool = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = (int)(pool / ((long long)cv.L * cv.H));
+    const int pool_local = (int)(pool % ((long long)cv.L * cv.H));
+    const int n = cv.len[pool];
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    u64* masks = cv.evict_mask + (size_t)b * cv.P_seq;
+    const int np = (n + PAGE - 1) / PAGE;
+    for (int lp = tid; lp < np; lp += blockDim.x) masks[bt[lp]] = 0ull;
+    if (n <= keep) return;
+    long long r = n - keep;                                      // evict the r smallest keys
+    const int t1i = (int)t1;
+    auto key_of = [&](int idx) -> u64 {
+        const size_t slot = ((size_t)b * cv.P_seq + bt[idx / PAGE]) * PAGE + idx % PAGE;
+        const int pos = cv.pos[slot];
+        const float S = retention_score(cv.lam[slot], cv.c[slot], (float)(t1i - pos));
+        if (S != S) latch_error(cv.err, TRIMKV_E_NONFINITE);
+        return make_key(S, ((uint32_t)pos << cv.pool_bits) | (uint32_t)pool_local);
+    };
+    const bool inreg = n <= PER * 256;
+    u64 kr[PER];
+    u64 vor = 0ull, vand = ~0ull;
+    if (inreg) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int idx = tid + i * 256;
+            kr[i] = 0ull;
+            if (idx < n) { kr[i] = key_of(idx); vor |= kr[i]; vand &= kr[i]; }
+        }
+    } else {
+        for (int idx = tid; idx < n; idx += 256) { const u64 k = key_of(idx); vor |= k; vand &= k; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        vor |= __shfl_xor_sync(0xffffffffu, vor, o);
+        vand &= __shfl_xor_sync(0xffffffffu, vand, o);
+    }
+    if (lane == 0) { s_or[warp] = vor; s_and[warp] = vand; }
+    __syncthreads();
+    vor = 0ull; vand = ~0ull;
+    for (int w = 0; w < 8; ++w) { vor |= s_or[w]; vand &= s_and[w]; }
+    const u64 diff = vor ^ vand;
+    int top = diff ? 64 - __clzll((long long)diff) : 0;
+    u64 prefix = top >= 64 ? 0ull : (vor >> top);
+    while (top > 0) {
+        const int dbits = top < DB ? top : DB;
+        const int sh = top - dbits;
+        hist[tid] = 0u;
+        hist[tid + 256] = 0u;
+        if (tid == 0) s_found = 0;
+        __syncthreads();
+        auto count = [&](u64 key) {
+            const bool match = top >= 64 ? true : ((key >> top) == prefix);
+            if (match) atomicAdd(&hist[(unsigned)((key >> sh) & ((1u << dbits) - 1u))], 1u);
+        };
+        if (inreg) {
+#pragma unroll
+            for (int i = 0; i < PER; ++i)
+                if (tid + i * 256 < n) count(kr[i]);
+        } else {
+            for (int idx = tid; idx < n; idx += 256) count(key_of(idx));
+        }
+        __syncthreads();
+        const unsigned h0 = hist[2 * tid], h1 = hist[2 * tid + 1];
+        unsigned incl = h0 + h1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned tt = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += tt;
+        }
+        if (lane == 31) wtot[warp] = incl;
+        __syncthreads();
+        unsigned off = 0;
+        for (int w = 0; w < warp; ++w) off += wtot[w];
+        const long long excl = (long long)off + incl - (h0 + h1);
+        if (r > excl && r <= excl + h0) {
+            s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid);
+            s_r = r - excl;
+            s_found = 1;
+        } else if (r > excl + h0 && r <= excl + h0 + h1) {
+            s_prefix = (top >= 64 ? 0ull : (prefix << dbits)) | (u64)(2 * tid + 1);
+            s_r = r - excl - h0;
+            s_found = 1;
+        }
+        __syncthreads();
+        if (!s_found) {                                          // cannot happen: the counts cover all n keys
+            if (tid == 0) latch_error(cv.err, TRIMKV_E_STATE);
+            return;
+        }
+        prefix = s_prefix;
+        r = s_r;
+        top = sh;
+        __syncthreads();
+    }
+    const u64 tau = prefix;                                      // the r-th smallest key of the pool
+    auto flag = [&](int idx, u64 key) {
+        if (key <= tau) atomicOr(masks + bt[idx / PAGE], 1ull << (idx % PAGE));
+    };
+    if (inreg) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i)
+            if (tid + i * 256 < n) flag(tid + i * 256, kr[i]);
+    } else {
+        for (int idx = tid; idx < n; idx += 256) flag(idx, key_of(idx));
+    }
+}
+
 __global__ void state_init_kernel(SelState* sel, int B) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
@@ -1079,6 +1199,13 @@ void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long
                                                  sb.stats, compact_cursor, cv.err);
     redo_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, cv.evict_mask, cv.P_seq, k_evict, cv.err);
     count_launch(5);
+}
+
+void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st) {
+    const long long pools = (long long)cv.B * cv.L * cv.H;
+    cudaMemsetAsync(compact_cursor, 0, (size_t)cv.B * sizeof(int32_t), st);
+    pool_select_kernel<<<(unsigned)pools, 256, 0, st>>>(cv, t + 1, keep_per_pool);
+    count_launch();
 }
 
 void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,

@@ -165,6 +165,8 @@ struct SelectBuffers {
 // compact_cursor [B]: zeroed by the selection for the compaction that follows.
 void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, long long k_evict,
                          int32_t* compact_cursor, int distrust_sample, cudaStream_t st);
+// Fixed per-pool budget: every pool keeps its keep_per_pool best entries (masks as for launch_select_cache).
+void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st);
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max, cudaStream_t st);
 
 void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,

@@ -191,11 +191,24 @@ trimkv_status gate_ready(const trimkv* h, int layer0, int nlayers) {
     return TRIMKV_OK;
 }
 
+// Entries per sequence to evict now: global budget, or (fixed per-pool budget: every pool holds the same number of
+// entries, one per token seen, cut back to the budget at each eviction) the excess of the pools.
+long long eviction_due(const trimkv* h) {
+    if (h->cfg.per_pool_budget > 0) {
+        const long long per_pool = h->entries / ((long long)h->L * h->H);
+        return std::max<long long>(0, per_pool - h->cfg.per_pool_budget) * h->L * h->H;
+    }
+    return h->entries - h->M;
+}
+
 // Selection on `sel_st`, compaction on `st`; when the two differ the caller orders them with events.
 trimkv_status select_impl(trimkv* h, long long k, cudaStream_t sel_st) {
     PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
     if (pm) pm->mark(PH_SELECT, 0, sel_st);
-    launch_select_cache(h->cv, h->sb, h->tokens[0], h->entries, k, h->cursor, h->cfg.reserved & 1, sel_st);
+    if (h->cfg.per_pool_budget > 0)
+        launch_select_pools(h->cv, h->tokens[0], h->cfg.per_pool_budget, h->cursor, sel_st);
+    else
+        launch_select_cache(h->cv, h->sb, h->tokens[0], h->entries, k, h->cursor, h->cfg.reserved & 1, sel_st);
     if (pm) pm->mark(PH_SELECT, 1, sel_st);
     return TRIMKV_OK;
 }
@@ -205,7 +218,7 @@ trimkv_status compact_impl(trimkv* h, cudaStream_t st) {
     if (pm) pm->mark(PH_COMPACT, 0, st);
     launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
     if (pm) pm->mark(PH_COMPACT, 1, st);
-    h->entries = h->M;
+    h->entries -= eviction_due(h);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
 }
@@ -214,7 +227,7 @@ trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
     const long long t = h->tokens[0];
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layer %d holds %lld tokens, layer 0 holds %lld", l, h->tokens[l], t);
-    const long long k = h->entries - h->M;
+    const long long k = eviction_due(h);
     if (k <= 0) return TRIMKV_OK;
     select_impl(h, k, st);
     return compact_impl(h, st);
@@ -275,6 +288,9 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         return fail(TRIMKV_E_ARG, "hidden and gate_hidden must be multiples of 4, gate_embed positive");
     if (cfg->hidden > 0 && cfg->gate_hidden > 1536) return fail(TRIMKV_E_UNSUPPORTED, "gate_hidden must be at most 1536");
     if ((long long)cfg->layers * cfg->kv_heads > 65536) return fail(TRIMKV_E_UNSUPPORTED, "layers * kv_heads too large");
+    if (cfg->per_pool_budget < 0 || (cfg->per_pool_budget > 0 &&
+                                     (long long)cfg->per_pool_budget * cfg->layers * cfg->kv_heads > cfg->budget_entries))
+        return fail(TRIMKV_E_ARG, "per_pool_budget * layers * kv_heads must not exceed budget_entries (which sizes the cache)");
 
     trimkv* h = new (std::nothrow) trimkv();
     if (!h) return fail(TRIMKV_E_NOMEM, "host allocation failed");
@@ -514,7 +530,7 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
     if (two) CUDA_TRY(cudaEventRecord(h->ev_append, fs));
     for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
     h->entries += (long long)h->L * h->H;
-    const long long kev = h->entries - h->M;
+    const long long kev = eviction_due(h);
     trimkv_status s = attention_impl(h, 0, h->L, q, out, fs);
 
     const float* lam = lambda;

@@ -383,6 +383,38 @@ def test_retention_gated_attention_option(kv_dtype, atol):
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("horizon,per_pool", [(1, 50), (2, 64), (1, 700)])
+def test_fixed_per_pool_budget_variant(horizon, per_pool):
+    """The fixed-budget arm (every pool keeps its own M best entries; horizon 1 = the myopic score beta^(t+1-i)):
+    kept sets bit-exact against the oracle through chunks and decode steps, pools never above M, attention in tolerance;
+    with M = 700 the pool's keys exceed one page run and tails."""
+    w = BF16_SMALL.replace(horizon=horizon, budget_entries=per_pool * 6, batch=2, chunk=160)
+    pair = Pair(w, per_pool_budget=per_pool)
+    r = np.random.default_rng(31)
+    g = torch.Generator(device=DEV); g.manual_seed(31)
+    dt = torch.bfloat16
+    for n in (160, 160, 160, 160, 97, 1, 1, 1):
+        for l in range(w.layers):
+            k = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+            v = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+            lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), distinct=0 if n > 1 else 3, scale=0.05)
+            pair.append(l, k, v, lam, oracle_retention(lam, w.horizon))
+            if n == 1:
+                q = torch.randn(w.batch, w.q_heads, w.head_dim, generator=g, device=DEV).to(dt)
+                pair.check_attention(l, q, ATT_ATOL_BF16)
+        pair.evict()
+        pair.check_sets()
+        assert int(pair.gpu.lengths().max()) <= per_pool
+    # the whole step in one call as well
+    K = torch.randn(w.layers, w.batch, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+    Q = torch.randn(w.layers, w.batch, w.q_heads, w.head_dim, generator=g, device=DEV).to(dt)
+    lam = -torch.rand(w.layers, w.batch, w.kv_heads, generator=g, device=DEV) * 0.05
+    pair.gpu.decode_step_all(K, K, Q, torch.empty_like(Q), lam=lam)
+    assert int(pair.gpu.lengths().max()) <= per_pool and int(pair.gpu.lengths().min()) == min(per_pool, 160 * 4 + 97 + 4)
+    pair.gpu.sync_status()
+    pair.close()
+
+
 def test_step_all_matches_layerwise_oracle():
     w = BF16_SMALL.replace(budget_entries=400)
     lam_fn = lambda r, shape, l: random_lambda(shape, int(r.integers(1 << 30)))

@@ -23,7 +23,8 @@ class Pair:
         self.seqs = list(range(w.batch)) if oracle_seqs is None else list(oracle_seqs)
         self.oracle_kv = oracle_kv
         d = w.head_dim if oracle_kv else 0
-        self.orc = {b: orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, d, horizon=w.horizon)
+        self.orc = {b: orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, d, horizon=w.horizon,
+                                       per_pool_budget=int(overrides.get("per_pool_budget", 0)))
                     for b in self.seqs}
 
     def close(self):
