@@ -2,13 +2,19 @@
 // S = (t + 1 - i) * lambda + c  (log of Eq. (global_score)) under the total order
 // (score, then newer position first, then higher layer, then higher head are evicted first).
 //
-// Method: every entry maps to a unique 64-bit key whose integer order is the eviction order.  A
-// histogram pass over all keys (shared-memory histogram per CTA, 4094 equal-width bins over a key range
-// centred on the previous call's threshold) locates the bin that holds the k-th smallest key; if that
-// bin is too full the range is narrowed to it ("zoom") and the pass repeats.  A filter pass then marks
-// every key below the bin as evicted (one 64-bit mask per page, built with warp votes) and collects the
-// keys inside the bin; a single CTA ranks those candidates exactly (radix select on the differing bits).
-// The result is identical to a full sort; no floating-point value is compared after key construction.
+// Every entry maps to a unique 64-bit key whose integer order is the eviction order, so the result is identical
+// to a full sort and no floating-point value is compared after key construction.
+//
+// Cache path (one pass over the metadata): a Bernoulli sample of the sequence's keys brackets the k-th smallest
+// key; one filter pass counts the keys below the bracket (marking them in per-page 64-bit eviction masks built with
+// warp votes) and collects the keys inside it; one CTA per sequence verifies the bracket and ranks the collected
+// keys exactly (radix select on the differing bits).  A bracket that missed (probability below 1e-9) is redone
+// exactly by a single-CTA radix select over the whole sequence.
+// Flat-array path (standalone selection over fp32 scores): shared-memory histogram passes (4094 equal-width bins,
+// first centred on a small sample, then narrowed to the bin that holds the k-th key), filter, exact ranking.
+// Fixed per-pool budgets: one CTA per pool ranks that pool's keys exactly.
+#include <algorithm>
+
 #include "trimkv_internal.cuh"
 
 namespace tkv {
@@ -539,21 +545,22 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: 
     return x;
 }
 
-// One thread per page.  mode 0: every live slot is sampled (small sequences).  mode 1: every slot with probability
-// thresh / 2^32, decided per slot.  mode 2 (large sequences, 64 * p <= 1): at most one slot per page, the page being
-// chosen with probability 64 * p and the slot uniformly; slots beyond the page's fill are simply not sampled, so each
-// live slot still has probability p.
+// Bernoulli sample of the live slots with probability p each.  sub = 0: every live slot is taken (small sequences).
+// Otherwise a thread owns a block of `sub` consecutive slots of a page (sub a power of two, sub * p <= 1/2): it takes
+// the block with probability sub * p (thresh / 2^32) and then one slot of it uniformly; a slot beyond the page's fill
+// is simply not sampled, so every live slot has probability p.
 __global__ void __launch_bounds__(256)
-sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, int mode, uint32_t thresh,
+sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, int sub, uint32_t thresh,
               uint32_t seed) {
     const int b = blockIdx.y;
-    const long long page = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int per_page = sub > 0 ? PAGE / sub : 1;
+    const long long page = gid / per_page;
     if (page >= src.cv.P_seq) return;
     const int4 inf = src.info(b, page);
     if (inf.x < 0) return;
     SelState* st = sel + b;
     const CacheView& cv = src.cv;
-    const uint32_t base = (uint32_t)(page * PAGE) * 0x9E3779B1u + seed + (uint32_t)b * 0x85EBCA77u;
     auto take = [&](int off) {
         const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
         const int pos = cv.pos[s];
@@ -562,14 +569,16 @@ sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample
         const unsigned w = atomicAdd(&st->sample_count, 1u);
         if (w < SAMPLE_CAP) sample[(size_t)b * SAMPLE_CAP + w] = make_key(S, tie);
     };
-    if (mode == 2) {
-        if (mix32(base) < thresh) {                         // thresh = 64 * p * 2^32
-            const int off = (int)(mix32(base ^ 0x68E31DA4u) & (PAGE - 1));
-            if (off < inf.z) take(off);
-        }
-    } else {
-        for (int off = 0; off < inf.z; ++off)
-            if (mode == 0 || mix32(base + (uint32_t)off * 0x9E3779B1u) < thresh) take(off);
+    if (sub == 0) {
+        for (int off = 0; off < inf.z; ++off) take(off);
+        return;
+    }
+    const int blk = (int)(gid % per_page);
+    if (blk * sub >= inf.z) return;
+    const uint32_t base = (uint32_t)gid * 0x9E3779B1u + seed + (uint32_t)b * 0x85EBCA77u;
+    if (mix32(base) < thresh) {
+        const int off = blk * sub + (int)(mix32(base ^ 0x68E31DA4u) & (uint32_t)(sub - 1));
+        if (off < inf.z) take(off);
     }
 }
 
@@ -1182,16 +1191,18 @@ void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long
     CacheSrc src;
     src.cv = cv;
     src.t1 = t + 1;
-    int mode = 0;                                        // sample every key
+    int sub = 0;                                         // 0: sample every key
     uint32_t thresh = 0xffffffffu;
     if (n_total > SAMPLE_MEAN) {
         const double p = (double)SAMPLE_MEAN / (double)n_total;
-        if (p * PAGE <= 0.5) { mode = 2; thresh = (uint32_t)(4294967296.0 * p * PAGE); }
-        else { mode = 1; thresh = (uint32_t)(4294967296.0 * p); }
+        sub = PAGE;
+        while (sub > 1 && p * sub > 0.5) sub >>= 1;
+        thresh = (uint32_t)(4294967296.0 * std::min(p * sub, 0.999999));
     }
     const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u;
-    dim3 gs((unsigned)((cv.P_seq + 255) / 256), cv.B);
-    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, mode, thresh, seed);
+    const long long threads = cv.P_seq * (sub > 0 ? PAGE / sub : 1);
+    dim3 gs((unsigned)((threads + 255) / 256), cv.B);
+    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, sub, thresh, seed);
     bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample);
     dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
     filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
