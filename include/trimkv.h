@@ -141,6 +141,15 @@ TRIMKV_API trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const v
 TRIMKV_API trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
                                      const void* q, void* out, void* stream);
 
+/* The same step for callers whose per-token tensors live in HOST memory (same shapes; pinned memory makes the copies
+ * asynchronous).  The library copies them to staging buffers of the handle on its internal streams, each where its consumer
+ * runs (K, V, q ahead of attention; x or lambda beside it, ahead of the gate), and copies the attention output to out_host
+ * at the end of the step; everything is ordered after earlier work of `stream` and complete, for `stream`, when the call's
+ * work is.  The host buffers must stay untouched until then. */
+TRIMKV_API trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x_host, const float* lambda_host,
+                                          const void* k_host, const void* v_host, const void* q_host, void* out_host,
+                                          void* stream);
+
 /* trimkv_decode_step_all runs on two internal streams by default: K/V append, attention and compaction on one, the
  * gate and the selection beside them on the other (attention never reads retention terms, the selection never reads
  * K/V); both are forked from and joined back to the caller's stream.  enable = 0 runs every phase back to back on the

@@ -22,7 +22,7 @@ DTYPE_BF16, DTYPE_F32 = 0, 1
 EXPORTS = [
     "trimkv_default_config", "trimkv_create", "trimkv_create_ex", "trimkv_destroy", "trimkv_reset", "trimkv_set_gate",
     "trimkv_set_shared_projection", "trimkv_gate", "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention",
-    "trimkv_decode_step_all", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
+    "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static",
 ]
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
     L.trimkv_score_and_evict.argtypes = [vp, vp]
     L.trimkv_decode_attention.argtypes = [vp, i32, vp, vp, vp]
     L.trimkv_decode_step_all.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    L.trimkv_decode_step_all_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    L.trimkv_decode_step_all_host.restype = i32
     L.trimkv_get_lengths.argtypes = [vp, vp]
     L.trimkv_get_kept.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
     L.trimkv_get_pool.argtypes = [vp, i32, i32, i32, i32, C.POINTER(i32), vp, vp, vp, vp, vp]
@@ -212,6 +214,15 @@ class TrimKV:
         _check(lib().trimkv_decode_step_all(self._h, _ptr(x, f), _ptr(lam, f), _ptr(k, self.torch_dtype),
                                             _ptr(v, self.torch_dtype), _ptr(q, self.torch_dtype),
                                             _ptr(out, self.torch_dtype), _stream()))
+        return out
+
+    def decode_step_all_host(self, k, v, q, out, x=None, lam=None):
+        """Same step with HOST tensors (pinned for asynchronous copies); `out` is a host tensor as well."""
+        f = torch.float32
+        _check(lib().trimkv_decode_step_all_host(self._h, _ptr(x, f, cuda=False), _ptr(lam, f, cuda=False),
+                                                 _ptr(k, self.torch_dtype, cuda=False), _ptr(v, self.torch_dtype, cuda=False),
+                                                 _ptr(q, self.torch_dtype, cuda=False), _ptr(out, self.torch_dtype, cuda=False),
+                                                 _stream()))
         return out
 
     def reset(self):

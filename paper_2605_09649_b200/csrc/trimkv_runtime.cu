@@ -94,6 +94,8 @@ struct trimkv {
     AttnBuffers ab;
     int32_t *hole, *mover, *cursor;
     float *W1, *b1, *W2, *b2, *w_g, *gv, *gs0, *u, *g_lam, *g_c;
+    float* st_x = nullptr;                                   // staging of trimkv_decode_step_all_host: x or lambda
+    char *st_k = nullptr, *st_v = nullptr, *st_q = nullptr, *st_out = nullptr;
     float *W1hi = nullptr, *W1lo = nullptr, *xhi = nullptr, *xlo = nullptr;   // 3xTF32 operands of the tensor-core gate
     GateTcState* tc = nullptr;
     float b_g;
@@ -356,6 +358,11 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     h->rows_max = std::max<long long>((long long)h->B * cfg->max_chunk, (long long)h->L * h->B);
     A(dev_alloc(h, &h->g_lam, (size_t)h->rows_max * h->H, false));
     A(dev_alloc(h, &h->g_c, (size_t)h->rows_max * h->H, false));
+    A(dev_alloc(h, &h->st_x, (size_t)h->L * h->B * std::max(h->D, h->H), false));
+    A(dev_alloc(h, &h->st_k, (size_t)h->L * h->B * h->H * h->d * h->elt, false));
+    A(dev_alloc(h, &h->st_v, (size_t)h->L * h->B * h->H * h->d * h->elt, false));
+    A(dev_alloc(h, &h->st_q, (size_t)h->L * h->B * h->Hq * h->d * h->elt, false));
+    A(dev_alloc(h, &h->st_out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, false));
     if (h->D > 0) {
         A(dev_alloc(h, &h->W1, (size_t)h->L * h->dg * h->D, false));
         A(dev_alloc(h, &h->b1, (size_t)h->L * h->dg, false));
@@ -498,11 +505,19 @@ trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const void* q, voi
     return attention_impl(h, layer, 1, q, out, (cudaStream_t)stream);
 }
 
-trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
-                                     const void* q, void* out, void* stream) {
-    if (check_handle(h)) return TRIMKV_E_ARG;
-    if (!k || !v || !q || !out || (!x && !lambda)) return fail(TRIMKV_E_ARG, "NULL argument");
-    if (!aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out) || (x && !aligned16(x))) return fail(TRIMKV_E_ARG, "buffers must be 16-byte aligned");
+}  // extern "C"
+
+namespace {
+
+// Host-resident arguments of trimkv_decode_step_all_host: copied to / from the handle's staging buffers on the internal
+// streams, each copy placed where its consumer runs (K, V, q ahead of attention; x or lambda ahead of the gate).
+struct HostArgs {
+    const void *x, *lambda, *k, *v, *q;
+    void* out;
+};
+
+trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, const void* k, const void* v, const void* q,
+                            void* out, void* stream, const HostArgs* host) {
     const long long t = h->tokens[0];
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layers hold different token counts");
@@ -523,6 +538,14 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
         CUDA_TRY(cudaEventRecord(h->ev_fork, st));
         CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
         CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_fork, 0));
+    }
+    if (host) {
+        const size_t kvb = (size_t)h->L * h->B * h->H * h->d * h->elt, qb = (size_t)h->L * h->B * h->Hq * h->d * h->elt;
+        CUDA_TRY(cudaMemcpyAsync(h->st_k, host->k, kvb, cudaMemcpyHostToDevice, fs));
+        CUDA_TRY(cudaMemcpyAsync(h->st_v, host->v, kvb, cudaMemcpyHostToDevice, fs));
+        CUDA_TRY(cudaMemcpyAsync(h->st_q, host->q, qb, cudaMemcpyHostToDevice, fs));
+        if (host->x) CUDA_TRY(cudaMemcpyAsync(h->st_x, host->x, (size_t)h->L * h->B * h->D * 4, cudaMemcpyHostToDevice, sd));
+        else CUDA_TRY(cudaMemcpyAsync(h->st_x, host->lambda, (size_t)h->L * h->B * h->H * 4, cudaMemcpyHostToDevice, sd));
     }
     if (h->prof.on) h->prof.mark(PH_APPEND, 0, fs);
     launch_append(h->cv, 0, h->L, 1, t, nullptr, nullptr, h->cfg.horizon, k, v, APPEND_KV, fs);
@@ -550,6 +573,7 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
         CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
     }
     if (s == TRIMKV_OK && kev > 0) s = compact_impl(h, fs);
+    if (host) CUDA_TRY(cudaMemcpyAsync(host->out, out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, cudaMemcpyDeviceToHost, fs));
     if (two) {
         CUDA_TRY(cudaEventRecord(h->ev_done, fs));
         CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
@@ -557,6 +581,28 @@ trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* l
     if (s != TRIMKV_OK) return s;
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
+                                     const void* q, void* out, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!k || !v || !q || !out || (!x && !lambda)) return fail(TRIMKV_E_ARG, "NULL argument");
+    if (!aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out) || (x && !aligned16(x))) return fail(TRIMKV_E_ARG, "buffers must be 16-byte aligned");
+    return step_all_impl(h, x, lambda, k, v, q, out, stream, nullptr);
+}
+
+trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x_host, const float* lambda_host, const void* k_host,
+                                          const void* v_host, const void* q_host, void* out_host, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!k_host || !v_host || !q_host || !out_host || (!x_host && !lambda_host)) return fail(TRIMKV_E_ARG, "NULL argument");
+    if (x_host && h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
+    HostArgs ha{x_host, lambda_host, k_host, v_host, q_host, out_host};
+    return step_all_impl(h, x_host ? h->st_x : nullptr, x_host ? nullptr : h->st_x, h->st_k, h->st_v, h->st_q, h->st_out,
+                         stream, &ha);
 }
 
 trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host) {

@@ -463,6 +463,49 @@ def test_decode_step_all_entry_point():
         cch.close()
 
 
+def test_decode_step_all_host_buffers_entry_point():
+    """trimkv_decode_step_all_host (pinned host tensors in, host tensor out) gives what the device-pointer call gives."""
+    w = workloads.WORKLOADS["llama8b_32k"].replace(layers=2, batch=2, budget_entries=2 * 8 * 40, chunk=64, context=64)
+    per_layer, w_g = workloads.gate_params(w, 2, device=DEV)
+    bank = workloads.ProjectionBank(w, 2, device=DEV)
+    caches = [binding.TrimKV.from_workload(w) for _ in range(2)]
+    for cch in caches:
+        for l, p in enumerate(per_layer):
+            cch.set_gate(l, *p)
+        cch.set_shared_projection(w_g, 4.0)
+    for l in range(w.layers):
+        x = workloads.hidden_states(w, 2, l, 0, 64, device=DEV)
+        _, k, v = workloads.project_qkv(w, bank, l, x)
+        for cch in caches:
+            cch.append(l, k, v, x=x)
+    for cch in caches:
+        cch.score_and_evict()
+    for step in range(4):
+        xs, ks, vs, qs = [], [], [], []
+        for l in range(w.layers):
+            x = workloads.hidden_states(w, 2, l, 64 + step, 1, device=DEV)
+            q, k, v = workloads.project_qkv(w, bank, l, x)
+            xs.append(x[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0]); qs.append(q[:, 0])
+        X, K, V, Q = [torch.stack(t).contiguous() for t in (xs, ks, vs, qs)]
+        out_dev = torch.empty_like(Q)
+        caches[0].decode_step_all(K, V, Q, out_dev, x=X)
+        hX, hK, hV, hQ = [t.cpu().pin_memory() for t in (X, K, V, Q)]
+        out_host = torch.empty_like(hQ).pin_memory()
+        caches[1].decode_step_all_host(hK, hV, hQ, out_host, x=hX)
+        torch.cuda.synchronize()
+        assert torch.equal(out_dev.cpu(), out_host)
+        assert torch.equal(caches[0].lengths(), caches[1].lengths())
+    # retention supplied instead of x
+    lam = (-torch.rand(w.layers, w.batch, w.kv_heads) * 0.01).pin_memory()
+    caches[0].decode_step_all(K, V, Q, out_dev, lam=lam.to(DEV))
+    caches[1].decode_step_all_host(hK, hV, hQ, out_host, lam=lam)
+    torch.cuda.synchronize()
+    assert torch.equal(out_dev.cpu(), out_host) and torch.equal(caches[0].lengths(), caches[1].lengths())
+    for cch in caches:
+        cch.sync_status()
+        cch.close()
+
+
 # ------------------------------------------------------------------------------------------- standalone selection
 def _oracle_keep_bits(scores_np, k_keep):
     n = len(scores_np)
