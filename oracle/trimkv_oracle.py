@@ -292,6 +292,25 @@ class OracleCache:
                 off += m
         return n - self.budget
 
+    def prefill_attention(self, layer, q):
+        """Causal attention of the chunk just appended to `layer` (its last n tokens), q [n, Hq, d] -> [n, Hq, d] fp64.
+
+        Token j of the chunk sits at position p = tokens[layer] - n + j + 1 and attends to the retained entries with
+        position <= p (Sec. 2.1: C_t = {1..t}, restricted to the retained set as in Eq. (1)): everything kept from before
+        the chunk plus the chunk's own tokens up to itself.
+        """
+        q = np.asarray(q, F64)
+        n = q.shape[0]
+        base = self.tokens[layer] - n
+        out = np.zeros((n, self.Hq, self.d), F64)
+        for j in range(n):
+            p = base + j + 1
+            for hq in range(self.Hq):
+                h = hq // self.g
+                vis = self.pos[layer][h] <= p
+                out[j, hq] = attention(q[j, hq], self.K[layer][h][vis], self.V[layer][h][vis])
+        return out
+
     def lengths(self):
         return np.array([[len(self.pos[l][h]) for h in range(self.H)] for l in range(self.L)], np.int32)
 

@@ -408,3 +408,36 @@ def test_per_pool_budget_variant():
         assert c.kept_positions(l, 1).tolist() == want
     assert (c.lengths() == M).all()
     assert g.lengths().sum() == M * L * H and (g.lengths() != M).any()        # the global budget reallocates
+
+
+def test_prefill_attention_is_causal_dense_attention_when_nothing_was_evicted():
+    """With a budget that evicts nothing, chunked causal attention over the cache equals textbook causal attention
+    (torch SDPA with is_causal) over the whole sequence; the last token of a chunk sees what a decode step would."""
+    L, H, Hq, d = 1, 2, 4, 8
+    c = orc.OracleCache(10 ** 9, L, H, Hq, d)
+    T = 11
+    k = rng.normal(size=(T, H, d)); v = rng.normal(size=(T, H, d)); q = rng.normal(size=(T, Hq, d))
+    lam = np.zeros((T, H), np.float32)
+    outs = []
+    for a, b in ((0, 4), (4, 5), (5, 11)):                       # chunks of 4, 1 and 6 tokens
+        c.append(0, k[a:b], v[a:b], lam=lam[a:b])
+        o = c.prefill_attention(0, q[a:b])
+        outs.append(o)
+        np.testing.assert_allclose(o[-1], c.decode_attention(0, q[b - 1]), rtol=1e-12)
+    got = np.concatenate(outs)                                    # [T, Hq, d]
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]               # [1, Hq, T, d]
+    tk = torch.from_numpy(np.repeat(k, Hq // H, axis=1)).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(np.repeat(v, Hq // H, axis=1)).permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-12)
+    # after an eviction the evicted positions are gone for later chunks, whatever their position
+    c2 = orc.OracleCache(6, 1, 1, 1, d)
+    lam2 = np.array([[-3.0], [-1e-4], [-3.0], [-1e-4], [-3.0], [-1e-4], [-3.0], [-1e-4]], np.float32)
+    c2.append(0, k[:8, :1], v[:8, :1], lam=lam2)
+    c2.score_and_evict()
+    kept = set(c2.kept_positions(0, 0).tolist())
+    assert len(kept) == 6 and {2, 4, 6, 8} <= kept
+    c2.append(0, k[8:10, :1], v[8:10, :1], lam=np.zeros((2, 1), np.float32))
+    o = c2.prefill_attention(0, q[8:10, :1])
+    idx = sorted(p - 1 for p in kept) + [8]
+    np.testing.assert_allclose(o[0, 0], orc.attention(q[8, 0], k[idx, 0], v[idx, 0]), rtol=1e-12)
