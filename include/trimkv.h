@@ -135,6 +135,12 @@ TRIMKV_API trimkv_status trimkv_score_and_evict(trimkv_t* h, void* stream);
  * scale 1/sqrt(d); an empty pool gives zeros. */
 TRIMKV_API trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const void* q, void* out, void* stream);
 
+/* Causal attention of a prompt chunk (Sec. 2.1, restricted to the retained set as in Eq. (1)): call it after
+ * trimkv_append(layer, n_new, ...) of the chunk and before the eviction round.  q, out: device [B, n_new, Hq, d] in
+ * kv_dtype; token j of the chunk attends to every entry kept from before the chunk and to the chunk's tokens 0..j.
+ * TRIMKV_E_UNSUPPORTED with retention_bias set. */
+TRIMKV_API trimkv_status trimkv_prefill_attention(trimkv_t* h, int layer, int n_new, const void* q, void* out, void* stream);
+
 /* One whole decode step for all layers at once (the benchmark path): gate on x [L, B, D] fp32
  * (or lambda [L, B, H] if x == NULL), append k, v [L, B, H, d], attention of q [L, B, Hq, d] into
  * out [L, B, Hq, d], then score_and_evict. */

@@ -22,7 +22,7 @@ DTYPE_BF16, DTYPE_F32 = 0, 1
 EXPORTS = [
     "trimkv_default_config", "trimkv_create", "trimkv_create_ex", "trimkv_destroy", "trimkv_reset", "trimkv_set_gate",
     "trimkv_set_shared_projection", "trimkv_gate", "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention",
-    "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
+    "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static",
 ]
@@ -71,6 +71,8 @@ def lib() -> C.CDLL:
     L.trimkv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.trimkv_score_and_evict.argtypes = [vp, vp]
     L.trimkv_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    L.trimkv_prefill_attention.argtypes = [vp, i32, i32, vp, vp, vp]
+    L.trimkv_prefill_attention.restype = i32
     L.trimkv_decode_step_all.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.trimkv_decode_step_all_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.trimkv_decode_step_all_host.restype = i32
@@ -207,6 +209,14 @@ class TrimKV:
             out = torch.empty_like(q)
         _check(lib().trimkv_decode_attention(self._h, layer, _ptr(q, self.torch_dtype), _ptr(out, self.torch_dtype),
                                              _stream()))
+        return out
+
+    def prefill_attention(self, layer: int, q, out=None):
+        """q [B, n, Hq, d]: causal attention of the n-token chunk just appended to `layer`."""
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib().trimkv_prefill_attention(self._h, layer, q.shape[1], _ptr(q, self.torch_dtype),
+                                              _ptr(out, self.torch_dtype), _stream()))
         return out
 
     def decode_step_all(self, k, v, q, out, x=None, lam=None):

@@ -195,6 +195,10 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
                       long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, const void* q,
                       void* out, cudaStream_t st, PhaseMarker* pm);
 
+// Causal attention of the chunk of n_new tokens just appended to `layer`; q, out: [B, n_new, Hq, d].
+void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const void* q, void* out,
+                              cudaStream_t st);
+
 void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
                         void* v, int n, cudaStream_t st);
 

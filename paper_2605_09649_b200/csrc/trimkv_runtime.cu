@@ -505,6 +505,21 @@ trimkv_status trimkv_decode_attention(trimkv_t* h, int layer, const void* q, voi
     return attention_impl(h, layer, 1, q, out, (cudaStream_t)stream);
 }
 
+trimkv_status trimkv_prefill_attention(trimkv_t* h, int layer, int n_new, const void* q, void* out, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (layer < 0 || layer >= h->L || !q || !out || !aligned16(q) || !aligned16(out)) return fail(TRIMKV_E_ARG, "bad layer, q or out");
+    if (n_new < 1 || n_new > h->cfg.max_chunk || n_new > h->tokens[layer])
+        return fail(TRIMKV_E_ARG, "n_new must be the size of the chunk last appended to this layer");
+    if (h->cfg.retention_bias) return fail(TRIMKV_E_UNSUPPORTED, "chunk attention supports the plain softmax only");
+    PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
+    launch_prefill_attention(h->cv, layer, n_new, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, q, out, st);
+    if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
 }  // extern "C"
 
 namespace {

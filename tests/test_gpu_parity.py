@@ -415,6 +415,35 @@ def test_fixed_per_pool_budget_variant(horizon, per_pool):
     pair.close()
 
 
+@pytest.mark.parametrize("kv_dtype,g,atol", [("bf16", 1, ATT_ATOL_BF16), ("bf16", 4, ATT_ATOL_BF16), ("bf16", 7, ATT_ATOL_BF16),
+                                             ("bf16", 8, ATT_ATOL_BF16), ("bf16", 12, ATT_ATOL_BF16), ("f32", 2, ATT_ATOL_F32)])
+def test_chunk_prefill_causal_attention(kv_dtype, g, atol):
+    """trimkv_prefill_attention: every token of an appended chunk attends to what was kept before the chunk and to the
+    chunk's tokens up to itself; chunks that do not fill token blocks, pages or tiles, with evictions in between."""
+    d = 128 if kv_dtype == "bf16" else 64
+    w = workloads.Workload("chunk", 2, 2, 2 * g, d, 0, 2, 420, kv_dtype, 0, 0, 160)
+    dt = workloads.torch_dtype(kv_dtype)
+    pair = Pair(w)
+    r = np.random.default_rng(41)
+    gen = torch.Generator(device=DEV); gen.manual_seed(41)
+    for n in (37, 160, 95, 1, 130):
+        for l in range(w.layers):
+            k = torch.randn(w.batch, n, w.kv_heads, d, generator=gen, device=DEV).to(dt)
+            v = torch.randn(w.batch, n, w.kv_heads, d, generator=gen, device=DEV).to(dt)
+            q = torch.randn(w.batch, n, w.q_heads, d, generator=gen, device=DEV).to(dt)
+            lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), scale=0.05)
+            pair.append(l, k, v, lam, oracle_retention(lam, w.horizon))
+            got = to_np(pair.gpu.prefill_attention(l, q))
+            for b in pair.seqs:
+                want = pair.orc[b].prefill_attention(l, to_np(q[b]))
+                err = np.abs(got[b] - want).max()
+                assert err <= atol, f"chunk attention error {err} (n={n}, layer {l}, sequence {b})"
+        pair.evict()
+        pair.check_sets()
+    pair.gpu.sync_status()
+    pair.close()
+
+
 def test_step_all_matches_layerwise_oracle():
     w = BF16_SMALL.replace(budget_entries=400)
     lam_fn = lambda r, shape, l: random_lambda(shape, int(r.integers(1 << 30)))
