@@ -214,10 +214,12 @@ def run_ours(args, w):
             evs = []
             for l in range(w.layers):
                 x = workloads.hidden_states(w, seed, l, start + done, n, device=dev)
-                _, k, v = workloads.project_qkv(w, bank, l, x)
+                qc, k, v = workloads.project_qkv(w, bank, l, x)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
                 cache.append(l, k, v, x=x)
+                if args.prefill_attention:
+                    cache.prefill_attention(l, qc)
                 if l == w.layers - 1:
                     cache.score_and_evict()
                 b.record()
@@ -370,7 +372,8 @@ def run_ours(args, w):
                    "turns": w.turns, "tokens_before_timed_region": tokens_seen,
                    "prefill": {"chunks": prefill_chunks, "ms_per_chunk": prefill_ms / max(prefill_chunks, 1),
                                "tokens_per_s": w.batch * w.chunk / (prefill_ms / max(prefill_chunks, 1) * 1e-3) if prefill_ms > 0 else None,
-                               "what": "gate + append of every layer and one eviction per chunk (no chunk attention)"},
+                               "what": "gate + append of every layer and one eviction per chunk" +
+                                       (", with the chunk's causal attention" if args.prefill_attention else " (no chunk attention)")},
                    "earlier_turn_decode_ms_per_step": early_decode_ms / early_decode_steps if early_decode_steps else None},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
@@ -453,6 +456,8 @@ def main():
                     help="decode attention with the retention-gated weights of Sec. 2.2 (reads 8 more bytes per entry)")
     ap.add_argument("--fixed-budget", action="store_true",
                     help="the fixed per-head budget variant (every pool keeps budget / (layers * kv_heads) entries)")
+    ap.add_argument("--prefill-attention", action="store_true",
+                    help="also run the chunk's causal attention over the cache during the (untimed) prefill and report it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
     ap.add_argument("--sweep-max", type=int, default=28)
