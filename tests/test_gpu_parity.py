@@ -444,6 +444,43 @@ def test_chunk_prefill_causal_attention(kv_dtype, g, atol):
     pair.close()
 
 
+@pytest.mark.parametrize("seed", list(range(8)))
+def test_random_shapes_and_schedules(seed):
+    """Randomised shapes (layers, heads, group, batch, budget down to fewer entries than pools) and schedules (chunks
+    of random size, decode steps, evictions) against the oracle: kept sets bit-exact after every eviction, decode and
+    chunk attention within tolerance."""
+    r = np.random.default_rng(1000 + seed)
+    L, H = int(r.integers(1, 4)), int(r.integers(1, 4))
+    g = int(r.choice([1, 2, 3, 4, 7, 8]))
+    B = int(r.integers(1, 4))
+    budget = int(r.choice([L * H - 1 if L * H > 1 else 1, 3 * L * H, 40 * L * H + 7, 300]))
+    horizon = int(r.choice([0, 1, 2, 5]))
+    w = workloads.Workload("fuzz", L, H, H * g, 128, 0, B, budget, "bf16", 0, 0, 200, horizon=horizon)
+    pair = Pair(w)
+    gen = torch.Generator(device=DEV); gen.manual_seed(seed)
+    dt = torch.bfloat16
+    for it in range(int(r.integers(4, 9))):
+        n = int(r.choice([1, 1, 2, 17, 64, 65, 130, 200]))
+        scale = float(r.choice([1e-4, 0.02, 1.0]))
+        for l in range(L):
+            k = torch.randn(B, n, H, 128, generator=gen, device=DEV).to(dt)
+            v = torch.randn(B, n, H, 128, generator=gen, device=DEV).to(dt)
+            lam = random_lambda((B, n, H), int(r.integers(1 << 30)), distinct=int(r.choice([0, 0, 2])), scale=scale)
+            pair.append(l, k, v, lam, oracle_retention(lam, horizon))
+            q = torch.randn(B, n, H * g, 128, generator=gen, device=DEV).to(dt)
+            if n > 1:
+                got = to_np(pair.gpu.prefill_attention(l, q))
+                for b in pair.seqs:
+                    err = np.abs(got[b] - pair.orc[b].prefill_attention(l, to_np(q[b]))).max()
+                    assert err <= ATT_ATOL_BF16, f"chunk attention error {err}"
+            pair.check_attention(l, q[:, -1].contiguous(), ATT_ATOL_BF16)
+        pair.evict()
+        pair.check_sets()
+        assert int(pair.gpu.lengths().sum()) == B * min(budget, sum(pair.orc[0].tokens) * H)
+    pair.gpu.sync_status()
+    pair.close()
+
+
 def test_step_all_matches_layerwise_oracle():
     w = BF16_SMALL.replace(budget_entries=400)
     lam_fn = lambda r, shape, l: random_lambda(shape, int(r.integers(1 << 30)))
