@@ -977,45 +977,46 @@ redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_ma
     if (tid == 0) st->resolved = 1;
 }
 
-// Flat arrays: centres the first histogram pass on the data.  1024 threads read 4096 evenly spaced scores; the bins
-// then span the sampled score range widened by an eighth on both sides (any range is correct: keys outside it fall
-// into the catch-all bins and cost a further pass at worst; a fitting one settles the selection in one pass).
+// Flat arrays: centres the first histogram pass on the threshold.  4096 evenly spaced scores are sampled and ranked by
+// bracket_kernel exactly as for the cache path; the bracket of the k-th key (a tenth of the key range or less) becomes
+// the binned range of the first pass, whose bins are then fine enough to settle the selection at once.  Any range is
+// correct: keys outside it fall into the catch-all bins and cost a further pass at worst.
 __global__ void __launch_bounds__(1024)
-seed_range_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st) {
-    __shared__ uint32_t wmin[32], wmax[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t smin = 0xffffffffu, smax = 0u;
-    const long long step = n / 4096 > 0 ? n / 4096 : 1;
-    for (int i = 0; i < 4; ++i) {
-        const long long idx = (long long)(tid * 4 + i) * step;
-        if (idx < n) {
-            const float x = s[idx];
-            if (x == x) {
-                const uint32_t sc = orderable_key(x);
-                smin = min(smin, sc);
-                smax = max(smax, sc);
-            }
-        }
+flat_sample_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, u64* __restrict__ sample) {
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= SAMPLE_CAP) return;
+    const long long step = n / SAMPLE_CAP > 0 ? n / SAMPLE_CAP : 1;
+    const long long idx = (long long)gid * step;
+    if (idx >= n) return;
+    const float x = s[idx];
+    if (x != x) return;                                   // NaN is reported by the histogram pass
+    const unsigned w = atomicAdd(&st->sample_count, 1u);
+    const u64 key = compose_key(orderable_key(x), (uint32_t)idx);
+    if (w < SAMPLE_CAP) sample[w] = key;
+    atomicMin(&st->kmin, key);                            // smallest sampled key: lower end when the bracket has none
+}
+
+__global__ void flat_range_kernel(SelState* __restrict__ st) {
+    u64 c_lo = st->cand_lo;
+    const u64 c_hi = st->cand_hi, smin = st->kmin;
+    st->passes = 0;
+    st->sample_count = 0;
+    st->kmin = ~0ull;                                     // as the histogram pass expects it
+    if (c_lo == 0ull && smin < c_hi) {                    // bracket open below: start a little under the sampled minimum
+        const u64 pad = (c_hi - smin) / 8 + 1;
+        c_lo = smin > pad ? smin - pad : 0ull;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        smin = min(smin, __shfl_xor_sync(0xffffffffu, smin, o));
-        smax = max(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+    if (c_hi <= c_lo) return;                             // keep the full-range default
+    u64 lo = c_lo;
+    int bits = 64 - __clzll((long long)(c_hi - lo));
+    int shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
+    if (shift >= 32) {                                    // bins depend on the score word alone: start on a score boundary
+        lo &= ~0xffffffffull;
+        bits = 64 - __clzll((long long)(c_hi - lo));
+        shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
     }
-    if (lane == 0) { wmin[warp] = smin; wmax[warp] = smax; }
-    __syncthreads();
-    if (tid == 0) {
-        for (int w = 0; w < 32; ++w) { smin = min(smin, wmin[w]); smax = max(smax, wmax[w]); }
-        if (smin < smax) {
-            const uint32_t pad = (smax - smin) / 8u + 1u;
-            const uint32_t a = smin > pad ? smin - pad : 0u;
-            const uint32_t b = smax < 0xffffffffu - pad ? smax + pad : 0xffffffffu;
-            const u64 lo = (u64)a << 32, hi = ((u64)b << 32) | 0xffffffffull;
-            const int bits = 64 - __clzll((long long)(hi - lo));
-            const int shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
-            if (shift >= 32) { st->lo = lo; st->shift = shift; }
-        }
-    }
+    st->lo = lo;
+    st->shift = shift;
 }
 
 // ------------------------------------------------------------------ fixed per-pool budget (TrimKV arm)
@@ -1225,8 +1226,11 @@ void launch_select_array(const float* scores, long long n, long long k_evict, u6
     src.s = scores;
     src.n = n;
     src.err = err;
-    seed_range_kernel<<<1, 1024, 0, st>>>(scores, n, sb.sel);
-    count_launch();
+    u64* sample = reinterpret_cast<u64*>(sb.cand);        // the candidate buffer is idle until the filter pass
+    flat_sample_kernel<<<SAMPLE_CAP / 1024, 1024, 0, st>>>(scores, n, sb.sel, sample);
+    bracket_kernel<<<1, 1024, 0, st>>>(sb.sel, sample, k_evict, n, 0);
+    flat_range_kernel<<<1, 1, 0, st>>>(sb.sel);
+    count_launch(3);
     run_select_flat(src, sb, k_evict, 7, (unsigned)sb.cand_cap, evict_mask, err, st);
 }
 
