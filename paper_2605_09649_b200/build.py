@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtrimkv.so")
-SOURCES = ["trimkv_runtime.cu", "gate.cu", "gate_tc.cu", "cache.cu", "select.cu", "select_static.cu", "attention.cu", "prefill_attention.cu"]
+SOURCES = ["trimkv_runtime.cu", "gate.cu", "gate_tc.cu", "cache.cu", "select.cu", "select_static.cu", "attention.cu", "prefill_attention.cu", "prefill_attention_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

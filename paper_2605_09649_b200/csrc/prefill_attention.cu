@@ -371,8 +371,12 @@ prefill_attn_plain_kernel(CacheView cv, int layer, int n_new, int g, int Hq, con
 
 }  // namespace
 
-void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const void* q, void* out,
-                              cudaStream_t st) {
+void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const PrefillTcState* tc,
+                              const void* q, void* out, cudaStream_t st) {
+    if (tc && prefill_tc_wanted(cv, n_new, Hq)) {
+        launch_prefill_attention_tc(tc, cv, layer, n_new, Hq, q, out, st);
+        return;
+    }
     const int g = Hq / cv.H;
     const float scale = 1.0f / sqrtf((float)cv.d);
     if (is_bf16 && cv.d == 128 && g <= P_COLS) {

@@ -1,0 +1,444 @@
+// Tensor-core (tcgen05) form of the chunk's causal attention over the ragged per-(layer, head) pools (Sec. 2.1 attention
+// restricted to the retained set, Eq. (1) with r in {0,1}; same contract as the mma.sync kernel next door): chunk token j
+// sees entry e of its pool iff e < n_old + j + 1.  bf16, d = 128.
+//
+// One CTA per (pool, block of 256 / g chunk tokens): 256 (token, query head) rows in two groups of 128 that share every
+// K/V tile.  A tile is one 64-entry page.  The page's rows are stored with their 16-byte chunks permuted inside each
+// 128-byte half by (slot & 7); copied half by half with TMA (box 64 columns x 64 rows of the arena seen as a matrix of
+// 256-byte rows) they land in shared memory exactly in the tensor core's 128-byte-swizzle layout: K halves as K-major
+// operands of S = Q K^T, V halves as MN-major operands of O += P V.  Roles: warps 0-3 / 4-7 are the softmax warps of
+// group 0 / 1 (a thread owns one row: S read from tensor memory, masked, exponentiated, P written back to shared memory
+// as bf16), warp 8 issues the TMA copies into a 4-stage ring, warp 9 issues the MMAs (S of tile i + 1 before P V of tile i,
+// so the tensor pipe works while the softmax warps compute).  O accumulates in tensor memory; the running maximum is only
+// raised (and O rescaled) when it grows by more than 2^8, which keeps every exponential finite and leaves the final O / l
+// unchanged.  Every wait is bounded; a wait that runs out latches TRIMKV_E_TIMEOUT.
+#include <cuda.h>
+
+#include "trimkv_internal.cuh"
+
+namespace tkv {
+
+namespace {
+
+constexpr int A_TILE = 64;                            // entries per tile: one page
+constexpr int A_ROWS = 128;                           // query rows per softmax group
+constexpr int A_STAGES = 4;
+constexpr int A_PLANE = A_TILE * 128;                 // 8 KB: 64 entries x one 128-byte half of the row
+constexpr int A_STAGE_BYTES = 4 * A_PLANE;            // K half 0, K half 1, V half 0, V half 1
+constexpr int A_QPLANE = A_ROWS * 128;                // 16 KB: 128 query rows x one half
+constexpr int A_Q_BYTES = 2 * 2 * A_QPLANE;           // two groups, two halves
+constexpr int A_P_BYTES = 2 * A_QPLANE;               // two groups: 128 rows x 64 probabilities (bf16)
+constexpr int A_OFF_Q = A_STAGES * A_STAGE_BYTES;
+constexpr int A_OFF_P = A_OFF_Q + A_Q_BYTES;
+constexpr int A_OFF_BAR = A_OFF_P + A_P_BYTES;
+constexpr int A_SMEM = A_OFF_BAR + 256 + 1024;        // barriers and flags, alignment slack
+constexpr int A_THREADS = 320;
+constexpr unsigned A_WAIT_LIMIT = 1u << 22;
+constexpr int A_TMEM_COLS = 512;                      // S of group 0, 1: columns 0-63, 64-127; O: 128-255, 256-383
+constexpr float A_RESCALE_STEP = 8.0f;                // log2 units the running maximum may lag behind
+
+__device__ __forceinline__ uint32_t a_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void a_bar_init(uint32_t bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void a_bar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void a_bar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool a_bar_wait(uint32_t bar, uint32_t parity) {      // false: gave up
+    for (unsigned it = 0; it < A_WAIT_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void a_tma_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart (stride byte
+// offset).  lead_bytes: distance between 64-element blocks along M/N of an MN-major operand (unused for K-major: 16).
+__device__ __forceinline__ uint64_t a_desc(uint32_t saddr, uint32_t lead_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lead_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptors: D fp32, A and B bf16, M = 128.  S: both K-major, N = 64.  P V: B (V) MN-major, N = 128.
+constexpr uint32_t A_IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+constexpr uint32_t A_IDESC_PV =
+    (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+
+__device__ __forceinline__ void a_umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void a_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void a_tmem_ld32(uint32_t taddr, uint32_t* t) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(t[0]), "=r"(t[1]), "=r"(t[2]), "=r"(t[3]), "=r"(t[4]), "=r"(t[5]), "=r"(t[6]), "=r"(t[7]), "=r"(t[8]),
+          "=r"(t[9]), "=r"(t[10]), "=r"(t[11]), "=r"(t[12]), "=r"(t[13]), "=r"(t[14]), "=r"(t[15]), "=r"(t[16]),
+          "=r"(t[17]), "=r"(t[18]), "=r"(t[19]), "=r"(t[20]), "=r"(t[21]), "=r"(t[22]), "=r"(t[23]), "=r"(t[24]),
+          "=r"(t[25]), "=r"(t[26]), "=r"(t[27]), "=r"(t[28]), "=r"(t[29]), "=r"(t[30]), "=r"(t[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void a_tmem_st32(uint32_t taddr, const uint32_t* t) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(t[0]), "r"(t[1]), "r"(t[2]), "r"(t[3]), "r"(t[4]), "r"(t[5]), "r"(t[6]), "r"(t[7]), "r"(t[8]), "r"(t[9]), "r"(t[10]),
+        "r"(t[11]), "r"(t[12]), "r"(t[13]), "r"(t[14]), "r"(t[15]), "r"(t[16]), "r"(t[17]), "r"(t[18]), "r"(t[19]), "r"(t[20]),
+        "r"(t[21]), "r"(t[22]), "r"(t[23]), "r"(t[24]), "r"(t[25]), "r"(t[26]), "r"(t[27]), "r"(t[28]), "r"(t[29]), "r"(t[30]),
+        "r"(t[31])
+        : "memory");
+}
+__device__ __forceinline__ void a_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void a_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// grid = (token blocks, B * H pools of `layer`); q, out: [B, n_new, Hq, 128] bf16.  map_kv: the K/V arena as a matrix of
+// 256-byte rows (128 bf16), box 64 columns x 64 rows.
+__global__ void __launch_bounds__(A_THREADS, 1)
+prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv, int layer, int n_new, int g, int Hq,
+                       const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float scale_log2) {
+    extern __shared__ unsigned char a_smem_raw[];
+    const uint32_t raw = a_smem(a_smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                        // operand tiles need 1024-byte alignment
+    unsigned char* gen = a_smem_raw + (base - raw);
+    const uint32_t bars = base + A_OFF_BAR;
+    const uint32_t full0 = bars, empty0 = bars + 32, s_ready0 = bars + 64, s_free0 = bars + 80, p_ready0 = bars + 96,
+                   pv_done0 = bars + 112;
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen + A_OFF_BAR + 128);
+    volatile int* s_fail = reinterpret_cast<volatile int*>(gen + A_OFF_BAR + 136);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const int tt = 256 / g;                                              // chunk tokens per CTA
+    const int i0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * tt;          // longest blocks first
+    const int h = blockIdx.y % cv.H, b = blockIdx.y / cv.H;
+    const long long pool = ((long long)b * cv.L + layer) * cv.H + h;
+    const int n_old = cv.len[pool] - n_new;                              // entries kept from before the chunk
+    if (i0 >= n_new || n_old < 0) return;                                // (n_old < 0: the append failed; its error is latched)
+    const int limit_max = n_old + min(n_new, i0 + tt);                   // entries any token of this block may see
+    const int ntile = (limit_max + A_TILE - 1) / A_TILE;
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < A_STAGES; ++s) { a_bar_init(full0 + 8 * s, 1); a_bar_init(empty0 + 8 * s, 1); }
+        for (int gq = 0; gq < 2; ++gq) {
+            a_bar_init(s_ready0 + 8 * gq, 1);
+            a_bar_init(s_free0 + 8 * gq, 4);
+            a_bar_init(p_ready0 + 8 * gq, 4);
+            a_bar_init(pv_done0 + 8 * gq, 1);
+        }
+        *s_fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(a_smem((const void*)s_tmem)),
+                     "r"(A_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // ---- per-row facts of the softmax threads, and the Q tile: row R of the block = (token i0 + R / g, head R % g)
+    const int grp = (warp >> 2) & 1, wl = warp & 3;
+    const int r = wl * 32 + lane;                                        // row inside the group = tensor-memory lane
+    const int R = grp * A_ROWS + r;
+    const int tok = i0 + R / g, head = R % g;
+    const bool valid = warp < 8 && R < tt * g && tok < n_new;
+    const int limit = valid ? n_old + tok + 1 : 0;                       // entries this row sees
+    if (warp < 8) {
+        const uint4* src = reinterpret_cast<const uint4*>(q + (((size_t)b * n_new + (valid ? tok : 0)) * Hq + (size_t)h * g + head) * 128);
+        unsigned char* qdst = gen + A_OFF_Q + grp * 2 * A_QPLANE + r * 128;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const uint4 v = valid ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(qdst + (c >> 3) * A_QPLANE + (((c & 7) ^ (r & 7)) << 4)) = v;
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");         // Q and the barriers, before the async proxy uses them
+    a_fence_before();
+    __syncthreads();
+    a_fence_after();
+    const uint32_t tmem = *s_tmem;
+
+    if (warp == 8) {
+        // ---- TMA producer: lane l holds the page of tile i0 + l of the current run of 32 tiles
+        int page_id = 0;
+        for (int i = 0; i < ntile; ++i) {
+            if ((i & 31) == 0) page_id = (i + lane < ntile) ? bt[i + lane] : 0;
+            const int page = __shfl_sync(0xffffffffu, page_id, i & 31);
+            const int s = i % A_STAGES;
+            int ok = 1;
+            if (lane == 0) {
+                if (i >= A_STAGES) ok = a_bar_wait(empty0 + 8 * s, ((i / A_STAGES) - 1) & 1) ? 1 : 0;
+                if (ok) {
+                    const uint32_t dst = base + s * A_STAGE_BYTES;
+                    const int krow = (int)((((long long)b * cv.P_seq + page) * 2) * PAGE);
+                    a_bar_expect_tx(full0 + 8 * s, A_STAGE_BYTES);
+                    a_tma_2d(dst, &map_kv, 0, krow, full0 + 8 * s);
+                    a_tma_2d(dst + A_PLANE, &map_kv, 64, krow, full0 + 8 * s);
+                    a_tma_2d(dst + 2 * A_PLANE, &map_kv, 0, krow + PAGE, full0 + 8 * s);
+                    a_tma_2d(dst + 3 * A_PLANE, &map_kv, 64, krow + PAGE, full0 + 8 * s);
+                }
+            }
+            if (__shfl_sync(0xffffffffu, ok, 0) == 0) {
+                if (lane == 0) *s_fail = 1;
+                break;
+            }
+        }
+    } else if (warp == 9) {
+        if (lane == 0) {
+            // ---- MMA issuer
+            bool ok = true;
+            auto issue_pv = [&](int t) {                                 // O_g += P_g V of tile t, both groups
+                const uint32_t st = base + (t % A_STAGES) * A_STAGE_BYTES;
+                for (int gq = 0; gq < 2 && ok; ++gq) {
+                    if (!a_bar_wait(p_ready0 + 8 * gq, t & 1)) { ok = false; break; }
+                    a_fence_after();
+                    const uint64_t pdesc = a_desc(base + A_OFF_P + gq * A_QPLANE, 16);
+                    const uint64_t vdesc = a_desc(st + 2 * A_PLANE, A_PLANE);     // the second 64 dims: one plane further
+#pragma unroll
+                    for (int j = 0; j < A_TILE / 16; ++j)                // 16 entries per instruction: P +32 bytes, V +2 row groups
+                        a_umma(tmem + 128 + gq * 128, pdesc + (uint64_t)(j * 32 >> 4), vdesc + (uint64_t)(j * 2048 >> 4), A_IDESC_PV,
+                               (t | j) != 0);
+                    a_commit(pv_done0 + 8 * gq);
+                }
+                if (ok) a_commit(empty0 + 8 * (t % A_STAGES));           // the stage is free when these MMAs have read it
+            };
+            for (int i = 0; i < ntile && ok; ++i) {
+                const int s = i % A_STAGES;
+                if (!a_bar_wait(full0 + 8 * s, (i / A_STAGES) & 1)) { ok = false; break; }
+                a_fence_after();
+                const uint32_t st = base + s * A_STAGE_BYTES;
+                for (int gq = 0; gq < 2 && ok; ++gq) {                   // S_g = Q_g K^T of tile i
+                    if (i > 0) {
+                        if (!a_bar_wait(s_free0 + 8 * gq, (i - 1) & 1)) { ok = false; break; }
+                        a_fence_after();
+                    }
+#pragma unroll
+                    for (int p = 0; p < 2; ++p) {
+                        const uint64_t qdesc = a_desc(base + A_OFF_Q + (gq * 2 + p) * A_QPLANE, 16);
+                        const uint64_t kdesc = a_desc(st + p * A_PLANE, 16);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)                      // 16 of d per instruction: 32 bytes along the row
+                            a_umma(tmem + gq * 64, qdesc + (uint64_t)(j * 32 >> 4), kdesc + (uint64_t)(j * 32 >> 4), A_IDESC_S,
+                                   (p | j) != 0);
+                    }
+                    a_commit(s_ready0 + 8 * gq);
+                }
+                if (ok && i > 0) issue_pv(i - 1);
+            }
+            if (ok) issue_pv(ntile - 1);
+            if (!ok) *s_fail = 1;
+        }
+    } else {
+        // ---- softmax warps
+        const uint32_t lane_addr = tmem + ((uint32_t)(wl * 32) << 16);
+        const uint32_t s_col = (uint32_t)(grp * 64), o_col = (uint32_t)(128 + grp * 128);
+        unsigned char* prow = gen + A_OFF_P + grp * A_QPLANE + r * 128;
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int i = 0; i < ntile; ++i) {
+            ok = __all_sync(0xffffffffu, a_bar_wait(s_ready0 + 8 * grp, i & 1));
+            if (!ok) break;
+            a_fence_after();
+            uint32_t sv[64];
+            a_tmem_ld32(lane_addr + s_col, sv);
+            a_tmem_ld32(lane_addr + s_col + 32, sv + 32);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            a_fence_before();
+            __syncwarp();
+            if (lane == 0) a_bar_arrive(s_free0 + 8 * grp);              // S may be overwritten by the next tile's product
+            const int e0 = i * A_TILE;
+            float mx = -INFINITY;
+            if (e0 + A_TILE <= limit) {
+#pragma unroll
+                for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
+            } else {
+#pragma unroll
+                for (int e = 0; e < 64; ++e) {
+                    const float v = (e0 + e < limit) ? __uint_as_float(sv[e]) : -INFINITY;
+                    sv[e] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+            }
+            const float m_new = mx * scale_log2;                         // scale_log2 > 0
+            const bool resc = __any_sync(0xffffffffu, m_new > m_used + A_RESCALE_STEP);
+            float alpha = 1.0f;
+            if (resc) {
+                const float mn = fmaxf(m_used, m_new);
+                alpha = (m_used == -INFINITY) ? 0.0f : exp2f(m_used - mn);
+                m_used = mn;
+            }
+            const float mref = (m_used == -INFINITY) ? 0.0f : m_used;    // a row that has seen nothing yet: every p = 0
+            float sum = 0.f;
+            uint32_t pk[32];
+#pragma unroll
+            for (int e = 0; e < 64; e += 2) {
+                const float p0 = exp2f(fmaf(__uint_as_float(sv[e]), scale_log2, -mref));
+                const float p1 = exp2f(fmaf(__uint_as_float(sv[e + 1]), scale_log2, -mref));
+                sum += p0 + p1;
+                const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+                pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&pp);
+            }
+            l = l * alpha + sum;
+            if (i > 0) {                                                 // P V of the previous tile: O complete, P buffer free
+                ok = __all_sync(0xffffffffu, a_bar_wait(pv_done0 + 8 * grp, (i - 1) & 1));
+                if (!ok) break;
+                a_fence_after();
+                if (resc) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t ov[32];
+                        a_tmem_ld32(lane_addr + o_col + c * 32, ov);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+                        a_tmem_st32(lane_addr + o_col + c * 32, ov);
+                    }
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            a_fence_before();
+            __syncwarp();
+            if (lane == 0) a_bar_arrive(p_ready0 + 8 * grp);
+        }
+        if (ok) ok = __all_sync(0xffffffffu, a_bar_wait(pv_done0 + 8 * grp, (ntile - 1) & 1));
+        if (!ok) {
+            if (lane == 0) *s_fail = 1;
+        } else {
+            a_fence_after();
+            const float inv = l > 0.f ? 1.0f / l : 0.f;
+            uint4* op = reinterpret_cast<uint4*>(out + (((size_t)b * n_new + (valid ? tok : 0)) * Hq + (size_t)h * g + head) * 128);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t ov[32];
+                a_tmem_ld32(lane_addr + o_col + c * 32, ov);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int k2 = 0; k2 < 4; ++k2) {
+                            const __nv_bfloat162 pp = __floats2bfloat162_rn(__uint_as_float(ov[e + 2 * k2]) * inv,
+                                                                             __uint_as_float(ov[e + 2 * k2 + 1]) * inv);
+                            w[k2] = *reinterpret_cast<const uint32_t*>(&pp);
+                        }
+                        op[c * 4 + (e >> 3)] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+        }
+    }
+    a_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(A_TMEM_COLS) : "memory");
+    }
+    if (threadIdx.x == 0 && *s_fail) latch_error(cv.err, TRIMKV_E_TIMEOUT);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ host side
+struct PrefillTcState {
+    CUtensorMap map_kv;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFnA)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFnA a_encode_fn() {
+    static EncodeTiledFnA fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFnA>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool prefill_tc_supported(const CacheView& cv, int is_bf16, int Hq) {
+    const int g = cv.H > 0 ? Hq / cv.H : 0;
+    const long long rows = (long long)cv.B * cv.P_seq * 2 * PAGE;
+    return is_bf16 && cv.d == 128 && cv.swizzle && g >= 1 && g <= 128 && rows < (1LL << 31);
+}
+
+// The arena kv[b][page][2][64][256 bytes] as a bf16 matrix [rows][128]; box 64 columns x 64 rows, no swizzle (the rows
+// are stored permuted already), nothing is ever read outside it.
+PrefillTcState* prefill_tc_create(const CacheView& cv, int is_bf16, int Hq) {
+    if (!prefill_tc_supported(cv, is_bf16, Hq)) return nullptr;
+    EncodeTiledFnA fn = a_encode_fn();
+    if (!fn) return nullptr;
+    PrefillTcState* s = new PrefillTcState();
+    const cuuint64_t dims[2] = {128, (cuuint64_t)cv.B * (cuuint64_t)cv.P_seq * 2 * PAGE};
+    const cuuint64_t strides[1] = {256};
+    const cuuint32_t box[2] = {64, (cuuint32_t)A_TILE};
+    const cuuint32_t estr[2] = {1, 1};
+    const bool ok = fn(&s->map_kv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, cv.kv, dims, strides, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS &&
+                    cudaFuncSetAttribute(prefill_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, A_SMEM) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        delete s;
+        return nullptr;
+    }
+    return s;
+}
+
+void prefill_tc_destroy(PrefillTcState* s) { delete s; }
+
+// Rows of a block that carry a query: worth it once at least half of the 256 do.
+bool prefill_tc_wanted(const CacheView& cv, int n_new, int Hq) { return (long long)n_new * (Hq / cv.H) >= 128; }
+
+void launch_prefill_attention_tc(const PrefillTcState* s, const CacheView& cv, int layer, int n_new, int Hq, const void* q,
+                                 void* out, cudaStream_t st) {
+    const int g = Hq / cv.H;
+    const int tt = 256 / g;
+    dim3 grid((n_new + tt - 1) / tt, cv.B * cv.H);
+    prefill_attn_tc_kernel<<<grid, A_THREADS, A_SMEM, st>>>(s->map_kv, cv, layer, n_new, g, Hq, (const __nv_bfloat16*)q,
+                                                            (__nv_bfloat16*)out, 1.4426950408889634f / sqrtf((float)cv.d));
+    count_launch();
+}
+
+}  // namespace tkv

@@ -196,8 +196,16 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
                       void* out, cudaStream_t st, PhaseMarker* pm);
 
 // Causal attention of the chunk of n_new tokens just appended to `layer`; q, out: [B, n_new, Hq, d].
-void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const void* q, void* out,
-                              cudaStream_t st);
+// tc: state of the tensor-core (tcgen05) form, or null; used when the chunk is large enough to fill its tiles.
+struct PrefillTcState;
+bool prefill_tc_supported(const CacheView& cv, int is_bf16, int Hq);
+PrefillTcState* prefill_tc_create(const CacheView& cv, int is_bf16, int Hq);
+void prefill_tc_destroy(PrefillTcState* s);
+bool prefill_tc_wanted(const CacheView& cv, int n_new, int Hq);
+void launch_prefill_attention_tc(const PrefillTcState* s, const CacheView& cv, int layer, int n_new, int Hq, const void* q,
+                                 void* out, cudaStream_t st);
+void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const PrefillTcState* tc,
+                              const void* q, void* out, cudaStream_t st);
 
 void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
                         void* v, int n, cudaStream_t st);

@@ -98,6 +98,7 @@ struct trimkv {
     char *st_k = nullptr, *st_v = nullptr, *st_q = nullptr, *st_out = nullptr;
     float *W1hi = nullptr, *W1lo = nullptr, *xhi = nullptr, *xlo = nullptr;   // 3xTF32 operands of the tensor-core gate
     GateTcState* tc = nullptr;
+    PrefillTcState* ptc = nullptr;   // tensor-core chunk attention (bf16, d = 128), else null
     float b_g;
     bool shared_set;
     std::vector<char> gate_set;
@@ -392,6 +393,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
             s = fail(TRIMKV_E_CUDA, "stream or event creation failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
     if (s == TRIMKV_OK) s = init_cache_state(h);
+    if (s == TRIMKV_OK) h->ptc = prefill_tc_create(h->cv, cfg->kv_dtype == TRIMKV_DTYPE_BF16, h->Hq);
     if (s != TRIMKV_OK) {
         char keep[sizeof(g_err)];
         memcpy(keep, g_err, sizeof(keep));
@@ -414,6 +416,7 @@ void trimkv_destroy(trimkv_t* h) {
     if (h->fast) cudaStreamDestroy(h->fast);
     for (void* p : h->allocs) cudaFree(p);
     gate_tc_destroy(h->tc);
+    prefill_tc_destroy(h->ptc);
     delete h;
 }
 
@@ -514,7 +517,7 @@ trimkv_status trimkv_prefill_attention(trimkv_t* h, int layer, int n_new, const 
     PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
     cudaStream_t st = (cudaStream_t)stream;
     if (pm) pm->mark(PH_ATTN_MAIN, 0, st);
-    launch_prefill_attention(h->cv, layer, n_new, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, q, out, st);
+    launch_prefill_attention(h->cv, layer, n_new, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, h->ptc, q, out, st);
     if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
