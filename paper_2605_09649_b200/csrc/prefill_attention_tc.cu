@@ -116,6 +116,38 @@ __device__ __forceinline__ void a_tmem_st32(uint32_t taddr, const uint32_t* t) {
         "r"(t[31])
         : "memory");
 }
+// Two fp32 values per 64-bit register: the packed fma / add forms halve the instruction count of the softmax loop.
+__device__ __forceinline__ uint64_t a_pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void a_unpack2(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t a_fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t a_add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float a_ex2(float x) {                      // 2^x, one instruction; 2^-inf = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float a_max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t a_bf16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 __device__ __forceinline__ void a_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void a_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -273,18 +305,19 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
             __syncwarp();
             if (lane == 0) a_bar_arrive(s_free0 + 8 * grp);              // S may be overwritten by the next tile's product
             const int e0 = i * A_TILE;
-            float mx = -INFINITY;
-            if (e0 + A_TILE <= limit) {
+            if (e0 + A_TILE > limit) {                                   // the tile crosses this row's causal limit
 #pragma unroll
-                for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
-            } else {
-#pragma unroll
-                for (int e = 0; e < 64; ++e) {
-                    const float v = (e0 + e < limit) ? __uint_as_float(sv[e]) : -INFINITY;
-                    sv[e] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
-                }
+                for (int e = 0; e < 64; ++e)
+                    if (e0 + e >= limit) sv[e] = 0xff800000u;            // -inf
             }
+            float mq[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four independent chains
+#pragma unroll
+            for (int e = 0; e < 64; e += 8) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    mq[c] = a_max3(mq[c], __uint_as_float(sv[e + 2 * c]), __uint_as_float(sv[e + 2 * c + 1]));
+            }
+            const float mx = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
             const float m_new = mx * scale_log2;                         // scale_log2 > 0
             const bool resc = __any_sync(0xffffffffu, m_new > m_used + A_RESCALE_STEP);
             float alpha = 1.0f;
@@ -294,15 +327,23 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                 m_used = mn;
             }
             const float mref = (m_used == -INFINITY) ? 0.0f : m_used;    // a row that has seen nothing yet: every p = 0
-            float sum = 0.f;
+            const uint64_t sc2 = a_pack2(scale_log2, scale_log2), nm2 = a_pack2(-mref, -mref);
+            uint64_t sq[4] = {0ull, 0ull, 0ull, 0ull};                   // packed partial sums, four chains
             uint32_t pk[32];
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
-                const float p0 = exp2f(fmaf(__uint_as_float(sv[e]), scale_log2, -mref));
-                const float p1 = exp2f(fmaf(__uint_as_float(sv[e + 1]), scale_log2, -mref));
-                sum += p0 + p1;
-                const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-                pk[e >> 1] = *reinterpret_cast<const uint32_t*>(&pp);
+                const uint64_t x2 = a_fma2(a_pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), sc2, nm2);
+                float x0, x1;
+                a_unpack2(x2, x0, x1);
+                const float p0 = a_ex2(x0), p1 = a_ex2(x1);
+                sq[(e >> 1) & 3] = a_add2(sq[(e >> 1) & 3], a_pack2(p0, p1));
+                pk[e >> 1] = a_bf16x2(p0, p1);
+            }
+            float sum;
+            {
+                float a0, a1;
+                a_unpack2(a_add2(a_add2(sq[0], sq[1]), a_add2(sq[2], sq[3])), a0, a1);
+                sum = a0 + a1;
             }
             l = l * alpha + sum;
             if (i > 0) {                                                 // P V of the previous tile: O complete, P buffer free
