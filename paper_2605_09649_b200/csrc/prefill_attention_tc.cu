@@ -27,14 +27,13 @@ constexpr int A_PLANE = A_TILE * 128;                 // 8 KB: 64 entries x one 
 constexpr int A_STAGE_BYTES = 4 * A_PLANE;            // K half 0, K half 1, V half 0, V half 1
 constexpr int A_QPLANE = A_ROWS * 128;                // 16 KB: 128 query rows x one half
 constexpr int A_Q_BYTES = 2 * 2 * A_QPLANE;           // two groups, two halves
-constexpr int A_P_BYTES = 2 * A_QPLANE;               // two groups: 128 rows x 64 probabilities (bf16)
 constexpr int A_OFF_Q = A_STAGES * A_STAGE_BYTES;
-constexpr int A_OFF_P = A_OFF_Q + A_Q_BYTES;
-constexpr int A_OFF_BAR = A_OFF_P + A_P_BYTES;
+constexpr int A_OFF_BAR = A_OFF_Q + A_Q_BYTES;
 constexpr int A_SMEM = A_OFF_BAR + 256 + 1024;        // barriers and flags, alignment slack
-constexpr int A_THREADS = 320;
+constexpr int A_THREADS = 352;                       // 8 softmax warps, the TMA warp, one MMA-issuing warp per group
 constexpr unsigned A_WAIT_LIMIT = 1u << 22;
-constexpr int A_TMEM_COLS = 512;                      // S of group 0, 1: columns 0-63, 64-127; O: 128-255, 256-383
+constexpr int A_TMEM_COLS = 512;                      // S of group 0, 1: columns 0-63, 64-127; O: 128-255, 256-383;
+constexpr int A_COL_P = 384;                          // P (bf16 pairs, the A operand of P V): 384-415, 416-447
 constexpr float A_RESCALE_STEP = 8.0f;                // log2 units the running maximum may lag behind
 
 __device__ __forceinline__ uint32_t a_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -89,6 +88,15 @@ __device__ __forceinline__ void a_umma(uint32_t tmem_d, uint64_t adesc, uint64_t
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// A operand in tensor memory: row = lane, two bf16 per 32-bit column (lower k in the low half), 8 columns per K = 16.
+__device__ __forceinline__ void a_umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void a_commit(uint32_t bar) {
@@ -178,7 +186,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
     const int32_t* bt = cv.block_table + pool * cv.maxpp;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < A_STAGES; ++s) { a_bar_init(full0 + 8 * s, 1); a_bar_init(empty0 + 8 * s, 1); }
+        for (int s = 0; s < A_STAGES; ++s) { a_bar_init(full0 + 8 * s, 1); a_bar_init(empty0 + 8 * s, 2); }   // both issuers free a stage
         for (int gq = 0; gq < 2; ++gq) {
             a_bar_init(s_ready0 + 8 * gq, 1);
             a_bar_init(s_free0 + 8 * gq, 4);
@@ -241,47 +249,39 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                 break;
             }
         }
-    } else if (warp == 9) {
+    } else if (warp >= 9) {
         if (lane == 0) {
-            // ---- MMA issuer
+            // ---- MMA issuer of group gq: S of tile i, then P V of tile i - 1; the two issuers never wait for each other
+            const int gq = warp - 9;
             bool ok = true;
-            auto issue_pv = [&](int t) {                                 // O_g += P_g V of tile t, both groups
+            const uint32_t d_s = tmem + gq * 64, d_o = tmem + 128 + gq * 128, a_p = tmem + A_COL_P + gq * 32;
+            const uint64_t qdesc0 = a_desc(base + A_OFF_Q + (gq * 2) * A_QPLANE, 16), qdesc1 = a_desc(base + A_OFF_Q + (gq * 2 + 1) * A_QPLANE, 16);
+            auto issue_pv = [&](int t) {                                 // O += P V of tile t
                 const uint32_t st = base + (t % A_STAGES) * A_STAGE_BYTES;
-                for (int gq = 0; gq < 2 && ok; ++gq) {
-                    if (!a_bar_wait(p_ready0 + 8 * gq, t & 1)) { ok = false; break; }
-                    a_fence_after();
-                    const uint64_t pdesc = a_desc(base + A_OFF_P + gq * A_QPLANE, 16);
-                    const uint64_t vdesc = a_desc(st + 2 * A_PLANE, A_PLANE);     // the second 64 dims: one plane further
+                if (!a_bar_wait(p_ready0 + 8 * gq, t & 1)) { ok = false; return; }
+                a_fence_after();
+                const uint64_t vdesc = a_desc(st + 2 * A_PLANE, A_PLANE);         // the second 64 dims: one plane further
 #pragma unroll
-                    for (int j = 0; j < A_TILE / 16; ++j)                // 16 entries per instruction: P +32 bytes, V +2 row groups
-                        a_umma(tmem + 128 + gq * 128, pdesc + (uint64_t)(j * 32 >> 4), vdesc + (uint64_t)(j * 2048 >> 4), A_IDESC_PV,
-                               (t | j) != 0);
-                    a_commit(pv_done0 + 8 * gq);
-                }
-                if (ok) a_commit(empty0 + 8 * (t % A_STAGES));           // the stage is free when these MMAs have read it
+                for (int j = 0; j < A_TILE / 16; ++j)                    // 16 entries per instruction: P +8 columns, V +2 row groups
+                    a_umma_ts(d_o, a_p + j * 8, vdesc + (uint64_t)(j * 2048 >> 4), A_IDESC_PV, (t | j) != 0);
+                a_commit(pv_done0 + 8 * gq);
+                a_commit(empty0 + 8 * (t % A_STAGES));                   // this group is done with the stage
             };
             for (int i = 0; i < ntile && ok; ++i) {
                 const int s = i % A_STAGES;
                 if (!a_bar_wait(full0 + 8 * s, (i / A_STAGES) & 1)) { ok = false; break; }
+                if (i > 0 && !a_bar_wait(s_free0 + 8 * gq, (i - 1) & 1)) { ok = false; break; }
                 a_fence_after();
                 const uint32_t st = base + s * A_STAGE_BYTES;
-                for (int gq = 0; gq < 2 && ok; ++gq) {                   // S_g = Q_g K^T of tile i
-                    if (i > 0) {
-                        if (!a_bar_wait(s_free0 + 8 * gq, (i - 1) & 1)) { ok = false; break; }
-                        a_fence_after();
-                    }
+                const uint64_t kdesc0 = a_desc(st, 16), kdesc1 = a_desc(st + A_PLANE, 16);
 #pragma unroll
-                    for (int p = 0; p < 2; ++p) {
-                        const uint64_t qdesc = a_desc(base + A_OFF_Q + (gq * 2 + p) * A_QPLANE, 16);
-                        const uint64_t kdesc = a_desc(st + p * A_PLANE, 16);
+                for (int j = 0; j < 4; ++j)                              // S = Q K^T: 16 of d per instruction, 32 bytes along the row
+                    a_umma(d_s, qdesc0 + (uint64_t)(j * 32 >> 4), kdesc0 + (uint64_t)(j * 32 >> 4), A_IDESC_S, j != 0);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)                      // 16 of d per instruction: 32 bytes along the row
-                            a_umma(tmem + gq * 64, qdesc + (uint64_t)(j * 32 >> 4), kdesc + (uint64_t)(j * 32 >> 4), A_IDESC_S,
-                                   (p | j) != 0);
-                    }
-                    a_commit(s_ready0 + 8 * gq);
-                }
-                if (ok && i > 0) issue_pv(i - 1);
+                for (int j = 0; j < 4; ++j)
+                    a_umma(d_s, qdesc1 + (uint64_t)(j * 32 >> 4), kdesc1 + (uint64_t)(j * 32 >> 4), A_IDESC_S, 1u);
+                a_commit(s_ready0 + 8 * gq);
+                if (i > 0) issue_pv(i - 1);
             }
             if (ok) issue_pv(ntile - 1);
             if (!ok) *s_fail = 1;
@@ -290,7 +290,6 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
         // ---- softmax warps
         const uint32_t lane_addr = tmem + ((uint32_t)(wl * 32) << 16);
         const uint32_t s_col = (uint32_t)(grp * 64), o_col = (uint32_t)(128 + grp * 128);
-        unsigned char* prow = gen + A_OFF_P + grp * A_QPLANE + r * 128;
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < ntile; ++i) {
@@ -363,10 +362,8 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 }
             }
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            a_tmem_st32(lane_addr + A_COL_P + grp * 32, pk);             // P: the A operand of P V, two bf16 per column
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             a_fence_before();
             __syncwarp();
             if (lane == 0) a_bar_arrive(p_ready0 + 8 * grp);
