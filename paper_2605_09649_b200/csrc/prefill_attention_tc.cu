@@ -7,11 +7,13 @@
 // 128-byte half by (slot & 7); copied half by half with TMA (box 64 columns x 64 rows of the arena seen as a matrix of
 // 256-byte rows) they land in shared memory exactly in the tensor core's 128-byte-swizzle layout: K halves as K-major
 // operands of S = Q K^T, V halves as MN-major operands of O += P V.  Roles: warps 0-3 / 4-7 are the softmax warps of
-// group 0 / 1 (a thread owns one row: S read from tensor memory, masked, exponentiated, P written back to shared memory
-// as bf16), warp 8 issues the TMA copies into a 4-stage ring, warp 9 issues the MMAs (S of tile i + 1 before P V of tile i,
-// so the tensor pipe works while the softmax warps compute).  O accumulates in tensor memory; the running maximum is only
-// raised (and O rescaled) when it grows by more than 2^8, which keeps every exponential finite and leaves the final O / l
-// unchanged.  Every wait is bounded; a wait that runs out latches TRIMKV_E_TIMEOUT.
+// group 0 / 1 (a thread owns one row: S read from tensor memory, masked, exponentiated, P written back to tensor memory as
+// bf16 pairs, where the P V product reads it as its A operand), warp 8 issues the TMA copies into a 4-stage ring, warps 9
+// and 10 each issue the MMAs of one group (S of tile i + 1 before P V of tile i, so the tensor pipe works while the
+// softmax warps compute, and neither group's issuer ever waits for the other group).  O accumulates in tensor memory; the
+// running maximum is only raised (and O rescaled) when it grows by more than 2^8, which keeps every exponential finite and
+// leaves the final O / l unchanged.  A third of the exponentials are evaluated with FMAs instead of the special-function
+// unit.  Every wait is bounded; a wait that runs out latches TRIMKV_E_TIMEOUT.
 #include <cuda.h>
 
 #include "trimkv_internal.cuh"
@@ -34,6 +36,7 @@ constexpr int A_THREADS = 352;                       // 8 softmax warps, the TMA
 constexpr unsigned A_WAIT_LIMIT = 1u << 22;
 constexpr int A_TMEM_COLS = 512;                      // S of group 0, 1: columns 0-63, 64-127; O: 128-255, 256-383;
 constexpr int A_COL_P = 384;                          // P (bf16 pairs, the A operand of P V): 384-415, 416-447
+constexpr int A_POLY_EVERY = 3;                       // share of the exponentials computed with FMAs: 1 / A_POLY_EVERY
 constexpr float A_RESCALE_STEP = 8.0f;                // log2 units the running maximum may lag behind
 
 __device__ __forceinline__ uint32_t a_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -145,6 +148,26 @@ __device__ __forceinline__ float a_ex2(float x) {                      // 2^x, o
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// 2^x for two values on the FMA pipe (the special-function unit is the softmax loop's narrowest pipe, so a share of the
+// exponentials goes this way): x = n + f with n = round(x) taken from the mantissa of x + 1.5 * 2^23 and f in [-1/2, 1/2];
+// 2^f by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); n is added into the exponent field.
+// x is clamped at -125 from below, so a masked entry weighs 2^-125 instead of 0.
+__device__ __forceinline__ void a_exp2_fma2(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    a_unpack2(x2, x0, x1);
+    const uint64_t xc = a_pack2(fmaxf(x0, -125.0f), fmaxf(x1, -125.0f));
+    const uint64_t magic = a_pack2(12582912.0f, 12582912.0f), nmagic = a_pack2(-12582912.0f, -12582912.0f);
+    const uint64_t t2 = a_add2(xc, magic);
+    const uint64_t f2 = a_fma2(a_add2(t2, nmagic), a_pack2(-1.0f, -1.0f), xc);
+    uint64_t q2 = a_fma2(a_pack2(0.055171650f, 0.055171650f), f2, a_pack2(0.24261113f, 0.24261113f));
+    q2 = a_fma2(q2, f2, a_pack2(0.69326097f, 0.69326097f));
+    q2 = a_fma2(q2, f2, a_pack2(0.99992806f, 0.99992806f));
+    float q0, q1, t0, t1;
+    a_unpack2(q2, q0, q1);
+    a_unpack2(t2, t0, t1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
 }
 __device__ __forceinline__ float a_max3(float a, float b, float c) {
     float d;
@@ -332,9 +355,15 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
                 const uint64_t x2 = a_fma2(a_pack2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), sc2, nm2);
-                float x0, x1;
-                a_unpack2(x2, x0, x1);
-                const float p0 = a_ex2(x0), p1 = a_ex2(x1);
+                float p0, p1;
+                if ((e >> 1) % A_POLY_EVERY == A_POLY_EVERY - 1) {       // every A_POLY_EVERY-th pair on the FMA pipe
+                    a_exp2_fma2(x2, p0, p1);
+                } else {
+                    float x0, x1;
+                    a_unpack2(x2, x0, x1);
+                    p0 = a_ex2(x0);
+                    p1 = a_ex2(x1);
+                }
                 sq[(e >> 1) & 3] = a_add2(sq[(e >> 1) & 3], a_pack2(p0, p1));
                 pk[e >> 1] = a_bf16x2(p0, p1);
             }
