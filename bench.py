@@ -44,6 +44,16 @@ def load_peaks():
     return 6650.0, "fallback"
 
 
+def load_tensor_peaks():
+    """Measured dense bf16 matmul rates: burst (a kernel timed alone) and sustained (inside a long run), TFLOP/s."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        d = json.load(open(p))
+        return {"burst": float(d["bf16_tflops"]), "sustained": float(d["bf16_tflops_sustained"]), "kind": "measured"}
+    except Exception:
+        return {"burst": 1590.0, "sustained": 1400.0, "kind": "fallback"}
+
+
 def algorithmic_bytes(w, entries_per_seq):
     """Bytes one decode step must move (per rank): every kept K/V row once, the per-entry retention metadata
     (lambda, c, position: 12 B) twice (histogram pass + filter pass), the gate weights once."""
@@ -211,7 +221,8 @@ def run_ours(args, w):
         ms, chunks, done = 0.0, 0, 0
         while done < count:
             n = min(w.chunk, count - done)
-            evs = []
+            evs, aevs = [], []
+            n_old = cache.lengths().to(torch.float64) if args.prefill_attention else None     # [B, L, H] before the chunk
             for l in range(w.layers):
                 x = workloads.hidden_states(w, seed, l, start + done, n, device=dev)
                 qc, k, v = workloads.project_qkv(w, bank, l, x)
@@ -219,17 +230,29 @@ def run_ours(args, w):
                 a.record()
                 cache.append(l, k, v, x=x)
                 if args.prefill_attention:
+                    a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a2.record()
                     cache.prefill_attention(l, qc)
+                    b2.record()
+                    aevs.append((a2, b2))
                 if l == w.layers - 1:
                     cache.score_and_evict()
                 b.record()
                 evs.append((a, b))
             torch.cuda.synchronize()
             ms += sum(a.elapsed_time(b) for a, b in evs)
+            if aevs:
+                # causal work of this chunk: query head (b, j, hq) sees n_old + j + 1 entries of its pool, 4 d flops each
+                fl = 4.0 * w.head_dim * (w.q_heads // w.kv_heads) * (n * n_old.sum().item() + n_old.numel() * n * (n + 1) / 2)
+                attn_stats["ms"] += sum(a.elapsed_time(b) for a, b in aevs)
+                attn_stats["flops"] += fl
+                attn_stats["last_ms"] = sum(a.elapsed_time(b) for a, b in aevs)
+                attn_stats["last_flops"] = fl
             chunks += 1
             done += n
         return ms, chunks
 
+    attn_stats = {"ms": 0.0, "flops": 0.0, "last_ms": 0.0, "last_flops": 0.0}
     t_setup = time.time()
     tokens_seen = 0
     prefill_ms, prefill_chunks, early_decode_ms, early_decode_steps = 0.0, 0, 0.0, 0
@@ -345,6 +368,7 @@ def run_ours(args, w):
         cache.close()
         return
     peak, peak_kind = load_peaks()
+    tpk = load_tensor_peaks()
     ab = algorithmic_bytes(w, entries + w.layers * w.kv_heads)
     if args.retention_bias:                                        # lambda and position of every entry ride along
         extra_b = w.batch * (entries + w.layers * w.kv_heads) * 8
@@ -373,7 +397,18 @@ def run_ours(args, w):
                    "prefill": {"chunks": prefill_chunks, "ms_per_chunk": prefill_ms / max(prefill_chunks, 1),
                                "tokens_per_s": w.batch * w.chunk / (prefill_ms / max(prefill_chunks, 1) * 1e-3) if prefill_ms > 0 else None,
                                "what": "gate + append of every layer and one eviction per chunk" +
-                                       (", with the chunk's causal attention" if args.prefill_attention else " (no chunk attention)")},
+                                       (", with the chunk's causal attention" if args.prefill_attention else " (no chunk attention)"),
+                               "chunk_attention": None if not args.prefill_attention else {
+                                   "kernel": "prefill_attn_tc_kernel (tcgen05) where the shapes allow, else mma.sync",
+                                   "last_chunk_ms_all_layers": attn_stats["last_ms"],
+                                   "last_chunk_tflops": attn_stats["last_flops"] / (attn_stats["last_ms"] * 1e-3) / 1e12 if attn_stats["last_ms"] > 0 else None,
+                                   "bound": "tensor", "peak_tflops_burst": tpk["burst"], "peak_tflops_sustained": tpk["sustained"],
+                                   "peak_kind": f"of {tpk['kind']}",
+                                   "frac_of_burst": (attn_stats["last_flops"] / (attn_stats["last_ms"] * 1e-3) / 1e12 / tpk["burst"])
+                                                    if attn_stats["last_ms"] > 0 else None,
+                                   "frac_of_sustained": (attn_stats["last_flops"] / (attn_stats["last_ms"] * 1e-3) / 1e12 / tpk["sustained"])
+                                                        if attn_stats["last_ms"] > 0 else None,
+                                   "flops": "causal: 4 d per (query head, visible entry); masked tile parts not counted"}},
                    "earlier_turn_decode_ms_per_step": early_decode_ms / early_decode_steps if early_decode_steps else None},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
@@ -458,6 +493,8 @@ def main():
                     help="the fixed per-head budget variant (every pool keeps budget / (layers * kv_heads) entries)")
     ap.add_argument("--prefill-attention", action="store_true",
                     help="also run the chunk's causal attention over the cache during the (untimed) prefill and report it")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="override the layer count, budget scaled with it (development and small profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
     ap.add_argument("--sweep-max", type=int, default=28)
@@ -472,6 +509,8 @@ def main():
         w = w.replace(context=args.context)
     if args.b_g is not None:
         w = w.replace(b_g=args.b_g)
+    if args.layers is not None:                       # a shallower model of the same shapes (small profiling captures)
+        w = w.replace(layers=args.layers, budget_entries=w.budget_entries // w.layers * args.layers)
     if args.impl == "reference":
         run_reference(args, w)
     else:
