@@ -134,3 +134,48 @@ def test_full_size_step_matches_oracle_on_samples(name, context, seq):
             np.testing.assert_array_equal(got, want, err_msg=f"kept set differs in pool ({seq},{l},{h})")
     assert (cache.select_stats()[:, 0] == 0).all()                     # the sampled candidate range held
     cache.close()
+
+
+@pytest.mark.parametrize("name,context", [("llama8b_32k", 4608), ("qwen_vl_16k", 2560), ("stress_128k", 8704)])
+def test_full_size_chunk_attention_matches_oracle_on_samples(name, context):
+    """trimkv_prefill_attention at the full shapes, cache at its budget, chunk of the workload's size: sampled (sequence,
+    token, query head) outputs against the oracle's fp64 attention over the entries that token may see (everything kept
+    from before the chunk, then the chunk's own tokens up to itself), read back from the device in pool order."""
+    w = workloads.WORKLOADS[name]
+    seed = 0
+    cache = binding.TrimKV.from_workload(w)
+    per_layer, w_g = workloads.gate_params(w, seed, device=DEV)
+    for l, p in enumerate(per_layer):
+        cache.set_gate(l, *p)
+    cache.set_shared_projection(w_g, w.b_g)
+    bank = workloads.ProjectionBank(w, seed, device=DEV)
+    _prefill(cache, w, bank, seed, context)
+    rng = np.random.default_rng(11)
+    n = w.chunk
+    g = w.group
+    qs = {}                                              # the chunk goes to every layer; three layers are checked
+    for l in range(w.layers):
+        x = workloads.hidden_states(w, seed, l, context, n, device=DEV)
+        q, k, v = workloads.project_qkv(w, bank, l, x)
+        cache.append(l, k, v, x=x)
+        if l in (0, w.layers // 2, w.layers - 1):
+            qs[l] = (q, cache.prefill_attention(l, q))
+    cache.sync_status()
+    lens = cache.lengths().numpy()
+    for l, (q, out) in qs.items():
+        for _ in range(3):
+            b, h = int(rng.integers(w.batch)), int(rng.integers(w.kv_heads))
+            total = int(lens[b, l, h])
+            n_old = total - n
+            assert n_old >= 0
+            _, _, _, kk, vv = cache.pool(b, l, h, total, with_kv=True)
+            kk, vv = to_np(kk).astype(np.float64), to_np(vv).astype(np.float64)
+            for j in (0, int(rng.integers(n)), n - 1):
+                for hq in (h * g, h * g + int(rng.integers(g))):
+                    vis = n_old + j + 1
+                    want = orc.attention(to_np(q[b, j, hq]), kk[:vis], vv[:vis])
+                    err = np.abs(to_np(out[b, j, hq]) - want).max()
+                    assert err <= 2e-2, f"chunk attention error {err} at (seq {b}, layer {l}, token {j}, head {hq})"
+    cache.score_and_evict()
+    cache.sync_status()
+    cache.close()
