@@ -162,6 +162,15 @@ TRIMKV_API trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x
  * caller's stream instead (same results; for per-kernel timing).  Synchronises. */
 TRIMKV_API trimkv_status trimkv_set_overlap(trimkv_t* h, int enable);
 
+/* Changes the horizon h = T - t of the retention score (Sec. 4.2, Eq. (global_score): ln G~ = (t+1-i) ln beta +
+ * ln sum_{k<h} beta^k; h = 1 gives the myopic score beta^(t+1-i), h = 0 stands for h -> infinity, the limit
+ * beta^(t+1-i) / (1 - beta) stated below the equation) for an existing cache, e.g. between eviction rounds: the
+ * beta-only term c of EVERY stored entry is recomputed on the device from its stored lambda = ln beta (fp32, the same
+ * routine that appends use), and later appends use the new horizon.  Entries, K/V and lambda are untouched; the next
+ * selection ranks by the new score.  horizon in [0, 64], else TRIMKV_E_ARG.  Asynchronous on `stream`, ordered like
+ * trimkv_score_and_evict (the caller orders it against decode steps on other streams). */
+TRIMKV_API trimkv_status trimkv_set_horizon(trimkv_t* h, int horizon, void* stream);
+
 /* Pool lengths to host memory, int32 [B, L, H].  Synchronises; reports latched device errors. */
 TRIMKV_API trimkv_status trimkv_get_lengths(trimkv_t* h, int32_t* out_host);
 

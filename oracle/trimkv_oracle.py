@@ -239,6 +239,15 @@ class OracleCache:
             self.V[layer][h] = np.concatenate([self.V[layer][h], v[:, h, :].astype(F64)])
         self.tokens[layer] = base + n
 
+    def set_horizon(self, horizon):
+        """Switch the horizon h = T - t of Eq. (global_score) for stored and future entries: the beta-only term
+        c = ln sum_{k<h} beta^k of every entry is recomputed from its stored fp32 lambda (h = 1: c = 0, the myopic
+        score; h = 0: the h -> inf limit -ln(1 - beta))."""
+        self.horizon = int(horizon)
+        for l in range(self.L):
+            for h in range(self.H):
+                self.c[l][h] = horizon_term_from_lambda32(self.lam[l][h], self.horizon)
+
     def total_entries(self):
         return sum(len(self.pos[l][h]) for l in range(self.L) for h in range(self.H))
 

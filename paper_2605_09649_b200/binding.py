@@ -23,7 +23,7 @@ EXPORTS = [
     "trimkv_default_config", "trimkv_create", "trimkv_create_ex", "trimkv_destroy", "trimkv_reset", "trimkv_set_gate",
     "trimkv_set_shared_projection", "trimkv_gate", "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention",
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
-    "trimkv_sync_status", "trimkv_set_overlap", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
+    "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static",
 ]
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
     L.trimkv_sync_status.argtypes = [vp]
     L.trimkv_profile.argtypes = [vp, i32]
     L.trimkv_set_overlap.argtypes = [vp, i32]
+    L.trimkv_set_horizon.argtypes = [vp, i32, vp]
     L.trimkv_profile_read.argtypes = [vp, vp, vp]
     L.trimkv_last_error.argtypes = []
     L.trimkv_last_error.restype = C.c_char_p
@@ -96,7 +97,7 @@ def lib() -> C.CDLL:
                  "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention", "trimkv_decode_step_all",
                  "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
                  "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_select_topk",
-                 "trimkv_select_topk_static", "trimkv_set_overlap"):
+                 "trimkv_select_topk_static", "trimkv_set_overlap", "trimkv_set_horizon"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -246,6 +247,10 @@ class TrimKV:
     def profile(self, enable):
         """False/0 off, True/1 every phase, 2 the attention kernel alone."""
         _check(lib().trimkv_profile(self._h, int(enable)))
+
+    def set_horizon(self, horizon: int):
+        """New horizon T - t for stored and future entries (0 = infinite)."""
+        _check(lib().trimkv_set_horizon(self._h, int(horizon), _stream()))
 
     def set_overlap(self, enable: bool):
         _check(lib().trimkv_set_overlap(self._h, 1 if enable else 0))

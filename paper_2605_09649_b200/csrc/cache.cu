@@ -278,6 +278,17 @@ __global__ void gather_pool_kernel(CacheView cv, int b, long long pool, int n, i
     }
 }
 
+// c = ln sum_{k<horizon} beta^k of every live entry, from its stored lambda (Eq. (global_score), the beta-only term).
+// One CTA per page; the page table says which pages are live and how far they are filled.
+__global__ void __launch_bounds__(PAGE)
+rehorizon_kernel(CacheView cv, int horizon) {
+    const size_t pg = (size_t)blockIdx.y * cv.P_seq + blockIdx.x;
+    const int4 ow = cv.owner[pg];
+    if (ow.x < 0 || (int)threadIdx.x >= ow.z) return;
+    const size_t slot = pg * PAGE + threadIdx.x;
+    cv.c[slot] = horizon_term_f32(cv.lam[slot], horizon);
+}
+
 }  // namespace
 
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
@@ -291,6 +302,12 @@ void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t*
                     cudaStream_t st) {
     const long long pools = (long long)cv.B * cv.L * cv.H;
     compact_kernel<<<(unsigned)pools, 256, 0, st>>>(cv, hole, mover, cursor, e_max);
+    count_launch();
+}
+
+void launch_rehorizon(const CacheView& cv, int horizon, cudaStream_t st) {
+    dim3 grid((unsigned)cv.P_seq, (unsigned)cv.B);
+    rehorizon_kernel<<<grid, PAGE, 0, st>>>(cv, horizon);
     count_launch();
 }
 

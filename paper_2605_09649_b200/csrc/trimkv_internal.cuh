@@ -207,6 +207,9 @@ void launch_prefill_attention_tc(const PrefillTcState* s, const CacheView& cv, i
 void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq, int is_bf16, const PrefillTcState* tc,
                               const void* q, void* out, cudaStream_t st);
 
+// Rewrites c of every stored entry from its lambda for a new horizon.
+void launch_rehorizon(const CacheView& cv, int horizon, cudaStream_t st);
+
 void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32_t* pos, float* lam, float* c, void* k,
                         void* v, int n, cudaStream_t st);
 

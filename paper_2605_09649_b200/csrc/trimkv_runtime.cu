@@ -695,6 +695,15 @@ trimkv_status trimkv_profile(trimkv_t* h, int enable) {
     return TRIMKV_OK;
 }
 
+trimkv_status trimkv_set_horizon(trimkv_t* h, int horizon, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (horizon < 0 || horizon > 64) return fail(TRIMKV_E_ARG, "horizon must be in [0, 64]");
+    h->cfg.horizon = horizon;
+    launch_rehorizon(h->cv, horizon, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
 trimkv_status trimkv_set_overlap(trimkv_t* h, int enable) {
     if (check_handle(h)) return TRIMKV_E_ARG;
     CUDA_TRY(cudaDeviceSynchronize());

@@ -690,3 +690,44 @@ def test_selection_fast_path_in_steady_state():
     assert (stats[:, 0] == 0).all(), stats
     assert (stats[:, 1] < 40000).all(), stats
     cache.close()
+
+
+def test_set_horizon_rescores_stored_entries():
+    """trimkv_set_horizon: c of every stored entry is recomputed on the device from its lambda (within 1e-5 relative of
+    the oracle's fp64 evaluation; the oracle then takes the device's fp32 values so that the kept sets can be compared
+    bit for bit), later appends use the new horizon, and the next evictions rank by the new score."""
+    w = BF16_SMALL.replace(budget_entries=700, horizon=2)
+    pair = Pair(w)
+    r = np.random.default_rng(77)
+    gen = torch.Generator(device=DEV); gen.manual_seed(77)
+    horizon = 2
+
+    def feed(n):
+        for l in range(w.layers):
+            k = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=gen, device=DEV).to(torch.bfloat16)
+            lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), distinct=int(r.choice([0, 3])), scale=0.3)
+            pair.append(l, k, k, lam, oracle_retention(lam, horizon))
+
+    feed(150); pair.evict(); pair.check_sets()
+    feed(70)                                             # entries of the old horizon, not yet evicted
+    for horizon in (1, 5, 0, 2):
+        pair.gpu.set_horizon(horizon)
+        for b in pair.seqs:
+            oc = pair.orc[b]
+            oc.set_horizon(horizon)
+            for l in range(w.layers):
+                for h in range(w.kv_heads):
+                    pos, lam, c, _, _ = pair.gpu.pool(b, l, h, len(oc.pos[l][h]) + 1, with_kv=False)
+                    order = np.argsort(pos.numpy(), kind="stable")
+                    np.testing.assert_array_equal(pos.numpy()[order], oc.pos[l][h])
+                    np.testing.assert_array_equal(lam.numpy()[order], oc.lam[l][h])
+                    got = c.numpy()[order]
+                    np.testing.assert_allclose(got, oc.c[l][h], rtol=1e-5, atol=1e-7)
+                    oc.c[l][h] = got.copy()
+        pair.evict(); pair.check_sets()
+        feed(33); pair.evict(); pair.check_sets()
+        feed(9)
+    with pytest.raises(binding.TrimkvError):
+        pair.gpu.set_horizon(65)
+    pair.gpu.sync_status()
+    pair.close()

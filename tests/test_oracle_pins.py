@@ -441,3 +441,51 @@ def test_prefill_attention_is_causal_dense_attention_when_nothing_was_evicted():
     o = c2.prefill_attention(0, q[8:10, :1])
     idx = sorted(p - 1 for p in kept) + [8]
     np.testing.assert_allclose(o[0, 0], orc.attention(q[8, 0], k[idx, 0], v[idx, 0]), rtol=1e-12)
+
+
+def test_set_horizon_rescoring_closed_forms():
+    """Switching the horizon re-scores stored entries (Eq. (global_score)): with h = 1 the score is the myopic
+    (t + 1 - i) ln beta, so with beta < 1 equal everywhere the M most recent (position, layer, head) triples survive;
+    for two betas, exp(S) must equal the direct sum over s = t+1 .. t+h of beta^(s - i) for the new h; and a cache
+    switched to h behaves exactly like one built with h from the start."""
+    L, H, d = 2, 2, 4
+    rng = np.random.default_rng(5)
+    lam = -np.abs(rng.normal(0, 0.3, size=(12, H))).astype(np.float32)
+    k = rng.normal(size=(12, H, d)).astype(np.float32)
+    a = orc.OracleCache(20, L, H, H, d, horizon=2)
+    ref = {h: orc.OracleCache(20, L, H, H, d, horizon=h) for h in (1, 5, 0)}
+    for l in range(L):
+        a.append(l, k, k, lam=lam)
+        for h in ref:
+            ref[h].append(l, k, k, lam=lam)
+    for h in (1, 5, 0):
+        a.set_horizon(h)
+        for l in range(L):
+            for hh in range(H):
+                np.testing.assert_array_equal(a.c[l][hh], ref[h].c[l][hh])
+        # direct sum of the definition, fp64
+        t = 12
+        i = a.pos[0][0].astype(np.float64)
+        beta = np.exp(a.lam[0][0].astype(np.float64))
+        S = orc.score(a.lam[0][0], a.c[0][0], a.pos[0][0], t).astype(np.float64)
+        if h > 0:
+            direct = sum(beta ** (s - i) for s in range(t + 1, t + h + 1))
+        else:
+            direct = beta ** (t + 1 - i) / (1.0 - beta)
+        np.testing.assert_allclose(np.exp(S), direct, rtol=2e-6)
+    a.set_horizon(1)
+    assert all((a.c[l][hh] == 0).all() for l in range(L) for hh in range(H))
+    a.score_and_evict()
+    ref[1].score_and_evict()
+    for l in range(L):
+        for hh in range(H):
+            np.testing.assert_array_equal(a.kept_positions(l, hh), ref[1].kept_positions(l, hh))
+    # equal beta < 1 and h = 1: pure recency, 20 = 5 * L * H entries -> the last 5 positions of every pool
+    b = orc.OracleCache(20, L, H, H, d, horizon=3)
+    for l in range(L):
+        b.append(l, k, k, lam=np.full((12, H), -0.1, np.float32))
+    b.set_horizon(1)
+    b.score_and_evict()
+    for l in range(L):
+        for hh in range(H):
+            np.testing.assert_array_equal(b.kept_positions(l, hh), np.arange(8, 13))
