@@ -90,6 +90,17 @@ struct ArraySrc {
 
 __device__ __forceinline__ u64 compose_key(uint32_t sc, uint32_t tie) { return ((u64)sc << 32) | (u64)(~tie); }
 
+// Float-domain forms of 32-bit key comparisons, for any non-NaN x:
+//   x <  key_float_lt(k)  iff  orderable_key(x) <  k        x <= key_float_le(k)  iff  orderable_key(x) <= k
+// Keys at or below that of -inf / at or above that of +inf (NaN bit patterns) clamp to -inf / +inf.  No float has the
+// key 0x7fffffff (it would be -0, which is folded onto +0): "<" there means "< -0", "<=" means "<= the key before it".
+__device__ __forceinline__ float key_float_lt(uint32_t key) {
+    if (key <= 0x007fffffu) return __uint_as_float(0xff800000u);         // at or below key(-inf)
+    if (key >= 0xff800000u) return __uint_as_float(0x7f800000u);         // at or above key(+inf)
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+__device__ __forceinline__ float key_float_le(uint32_t key) { return key_float_lt(key == 0x7fffffffu ? 0x7ffffffeu : key); }
+
 // ------------------------------------------------------------------ threshold search (one CTA, 256 threads)
 __device__ void threshold_scan(SelState* st, uint32_t* hist_b, long long k, long long n_total, bool last_pass,
                                unsigned cand_target) {
@@ -234,37 +245,44 @@ hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, un
         if (shift >= 32 && (lo & 0xffffffffull) == 0ull) {
             const uint32_t lo32 = (uint32_t)(lo >> 32);
             const int sh32 = shift - 32;
-            uint32_t smin = 0xffffffffu, smax = 0u;
+            // Most scores fall outside the binned range (it brackets the k-th key): two float compares settle those.
+            const u64 end64 = (u64)lo32 + ((u64)REG_BINS << sh32) - 1ull;
+            const float lo_f = key_float_lt(lo32);
+            const float hi_f = end64 >= 0xffffffffull ? __uint_as_float(0x7f800000u) : key_float_le((uint32_t)end64);
+            float fmin_ = __uint_as_float(0x7f800000u), fmax_ = __uint_as_float(0xff800000u);
             bool bad = false;
+            // Straight-line per score (no divergent branches: with a sixth of the scores inside the range nearly every
+            // warp would run both sides of one anyway): the in-range work is predicated.
             auto one = [&](float x) {
                 bad |= (x != x);
+                fmin_ = fminf(fmin_, x);
+                fmax_ = fmaxf(fmax_, x);
+                const bool below = x < lo_f;
+                under += below ? 1u : 0u;
                 const uint32_t sc = orderable_key(x);
-                smin = min(smin, sc);
-                smax = max(smax, sc);
-                if (sc < lo32) {
-                    ++under;
-                } else {
-                    const uint32_t bi = (sc - lo32) >> sh32;
-                    if (bi < (uint32_t)REG_BINS) atomicAdd(&sh[bi + 1], 1u);
-                }
+                const uint32_t bi = (sc - lo32) >> sh32;
+                if (!below && x <= hi_f && bi < (uint32_t)REG_BINS) atomicAdd(&sh[bi + 1], 1u);
             };
             const long long n4 = src.n >> 2;
             const float4* s4 = reinterpret_cast<const float4*>(src.s);
             const long long T = (long long)gridDim.x * blockDim.x;
-            for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += 4 * T) {
+            long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+            for (; i + 3 * T < n4; i += 4 * T) {                         // four 16-byte groups in flight per thread
                 float4 v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (i + u * T < n4) v[u] = __ldg(s4 + i + u * T);
+                for (int u = 0; u < 4; ++u) v[u] = __ldg(s4 + i + u * T);
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (i + u * T < n4) { one(v[u].x); one(v[u].y); one(v[u].z); one(v[u].w); }
+                for (int u = 0; u < 4; ++u) { one(v[u].x); one(v[u].y); one(v[u].z); one(v[u].w); }
+            }
+            for (; i < n4; i += T) {
+                const float4 v = __ldg(s4 + i);
+                one(v.x); one(v.y); one(v.z); one(v.w);
             }
             if (blockIdx.x == 0 && threadIdx.x < (int)(src.n & 3)) one(src.s[(n4 << 2) + threadIdx.x]);
             if (bad) latch_error(src.err, TRIMKV_E_NONFINITE);
-            if (smin <= smax) {
-                kmin = (u64)smin << 32;
-                kmax = ((u64)smax << 32) | 0xffffffffull;
+            if (fmin_ <= fmax_) {
+                kmin = (u64)orderable_key(fmin_) << 32;
+                kmax = ((u64)orderable_key(fmax_) << 32) | 0xffffffffull;
             }
             fast_done = true;
         }
@@ -449,73 +467,104 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
 
 // Filter pass for flat arrays.  A warp takes 512 consecutive scores per trip; lane l reads elements 32 j + l, so the
 // ballot over the lanes for a given j is already 32 consecutive bits of the eviction mask.
-__global__ void __launch_bounds__(256)
-flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, Cand* __restrict__ cb,
-                   long long cand_cap, u64* __restrict__ evict_mask, int32_t* err) {
+constexpr int FBUF = 64;                                 // candidates a warp stages before it takes a slice of the global list
+
+// Appends the warp's staged candidates to the global list (one atomic per flush).
+__device__ __noinline__ void flat_flush(Cand* wb, int nbuf, SelState* st, Cand* cb, long long cand_cap, int32_t* err) {
+    const int lane = threadIdx.x & 31;
+    unsigned wbase = 0;
+    if (lane == 0) wbase = atomicAdd(&st->cand_count, (unsigned)nbuf);
+    wbase = __shfl_sync(0xffffffffu, wbase, 0);
+    for (int i = lane; i < nbuf; i += 32) {
+        if ((long long)wbase + i < cand_cap) cb[(long long)wbase + i] = wb[i];
+        else latch_error(err, TRIMKV_E_NOMEM);
+    }
+    __syncwarp();
+}
+
+// Stages the candidates of one ballot (cdb: lanes whose score at flat index idx is a candidate); returns the new fill.
+__device__ __noinline__ int flat_stage(Cand* wb, int nbuf, unsigned cdb, float x, long long idx, SelState* st, Cand* cb,
+                                       long long cand_cap, int32_t* err) {
+    const int lane = threadIdx.x & 31;
+    const int cnt = __popc(cdb);
+    if (nbuf + cnt > FBUF) {
+        flat_flush(wb, nbuf, st, cb, cand_cap, err);
+        nbuf = 0;
+    }
+    if (cdb & (1u << lane)) {
+        Cand cnd;
+        cnd.key = compose_key(orderable_key(x), (uint32_t)idx);
+        cnd.slot = (u64)idx;
+        wb[nbuf + __popc(cdb & ((1u << lane) - 1u))] = cnd;
+    }
+    __syncwarp();
+    return nbuf + cnt;
+}
+
+// WHOLE: the candidate range is made of whole score values (its ends carry no index tie-break), the usual case after
+// histogram passes over score words: two float compares decide an entry (a NaN is neither evicted nor a candidate; the
+// histogram pass has flagged it).  Otherwise the 64-bit keys are compared.
+template <bool WHOLE>
+__device__ __forceinline__ void flat_filter_body(const float* __restrict__ s, long long n, SelState* __restrict__ st,
+                                                 Cand* __restrict__ cb, long long cand_cap, u64* __restrict__ evict_mask,
+                                                 int32_t* err, Cand* wb) {
     constexpr int J = 16;
     const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
     const uint32_t lo32 = (uint32_t)(c_lo >> 32), hi32 = (uint32_t)(c_hi >> 32);
+    const float lo_f = key_float_lt(lo32), hi_f = key_float_le(hi32);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long words = (n + 63) / 64;
     const long long nchunk = (n + 32 * J - 1) / (32 * J);
     const long long W = (long long)gridDim.x * (blockDim.x >> 5);
-    // Candidates go through a per-warp buffer so that the single global counter sees one atomic per ~50 candidates
-    // (a quarter of a million same-address atomics would serialise the whole pass).
-    constexpr int FBUF = 64;
-    __shared__ Cand sbuf[8][FBUF];
-    Cand* wb = sbuf[warp];
     int nbuf = 0;                                        // warp-uniform
-    auto flush = [&]() {
-        unsigned wbase = 0;
-        if (lane == 0) wbase = atomicAdd(&st->cand_count, (unsigned)nbuf);
-        wbase = __shfl_sync(0xffffffffu, wbase, 0);
-        for (int i = lane; i < nbuf; i += 32) {
-            if ((long long)wbase + i < cand_cap) cb[(long long)wbase + i] = wb[i];
-            else latch_error(err, TRIMKV_E_NOMEM);
+    auto decide = [&](float x, long long idx, bool& ev, bool& cd) {
+        if (WHOLE) {
+            ev = x < lo_f;
+            cd = !ev && x <= hi_f;
+        } else {
+            const uint32_t sc = orderable_key(x);
+            // one 32-bit compare settles an entry unless its score word equals that of a range end
+            ev = sc < lo32;
+            cd = !ev && sc <= hi32;
+            if (cd && (sc == lo32 || sc == hi32)) {
+                const u64 key = compose_key(sc, (uint32_t)idx);
+                ev = key < c_lo;
+                cd = !ev && key <= c_hi;
+            }
         }
-        __syncwarp();
-        nbuf = 0;
     };
-    const unsigned below_lane = (1u << lane) - 1u;
     for (long long c = (long long)blockIdx.x * (blockDim.x >> 5) + warp; c < nchunk; c += W) {
         const long long base = c * (32 * J);
         const long long rem = n - base;                  // elements left from the start of this chunk
         const float* p = s + base + lane;
         float x[J];
+        unsigned evb[J];
         if (rem >= 32 * J) {
 #pragma unroll
             for (int j = 0; j < J; ++j) x[j] = __ldg(p + 32 * j);
-        } else {
 #pragma unroll
-            for (int j = 0; j < J; ++j) x[j] = (32 * j + lane < rem) ? __ldg(p + 32 * j) : __int_as_float(0x7f800000);
-        }
-        unsigned evb[J];
-#pragma unroll
-        for (int j = 0; j < J; ++j) {
-            const uint32_t sc = orderable_key(x[j]);
-            // one 32-bit compare settles an entry unless its score word equals that of a range end
-            bool ev = sc < lo32;
-            bool cd = !ev && sc <= hi32;
-            if (cd && (sc == lo32 || sc == hi32)) {
-                const u64 key = compose_key(sc, (uint32_t)(base + 32 * j + lane));
-                ev = key < c_lo;
-                cd = !ev && key <= c_hi;
+            for (int j = 0; j < J; ++j) {
+                bool ev, cd;
+                decide(x[j], base + 32 * j + lane, ev, cd);
+                evb[j] = __ballot_sync(0xffffffffu, ev);
+                const unsigned cdb = __ballot_sync(0xffffffffu, cd);
+                if (cdb) nbuf = flat_stage(wb, nbuf, cdb, x[j], base + 32 * j + lane, st, cb, cand_cap, err);
             }
-            if (rem < 32 * J && 32 * j + lane >= rem) { ev = false; cd = false; }
-            evb[j] = __ballot_sync(0xffffffffu, ev);
-            const unsigned cdb = __ballot_sync(0xffffffffu, cd);
-            if (cdb) {                                   // stage the candidates in this warp's shared-memory buffer
-                const int cnt = __popc(cdb);
-                if (nbuf + cnt > FBUF) { flush(); }
-                if (cd) {
-                    const long long idx = base + 32 * j + lane;
-                    Cand cnd;
-                    cnd.key = compose_key(sc, (uint32_t)idx);
-                    cnd.slot = (u64)idx;
-                    wb[nbuf + __popc(cdb & below_lane)] = cnd;
-                }
-                nbuf += cnt;
-                __syncwarp();
+        } else {                                         // the ragged last chunk
+#pragma unroll 1
+            for (int j = 0; j < J; ++j) {
+                const bool live = 32 * j + lane < rem;
+                const float xv = live ? __ldg(p + 32 * j) : 0.0f;
+                bool ev, cd;
+                decide(xv, base + 32 * j + lane, ev, cd);
+                ev = ev && live;
+                cd = cd && live;
+                const unsigned e = __ballot_sync(0xffffffffu, ev);
+#pragma unroll
+                for (int q = 0; q < J; ++q)
+                    if (q == j) evb[q] = e;
+                const unsigned cdb = __ballot_sync(0xffffffffu, cd);
+                if (cdb) nbuf = flat_stage(wb, nbuf, cdb, xv, base + 32 * j + lane, st, cb, cand_cap, err);
             }
         }
         if (lane < J / 2) {
@@ -528,7 +577,21 @@ flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restric
             if (wi < words) evict_mask[wi] = wv;
         }
     }
-    if (nbuf > 0) flush();
+    if (nbuf > 0) flat_flush(wb, nbuf, st, cb, cand_cap, err);
+}
+
+__global__ void __launch_bounds__(256)
+flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, Cand* __restrict__ cb,
+                   long long cand_cap, u64* __restrict__ evict_mask, int32_t* err) {
+    // Candidates go through a per-warp buffer so that the single global counter sees one atomic per ~50 candidates
+    // (a quarter of a million same-address atomics would serialise the whole pass).
+    __shared__ Cand sbuf[8][FBUF];
+    Cand* wb = sbuf[threadIdx.x >> 5];
+    const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
+    if ((c_lo & 0xffffffffull) == 0ull && (c_hi & 0xffffffffull) == 0xffffffffull)
+        flat_filter_body<true>(s, n, st, cb, cand_cap, evict_mask, err, wb);
+    else
+        flat_filter_body<false>(s, n, st, cb, cand_cap, evict_mask, err, wb);
 }
 
 // ------------------------------------------------------------------ sample bracket (cache path)

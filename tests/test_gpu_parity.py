@@ -590,8 +590,16 @@ def _unpack(keep_words, n):
 
 @pytest.mark.parametrize("n", [1, 63, 64, 65, 1000, 4097, (1 << 20) + 3])
 def test_select_topk_matches_full_sort(n):
-    for kind in ("uniform", "equal", "two", "special"):
-        if kind == "uniform":
+    for kind in ("uniform", "equal", "two", "special", "around_zero"):
+        if kind == "around_zero":
+            # both signs, denormals and the two zeros: histogram bin edges then fall on the sign boundary of the key space
+            s = (workloads.selection_scores(n, seed=n + 3, device=DEV) + 4.0) * 3e-39
+            idx = torch.arange(n, device=DEV)
+            s = torch.where(idx % 5 == 0, torch.zeros_like(s), s)
+            s = torch.where(idx % 9 == 0, -torch.zeros_like(s), s)
+            s = torch.where(idx % 23 == 0, torch.full_like(s, 1.4e-45), s)
+            s = torch.where(idx % 29 == 0, torch.full_like(s, -1.4e-45), s)
+        elif kind == "uniform":
             s = workloads.selection_scores(n, seed=n, device=DEV)
         elif kind == "equal":
             s = torch.full((n,), -0.75, device=DEV)
