@@ -580,7 +580,7 @@ __device__ __forceinline__ void flat_filter_body(const float* __restrict__ s, lo
     if (nbuf > 0) flat_flush(wb, nbuf, st, cb, cand_cap, err);
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)                // the grid is sized for four CTAs per SM
 flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, Cand* __restrict__ cb,
                    long long cand_cap, u64* __restrict__ evict_mask, int32_t* err) {
     // Candidates go through a per-warp buffer so that the single global counter sees one atomic per ~50 candidates
