@@ -5,7 +5,7 @@
 // Proj's second layer and the shared readout are both linear, so they compose exactly:
 //   s = w_g . (W2 u + b2) + b_g = v . u + s0,  v[l,h,:] = W2[l,h]^T w_g,  s0[l,h] = w_g . b2[l,h] + b_g.
 // v and s0 are folded once when the weights are set (fp64 accumulation); per token the gate then
-// streams W1 once (the bulk of the bytes) and 2 KB of v per (layer, head).
+// streams W1 once (the bulk of the bytes; stored transposed, input dimension major) and 2 KB of v per (layer, head).
 //
 // fp32 CUDA-core arithmetic: at decode the op streams the weights once (HBM bound); the 1e-5
 // relative output tolerance excludes single-pass bf16/tf32 tensor-core math.
@@ -15,35 +15,15 @@ namespace tkv {
 
 namespace {
 
-constexpr int GH_WARPS = 8;    // warps per CTA of the hidden-layer kernel
-constexpr int GH_DC = 512;     // floats of the input dimension per CTA (its x tile lives in shared memory)
-constexpr int GH_RW = 8;       // rows per CTA
-constexpr int GH_JP = 2;       // hidden units per warp pass
-constexpr int GH_JSPLIT = 4;   // CTAs that share the hidden units of one (layer, input chunk)
+constexpr int GH_THREADS = 128;  // threads per CTA of the hidden-layer kernel; a thread owns 4 consecutive hidden units
+constexpr int GH_DC = 128;       // input dimensions per CTA (its x tile lives in shared memory)
+constexpr int GH_RW = 8;         // rows per CTA
+constexpr int GH_U = 8;          // input dimensions (16-byte weight loads per lane) in flight
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
-}
-
-// Sums 16 per-lane values over the warp with 20 shuffles: afterwards lanes 0..15 hold the warp totals of v[0..15].
-__device__ __forceinline__ float warp_transpose_sum16(float (&v)[16], int lane) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], 16);   // fold the two half-warps
-#pragma unroll
-    for (int s = 8, n = 16; s >= 1; s >>= 1, n >>= 1) {
-        const bool upper = (lane & s) != 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (i < n / 2) {
-                const float send = upper ? v[i] : v[i + n / 2];
-                const float keep = upper ? v[i + n / 2] : v[i];
-                v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
-            }
-        }
-    }
-    return v[0];
 }
 
 __device__ __forceinline__ float4 ld_stream(const float* p) {   // read-once data: do not keep it in L1
@@ -72,71 +52,76 @@ gate_fold_kernel(const float* __restrict__ W2, const float* __restrict__ b2, con
     }
 }
 
-// Partial pre-activations: zpart[lb][chunk][r][j] = x[lb][r][chunk] . W1[layer][j][chunk] for GH_RW rows, one
-// GH_DC-float chunk of the input dimension and a quarter of the hidden units per CTA.  The x tile is staged in
-// shared memory once and W1 is streamed past it, two hidden units per warp pass with eight 16-byte loads in flight
-// per lane.  grid = (row tiles * chunks, GH_JSPLIT, layers): CTAs that share a slice of W1 are neighbours in launch
-// order (chunked-prefill calls re-read W1 from L2).
-__global__ void __launch_bounds__(GH_WARPS * 32, 2)
-gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1, float* __restrict__ zpart, int layer0,
+// Partial pre-activations: zpart[lb][chunk][r][j] = sum over the chunk's input dimensions d of x[lb][r][d] W1[layer][j][d],
+// for GH_RW rows and one GH_DC-wide chunk of the input dimension per CTA.  W1 is kept transposed (W1T[layer][d][j]): a
+// thread owns four consecutive hidden units, so a warp's weight load is 512 contiguous bytes, the x values of a dimension
+// are one broadcast read of shared memory for the whole warp, and every thread finishes its own sums (no shuffles).
+// GH_U dimensions are in flight per thread.  grid = (row tiles * chunks, ceil(dg / 512), layers).
+__global__ void __launch_bounds__(GH_THREADS)
+gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1T, float* __restrict__ zpart, int layer0,
                    int R, int D, int dg, int nchunk) {
-    __shared__ __align__(16) float xs[GH_RW][GH_DC];
+    __shared__ __align__(16) float xs[GH_DC][GH_RW];
     const int lb = blockIdx.z;
     const int layer = layer0 + lb;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int chunk = blockIdx.x % nchunk;
     const int r0 = (blockIdx.x / nchunk) * GH_RW;
     const int nr = min(GH_RW, R - r0);
     const int dbase = chunk * GH_DC;
-    const int jper = (dg + GH_JSPLIT - 1) / GH_JSPLIT;
-    const int jbeg = blockIdx.y * jper, jend = min(dg, jbeg + jper);
-
-    for (int i = threadIdx.x; i < GH_RW * (GH_DC / 4); i += blockDim.x) {
-        const int rr = i / (GH_DC / 4), dd = (i % (GH_DC / 4)) * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (rr < nr && dbase + dd < D) v = __ldg(reinterpret_cast<const float4*>(x + ((size_t)lb * R + r0 + rr) * D + dbase + dd));
-        *reinterpret_cast<float4*>(&xs[rr][dd]) = v;
+    const int dn = min(GH_DC, D - dbase);
+    for (int i = threadIdx.x; i < GH_DC * GH_RW; i += blockDim.x) {
+        const int rr = i / GH_DC, dd = i % GH_DC;
+        xs[dd][rr] = (rr < nr && dd < dn) ? __ldg(x + ((size_t)lb * R + r0 + rr) * D + dbase + dd) : 0.f;
     }
     __syncthreads();
-
-    const float* Wl = W1 + (size_t)layer * dg * D + dbase;
-    float* zp = zpart + (((size_t)lb * nchunk + chunk) * R + r0) * dg;
-    for (int j0 = jbeg + warp * GH_JP; j0 < jend; j0 += GH_WARPS * GH_JP) {
-        float4 w[GH_JP][GH_DC / 128];
+    const int j = (blockIdx.y * GH_THREADS + threadIdx.x) * 4;
+    if (j >= dg) return;
+    const float* Wp = W1T + ((size_t)layer * D + dbase) * dg + j;
+    float acc[4][GH_RW];
 #pragma unroll
-        for (int jj = 0; jj < GH_JP; ++jj)
+    for (int q = 0; q < 4; ++q)
 #pragma unroll
-            for (int sl = 0; sl < GH_DC / 128; ++sl) {
-                const int dd = sl * 128 + lane * 4;
-                w[jj][sl] = (j0 + jj < jend && dbase + dd < D) ? ld_stream(Wl + (size_t)(j0 + jj) * D + dd)
-                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        float acc[GH_JP * GH_RW];
+        for (int rr = 0; rr < GH_RW; ++rr) acc[q][rr] = 0.f;
+    // the weights of the next GH_U dimensions are requested before those of the current ones are used
+    float4 w[GH_U], wn[GH_U];
+    auto fetch = [&](float4 (&dst)[GH_U], int d0) {
 #pragma unroll
-        for (int a = 0; a < GH_JP * GH_RW; ++a) acc[a] = 0.f;
+        for (int u = 0; u < GH_U; ++u)
+            dst[u] = (d0 + u < dn) ? ld_stream(Wp + (size_t)(d0 + u) * dg) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    fetch(w, 0);
+    for (int d0 = 0; d0 < dn; d0 += GH_U) {
+        fetch(wn, d0 + GH_U);
 #pragma unroll
-        for (int sl = 0; sl < GH_DC / 128; ++sl) {
+        for (int u = 0; u < GH_U; ++u) {
+            const float4 xa = *reinterpret_cast<const float4*>(&xs[d0 + u][0]);   // rows 0-3 (zero beyond dn)
+            const float4 xb = *reinterpret_cast<const float4*>(&xs[d0 + u][4]);   // rows 4-7
+            const float xr[GH_RW] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+            const float wq[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
-            for (int rr = 0; rr < GH_RW; ++rr) {
-                const float4 xv = *reinterpret_cast<const float4*>(&xs[rr][sl * 128 + lane * 4]);
+            for (int q = 0; q < 4; ++q)
 #pragma unroll
-                for (int jj = 0; jj < GH_JP; ++jj) {
-                    float a = acc[jj * GH_RW + rr];
-                    a = fmaf(xv.x, w[jj][sl].x, a);
-                    a = fmaf(xv.y, w[jj][sl].y, a);
-                    a = fmaf(xv.z, w[jj][sl].z, a);
-                    a = fmaf(xv.w, w[jj][sl].w, a);
-                    acc[jj * GH_RW + rr] = a;
-                }
-            }
+                for (int rr = 0; rr < GH_RW; ++rr) acc[q][rr] = fmaf(xr[rr], wq[q], acc[q][rr]);
         }
-        static_assert(GH_JP * GH_RW == 16, "the warp reduction below sums exactly 16 values");
-        const float tot = warp_transpose_sum16(acc, lane);      // lane = jj * GH_RW + rr
-        if (lane < 16) {
-            const int jj = lane / GH_RW, rr = lane % GH_RW;
-            if (rr < nr && j0 + jj < jend) zp[(size_t)rr * dg + j0 + jj] = tot;
-        }
+#pragma unroll
+        for (int u = 0; u < GH_U; ++u) w[u] = wn[u];
     }
+    float* zp = zpart + (((size_t)lb * nchunk + chunk) * R + r0) * dg + j;
+#pragma unroll
+    for (int rr = 0; rr < GH_RW; ++rr)
+        if (rr < nr) *reinterpret_cast<float4*>(zp + (size_t)rr * dg) = make_float4(acc[0][rr], acc[1][rr], acc[2][rr], acc[3][rr]);
+}
+
+// W1T[d][j] = W1[j][d] for one layer (32 x 32 tiles through shared memory).  grid = (ceil(D / 32), ceil(dg / 32)).
+__global__ void __launch_bounds__(256)
+gate_transpose_kernel(const float* __restrict__ W1, float* __restrict__ W1T, int dg, int D) {
+    __shared__ float tile[32][33];
+    const int d0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int k = ty; k < 32; k += 8)
+        if (j0 + k < dg && d0 + tx < D) tile[k][tx] = W1[(size_t)(j0 + k) * D + d0 + tx];
+    __syncthreads();
+    for (int k = ty; k < 32; k += 8)
+        if (d0 + k < D && j0 + tx < dg) W1T[(size_t)(d0 + k) * dg + j0 + tx] = tile[tx][k];
 }
 
 constexpr int GO_RT = 8;  // rows per CTA of the output kernel
@@ -154,9 +139,16 @@ gate_out_kernel(const float* __restrict__ zpart, const float* __restrict__ b1, c
     const int nr = min(GO_RT, R - r0);
     for (int i = threadIdx.x * 4; i < nr * dg; i += blockDim.x * 4) {
         float4 z = __ldg(reinterpret_cast<const float4*>(b1 + (size_t)layer * dg + i % dg));
-        for (int ch = 0; ch < nchunk; ++ch) {           // fixed order: deterministic
-            const float4 p = *reinterpret_cast<const float4*>(zpart + (((size_t)lb * nchunk + ch) * R + r0) * dg + i);
-            z.x += p.x; z.y += p.y; z.z += p.z; z.w += p.w;
+        // the chunk partials are added in a fixed order (deterministic), their loads issued eight at a time
+        for (int ch0 = 0; ch0 < nchunk; ch0 += 8) {
+            float4 p[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                p[q] = (ch0 + q < nchunk)
+                           ? __ldcg(reinterpret_cast<const float4*>(zpart + (((size_t)lb * nchunk + ch0 + q) * R + r0) * dg + i))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { z.x += p[q].x; z.y += p[q].y; z.z += p[q].z; z.w += p[q].w; }
         }
         z.x = z.x / (1.0f + expf(-z.x)); z.y = z.y / (1.0f + expf(-z.y));
         z.z = z.z / (1.0f + expf(-z.z)); z.w = z.w / (1.0f + expf(-z.w));
@@ -211,6 +203,12 @@ void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, f
 
 int gate_chunks(int D) { return (D + GH_DC - 1) / GH_DC; }
 
+void launch_gate_transpose(const float* W1, float* W1T, int dg, int D, cudaStream_t st) {
+    dim3 grid((D + 31) / 32, (dg + 31) / 32);
+    gate_transpose_kernel<<<grid, 256, 0, st>>>(W1, W1T, dg, D);
+    count_launch();
+}
+
 void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, int layer0, int nlayers, int rows_per_layer,
                      float* beta, float* lam, float* c, cudaStream_t st) {
     dim3 g2((rows_per_layer + GO_RT - 1) / GO_RT, nlayers);
@@ -223,8 +221,8 @@ void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, i
 void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st) {
     const int nchunk = gate_chunks(gp.D);
-    dim3 g1(((rows_per_layer + GH_RW - 1) / GH_RW) * nchunk, GH_JSPLIT, nlayers);
-    gate_hidden_kernel<<<g1, GH_WARPS * 32, 0, st>>>(x, gp.W1, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
+    dim3 g1(((rows_per_layer + GH_RW - 1) / GH_RW) * nchunk, (gp.dg + 4 * GH_THREADS - 1) / (4 * GH_THREADS), nlayers);
+    gate_hidden_kernel<<<g1, GH_THREADS, 0, st>>>(x, gp.W1T, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
     count_launch();
     launch_gate_out(gp, z_scratch, nchunk, layer0, nlayers, rows_per_layer, beta, lam, c, st);
 }

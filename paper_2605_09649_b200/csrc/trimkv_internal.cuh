@@ -114,7 +114,7 @@ __device__ __forceinline__ void latch_error(int32_t* err, int code) {
 
 // ------------------------------------------------------------------ launchers (host)
 struct GateParams {
-    const float* W1;  // [L][dg][D]
+    const float* W1T; // [L][D][dg]  first layer, transposed (input dimension major)
     const float* b1;  // [L][dg]
     const float* W2;  // [L][H][de][dg]
     const float* b2;  // [L][H][de]
@@ -131,6 +131,9 @@ void launch_gate_fold(const GateParams& gp, int layer0, int nlayers, float* v, f
 // Number of input-dimension chunks the hidden layer is split into; the scratch of launch_gate holds
 // gate_chunks(D) * rows * dg floats per layer.
 int gate_chunks(int D);
+
+// W1T[d][j] = W1[j][d] for one layer's first-layer weights W1 [dg][D].
+void launch_gate_transpose(const float* W1, float* W1T, int dg, int D, cudaStream_t st);
 
 // rows_per_layer rows of x per layer, layers [layer0, layer0 + nlayers).
 void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,

@@ -93,7 +93,7 @@ struct trimkv {
     SelectBuffers sb;
     AttnBuffers ab;
     int32_t *hole, *mover, *cursor;
-    float *W1, *b1, *W2, *b2, *w_g, *gv, *gs0, *u, *g_lam, *g_c;
+    float *W1T, *b1, *W2, *b2, *w_g, *gv, *gs0, *u, *g_lam, *g_c;
     float* st_x = nullptr;                                   // staging of trimkv_decode_step_all_host: x or lambda
     char *st_k = nullptr, *st_v = nullptr, *st_q = nullptr, *st_out = nullptr;
     float *W1hi = nullptr, *W1lo = nullptr, *xhi = nullptr, *xlo = nullptr;   // 3xTF32 operands of the tensor-core gate
@@ -171,7 +171,7 @@ trimkv_status device_status(trimkv* h) {
 
 GateParams gate_params(const trimkv* h) {
     GateParams gp;
-    gp.W1 = h->W1; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.v = h->gv; gp.s0 = h->gs0; gp.b_g = h->b_g;
+    gp.W1T = h->W1T; gp.b1 = h->b1; gp.W2 = h->W2; gp.b2 = h->b2; gp.w_g = h->w_g; gp.v = h->gv; gp.s0 = h->gs0; gp.b_g = h->b_g;
     gp.D = h->D; gp.dg = h->dg; gp.de = h->de; gp.H = h->H; gp.horizon = h->cfg.horizon;
     return gp;
 }
@@ -315,7 +315,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     h->shared_set = false;
     h->b_g = 0.f;
     h->entries = 0;
-    h->W1 = h->b1 = h->W2 = h->b2 = h->w_g = h->gv = h->gs0 = h->u = h->g_lam = h->g_c = nullptr;
+    h->W1T = h->b1 = h->W2 = h->b2 = h->w_g = h->gv = h->gs0 = h->u = h->g_lam = h->g_c = nullptr;
 
     CacheView& cv = h->cv;
     memset(&cv, 0, sizeof(cv));
@@ -365,14 +365,13 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     A(dev_alloc(h, &h->st_q, (size_t)h->L * h->B * h->Hq * h->d * h->elt, false));
     A(dev_alloc(h, &h->st_out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, false));
     if (h->D > 0) {
-        A(dev_alloc(h, &h->W1, (size_t)h->L * h->dg * h->D, false));
+        A(dev_alloc(h, &h->W1T, (size_t)h->L * h->dg * h->D, false));
         A(dev_alloc(h, &h->b1, (size_t)h->L * h->dg, false));
         A(dev_alloc(h, &h->W2, (size_t)h->L * h->H * h->de * h->dg, false));
         A(dev_alloc(h, &h->b2, (size_t)h->L * h->H * h->de, false));
         A(dev_alloc(h, &h->w_g, (size_t)h->de, false));
         A(dev_alloc(h, &h->gv, (size_t)h->L * h->H * h->dg, false));
         A(dev_alloc(h, &h->gs0, (size_t)h->L * h->H, false));
-        A(dev_alloc(h, &h->u, (size_t)h->rows_max * h->dg * gate_chunks(h->D), false));
         if (s == TRIMKV_OK && gate_tc_supported(h->D, h->dg) && (long long)h->B * cfg->max_chunk >= TC_MIN_ROWS) {
             A(dev_alloc(h, &h->W1hi, (size_t)h->L * h->dg * h->D, true));
             A(dev_alloc(h, &h->W1lo, (size_t)h->L * h->dg * h->D, true));
@@ -380,6 +379,11 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
             A(dev_alloc(h, &h->xlo, (size_t)h->rows_max * h->D, true));
             if (s == TRIMKV_OK) h->tc = gate_tc_create(h->xhi, h->xlo, h->rows_max, h->W1hi, h->W1lo, h->L, h->dg, h->D);
         }
+        // scratch of the hidden layer: one slab per input-dimension chunk for the calls the streaming kernel takes (every
+        // call without the tensor-core form, else only those below its row threshold and the all-layer decode step)
+        const long long rows_stream = h->tc ? std::min<long long>(h->rows_max, std::max<long long>(TC_MIN_ROWS, (long long)h->L * h->B))
+                                            : h->rows_max;
+        A(dev_alloc(h, &h->u, (size_t)std::max<long long>(h->rows_max, rows_stream * gate_chunks(h->D)) * h->dg, false));
     }
     if (s == TRIMKV_OK) {
         int prio_lo = 0, prio_hi = 0;
@@ -431,12 +435,12 @@ trimkv_status trimkv_set_gate(trimkv_t* h, int layer, const float* W1, const flo
     if (h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
     if (layer < 0 || layer >= h->L || !W1 || !b1 || !W2 || !b2) return fail(TRIMKV_E_ARG, "bad layer or NULL weights");
     CUDA_TRY(cudaDeviceSynchronize());
-    CUDA_TRY(cudaMemcpy(h->W1 + (size_t)layer * h->dg * h->D, W1, (size_t)h->dg * h->D * 4, cudaMemcpyDeviceToDevice));
+    launch_gate_transpose(W1, h->W1T + (size_t)layer * h->dg * h->D, h->dg, h->D, 0);     // kept input-dimension major
     CUDA_TRY(cudaMemcpy(h->b1 + (size_t)layer * h->dg, b1, (size_t)h->dg * 4, cudaMemcpyDeviceToDevice));
     CUDA_TRY(cudaMemcpy(h->W2 + (size_t)layer * h->H * h->de * h->dg, W2, (size_t)h->H * h->de * h->dg * 4, cudaMemcpyDeviceToDevice));
     CUDA_TRY(cudaMemcpy(h->b2 + (size_t)layer * h->H * h->de, b2, (size_t)h->H * h->de * 4, cudaMemcpyDeviceToDevice));
     h->gate_set[layer] = 1;
-    if (h->tc) launch_split_tf32(h->W1 + (size_t)layer * h->dg * h->D, h->W1hi + (size_t)layer * h->dg * h->D,
+    if (h->tc) launch_split_tf32(W1, h->W1hi + (size_t)layer * h->dg * h->D,
                                  h->W1lo + (size_t)layer * h->dg * h->D, (long long)h->dg * h->D, 0);
     if (h->shared_set) launch_gate_fold(gate_params(h), layer, 1, h->gv, h->gs0, 0);
     CUDA_TRY(cudaDeviceSynchronize());
