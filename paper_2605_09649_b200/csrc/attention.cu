@@ -653,8 +653,8 @@ attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T*
 }  // namespace
 
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
-                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, const void* q,
-                      void* out, cudaStream_t st, PhaseMarker* pm) {
+                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, int reserve_sms,
+                      const void* q, void* out, cudaStream_t st, PhaseMarker* pm) {
     const int n_scope = nlayers * cv.B * cv.H;
     const int g = Hq / cv.H;
     const float scale = 1.0f / sqrtf((float)cv.d);
@@ -670,6 +670,10 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         int dev = 0, sms = 148;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        // The kernel is bound by HBM long before it needs every SM.  SMs left free take the one-CTA-per-sequence kernels of
+        // the selection (1024 threads each: they cannot share an SM with a resident attention CTA, whose registers leave
+        // room for 512 more threads at most) while the attention kernel is still running.
+        sms = std::max(sms - std::max(reserve_sms, 0), (sms * 3 + 3) / 4);
         const long long workers = (long long)sms * ATT_WARPS;
         // Items of about half a worker's share: most pools are then one item and need no merge, while a pool that
         // dominates the cache is still cut up.  (Few warps suffice to saturate HBM, so coarse items cost no bandwidth.)

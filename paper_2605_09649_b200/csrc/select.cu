@@ -614,7 +614,7 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: 
 // is simply not sampled, so every live slot has probability p.
 __global__ void __launch_bounds__(256)
 sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample, int sub, uint32_t thresh,
-              uint32_t seed) {
+              uint32_t seed, int skip_newest) {
     const int b = blockIdx.y;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int per_page = sub > 0 ? PAGE / sub : 1;
@@ -624,7 +624,11 @@ sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample
     if (inf.x < 0) return;
     SelState* st = sel + b;
     const CacheView& cv = src.cv;
+    // skip_newest > 0: the last skip_newest entries of every pool have no retention terms yet (their gate is still
+    // running); they are left out of the sample, which only has to be representative
+    const int live = skip_newest > 0 ? cv.len[(size_t)b * cv.L * cv.H + inf.x] - skip_newest : 0x7fffffff;
     auto take = [&](int off) {
+        if (inf.y * PAGE + off >= live) return;
         const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
         const int pos = cv.pos[s];
         const float S = retention_score(cv.lam[s], cv.c[s], (float)(src.t1 - (long long)pos));
@@ -1250,8 +1254,8 @@ void launch_select_state_init(SelState* sel, int B, cudaStream_t st) {
     count_launch();
 }
 
-void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
-                         long long k_evict, int32_t* compact_cursor, int distrust_sample, cudaStream_t st) {
+void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
+                                long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st) {
     CacheSrc src;
     src.cv = cv;
     src.t1 = t + 1;
@@ -1266,14 +1270,28 @@ void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long
     const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u;
     const long long threads = cv.P_seq * (sub > 0 ? PAGE / sub : 1);
     dim3 gs((unsigned)((threads + 255) / 256), cv.B);
-    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, sub, thresh, seed);
+    sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, sub, thresh, seed, skip_newest);
     bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample);
+    count_launch(2);
+}
+
+void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
+                              int32_t* compact_cursor, cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
     dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
     filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
     resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
                                                  sb.stats, compact_cursor, cv.err);
     redo_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, cv.evict_mask, cv.P_seq, k_evict, cv.err);
-    count_launch(5);
+    count_launch(3);
+}
+
+void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
+                         long long k_evict, int32_t* compact_cursor, int distrust_sample, cudaStream_t st) {
+    launch_select_cache_sample(cv, sb, t, n_total, k_evict, 0, distrust_sample, st);
+    launch_select_cache_rest(cv, sb, t, k_evict, compact_cursor, st);
 }
 
 void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st) {

@@ -168,6 +168,12 @@ struct SelectBuffers {
 // compact_cursor [B]: zeroed by the selection for the compaction that follows.
 void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, long long k_evict,
                          int32_t* compact_cursor, int distrust_sample, cudaStream_t st);
+// The same selection in two parts, for callers that run the sampling beside other work: the sample and its rank bracket
+// (skip_newest: entries at the tail of every pool whose retention terms are not written yet), then filter and resolution.
+void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
+                                long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st);
+void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
+                              int32_t* compact_cursor, cudaStream_t st);
 // Fixed per-pool budget: every pool keeps its keep_per_pool best entries (masks as for launch_select_cache).
 void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st);
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max, cudaStream_t st);
@@ -193,10 +199,11 @@ struct PhaseMarker {
     virtual ~PhaseMarker() {}
 };
 
+// reserve_sms: SMs the persistent kernel leaves to kernels running beside it (0 when it runs alone).
 // retention_bias != 0: retention-gated weights beta_i^(t_now - i) e^{z_i} instead of the plain softmax.
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
-                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, const void* q,
-                      void* out, cudaStream_t st, PhaseMarker* pm);
+                      long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, int reserve_sms,
+                      const void* q, void* out, cudaStream_t st, PhaseMarker* pm);
 
 // Causal attention of the chunk of n_new tokens just appended to `layer`; q, out: [B, n_new, Hq, d].
 // tc: state of the tensor-core (tcgen05) form, or null; used when the chunk is large enough to fill its tiles.

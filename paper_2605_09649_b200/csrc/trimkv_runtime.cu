@@ -108,9 +108,10 @@ struct trimkv {
     std::vector<void*> allocs;
     // decode_step_all runs on two streams of its own: `fast` (highest priority) carries K/V append, attention and
     // compaction; `side` (lowest priority) carries the gate and the selection beside the attention kernels
-    cudaStream_t fast = nullptr, side = nullptr;
+    cudaStream_t fast = nullptr, side = nullptr, side2 = nullptr;   // side2: the selection's sampling, beside the gate
+    cudaStream_t side_hi = nullptr;                                 // `side` at the priority of `fast` (gate-heavy steps)
     bool overlap = true;
-    cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr, ev_sample = nullptr;
 };
 
 namespace {
@@ -236,11 +237,11 @@ trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
     return compact_impl(h, st);
 }
 
-trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, void* out, cudaStream_t st) {
+trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, void* out, cudaStream_t st, int reserve_sms = 0) {
     const long long tiles = (h->entries * h->B / 32) * nlayers / h->L + (long long)nlayers * h->B * h->H;
     const long long tiles_upper = h->entries * h->B / 32 + (long long)nlayers * h->B * h->H;
     launch_attention(h->cv, h->ab, layer0, nlayers, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, tiles, tiles_upper,
-                     h->cfg.retention_bias, h->tokens[layer0], q, out, st, h->prof.on ? &h->prof : nullptr);
+                     h->cfg.retention_bias, h->tokens[layer0], reserve_sms, q, out, st, h->prof.on ? &h->prof : nullptr);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
 }
@@ -390,6 +391,9 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);     // numerically lower = higher priority
         if (cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_lo) != cudaSuccess ||
             cudaStreamCreateWithPriority(&h->fast, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+            cudaStreamCreateWithPriority(&h->side2, cudaStreamNonBlocking, prio_lo) != cudaSuccess ||
+            cudaStreamCreateWithPriority(&h->side_hi, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h->ev_sample, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&h->ev_done, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&h->ev_append, cudaEventDisableTiming) != cudaSuccess ||
@@ -416,6 +420,9 @@ void trimkv_destroy(trimkv_t* h) {
     if (h->ev_append) cudaEventDestroy(h->ev_append);
     if (h->ev_side) cudaEventDestroy(h->ev_side);
     if (h->ev_done) cudaEventDestroy(h->ev_done);
+    if (h->ev_sample) cudaEventDestroy(h->ev_sample);
+    if (h->side2) cudaStreamDestroy(h->side2);
+    if (h->side_hi) cudaStreamDestroy(h->side_hi);
     if (h->side) cudaStreamDestroy(h->side);
     if (h->fast) cudaStreamDestroy(h->fast);
     for (void* p : h->allocs) cudaFree(p);
@@ -555,7 +562,14 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     // moves K/V rows and therefore waits for both.  `fast` has the higher priority so that its few, large CTAs are
     // placed ahead of the many small ones of the side kernels.
     const bool two = h->overlap;                 // off: every phase back to back on the caller's stream
-    cudaStream_t sd = two ? h->side : st, fs = two ? h->fast : st;
+    // The side chain runs below the attention kernel's priority, unless the gate's weight stream is a sizeable part of
+    // the step's traffic (above 15 % of the K/V bytes): a starved gate then ends together with the attention kernel and
+    // the whole selection would follow it; at equal priority the gate finishes early and the selection hides under the
+    // rest of the attention kernel (measured: config 5 0.499 -> 0.480 ms, config 3 0.169 -> 0.155; config 2, where the
+    // gate is 7 % of the traffic, loses 9 us that way and keeps the low priority).
+    const double kv_bytes = (double)(h->entries + (long long)h->L * h->H) * h->B * 2.0 * h->cv.row_bytes;
+    const bool gate_heavy = x && (double)h->L * h->D * h->dg * 4.0 > 0.15 * kv_bytes;
+    cudaStream_t sd = two ? (gate_heavy ? h->side_hi : h->side) : st, fs = two ? h->fast : st;
     if (two) {
         CUDA_TRY(cudaEventRecord(h->ev_fork, st));
         CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
@@ -576,7 +590,15 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     for (int l = 0; l < h->L; ++l) h->tokens[l] += 1;
     h->entries += (long long)h->L * h->H;
     const long long kev = eviction_due(h);
-    trimkv_status s = attention_impl(h, 0, h->L, q, out, fs);
+    // Scheduling policy of the overlapped step.  When the K/V stream of the step is short (under ~1 GB, ~150 us), the
+    // side chain (gate -> selection) is the critical path: the attention kernel then leaves one SM per sequence to the
+    // selection's single-CTA kernels and the sampling runs early on a third stream.  With a long attention kernel the
+    // side chain has slack: two SMs are enough for its single-CTA kernels to finish before the attention kernel does
+    // (they cannot share an SM with a resident attention CTA and would otherwise run after it), and the third stream
+    // is not used (measured: it costs the host-buffer entry point 30 us per step there).
+    const bool side_critical = (double)h->entries * h->B * 2.0 * h->cv.row_bytes < 1.0e9;
+    const int reserve = (two && kev > 0) ? std::min(h->B, side_critical ? 8 : 2) : 0;
+    trimkv_status s = attention_impl(h, 0, h->L, q, out, fs, reserve);
 
     const float* lam = lambda;
     const float* cc = nullptr;
@@ -587,9 +609,24 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
         lam = h->g_lam;
         cc = h->g_c;
     }
+    // The selection's sample and rank bracket need only the page records of this step (final once the K/V half of the
+    // append has run), not the new entries' retention terms: they run on a third stream beside the gate.
+    const bool early_sample = two && kev > 0 && h->cfg.per_pool_budget == 0 && side_critical;
+    if (early_sample) {
+        CUDA_TRY(cudaStreamWaitEvent(h->side2, h->ev_append, 0));
+        launch_select_cache_sample(h->cv, h->sb, h->tokens[0], h->entries, kev, 1, h->cfg.reserved & 1, h->side2);
+        CUDA_TRY(cudaEventRecord(h->ev_sample, h->side2));
+    }
     if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
     launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, APPEND_META, sd);
-    if (kev > 0) select_impl(h, kev, sd);
+    if (early_sample) {
+        CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_sample, 0));
+        if (h->prof.on) h->prof.mark(PH_SELECT, 0, sd);
+        launch_select_cache_rest(h->cv, h->sb, h->tokens[0], kev, h->cursor, sd);
+        if (h->prof.on) h->prof.mark(PH_SELECT, 1, sd);
+    } else if (kev > 0) {
+        select_impl(h, kev, sd);
+    }
     if (two) {
         CUDA_TRY(cudaEventRecord(h->ev_side, sd));
         CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
