@@ -124,7 +124,7 @@ gate_transpose_kernel(const float* __restrict__ W1, float* __restrict__ W1T, int
         if (d0 + k < D && j0 + tx < dg) W1T[(size_t)(d0 + k) * dg + j0 + tx] = tile[tx][k];
 }
 
-constexpr int GO_RT = 8;  // rows per CTA of the output kernel
+constexpr int GO_RT = 2;  // rows per CTA of the output kernel (few: at decode the kernel is a chain of dependent loads per thread)
 
 // s[lb][r][h] = v[layer][h] . u[lb][r] + s0[layer][h]; then beta / lambda / c.   grid = (row tiles, layers).
 __global__ void __launch_bounds__(256)
