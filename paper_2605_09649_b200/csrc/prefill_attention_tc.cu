@@ -9,8 +9,9 @@
 // operands of S = Q K^T, V halves as MN-major operands of O += P V.  Roles: warps 0-3 / 4-7 are the softmax warps of
 // group 0 / 1 (a thread owns one row: S read from tensor memory, masked, exponentiated, P written back to tensor memory as
 // bf16 pairs, where the P V product reads it as its A operand), warp 8 issues the TMA copies into a 4-stage ring, warps 9
-// and 10 each issue the MMAs of one group (S of tile i + 1 before P V of tile i, so the tensor pipe works while the
-// softmax warps compute, and neither group's issuer ever waits for the other group).  O accumulates in tensor memory; the
+// and 10 each issue the MMAs of one group (S is double-buffered in tensor memory and issued two tiles ahead of the P V that
+// needs the softmax result, so the tensor pipe works while the softmax warps compute, and neither group's issuer ever
+// waits for the other group; P overwrites the first half of its tile's S).  O accumulates in tensor memory; the
 // running maximum is only raised (and O rescaled) when it grows by more than 2^8, which keeps every exponential finite and
 // leaves the final O / l unchanged.  A third of the exponentials are evaluated with FMAs instead of the special-function
 // unit.  Every wait is bounded; a wait that runs out latches TRIMKV_E_TIMEOUT.
@@ -34,8 +35,9 @@ constexpr int A_OFF_BAR = A_OFF_Q + A_Q_BYTES;
 constexpr int A_SMEM = A_OFF_BAR + 256 + 1024;        // barriers and flags, alignment slack
 constexpr int A_THREADS = 352;                       // 8 softmax warps, the TMA warp, one MMA-issuing warp per group
 constexpr unsigned A_WAIT_LIMIT = 1u << 22;
-constexpr int A_TMEM_COLS = 512;                      // S of group 0, 1: columns 0-63, 64-127; O: 128-255, 256-383;
-constexpr int A_COL_P = 384;                          // P (bf16 pairs, the A operand of P V): 384-415, 416-447
+constexpr int A_TMEM_COLS = 512;                      // group g: S of even / odd tiles at columns 128 g, 128 g + 64; O at 256 + 128 g.
+                                                      // P of a tile (bf16 pairs, the A operand of P V) overwrites the first 32
+                                                      // columns of that tile's S once the softmax threads hold S in registers
 constexpr int A_POLY_EVERY = 3;                       // share of the exponentials computed with FMAs: 1 / A_POLY_EVERY
 constexpr float A_RESCALE_STEP = 8.0f;                // log2 units the running maximum may lag behind
 
@@ -192,7 +194,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
     const uint32_t base = (raw + 1023u) & ~1023u;                        // operand tiles need 1024-byte alignment
     unsigned char* gen = a_smem_raw + (base - raw);
     const uint32_t bars = base + A_OFF_BAR;
-    const uint32_t full0 = bars, empty0 = bars + 32, s_ready0 = bars + 64, s_free0 = bars + 80, p_ready0 = bars + 96,
+    const uint32_t full0 = bars, empty0 = bars + 32, s_ready0 = bars + 64 /* [group][tile parity] */, p_ready0 = bars + 96,
                    pv_done0 = bars + 112;
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen + A_OFF_BAR + 128);
     volatile int* s_fail = reinterpret_cast<volatile int*>(gen + A_OFF_BAR + 136);
@@ -211,8 +213,8 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
     if (threadIdx.x == 0) {
         for (int s = 0; s < A_STAGES; ++s) { a_bar_init(full0 + 8 * s, 1); a_bar_init(empty0 + 8 * s, 2); }   // both issuers free a stage
         for (int gq = 0; gq < 2; ++gq) {
-            a_bar_init(s_ready0 + 8 * gq, 1);
-            a_bar_init(s_free0 + 8 * gq, 4);
+            a_bar_init(s_ready0 + 16 * gq, 1);
+            a_bar_init(s_ready0 + 16 * gq + 8, 1);
             a_bar_init(p_ready0 + 8 * gq, 4);
             a_bar_init(pv_done0 + 8 * gq, 1);
         }
@@ -274,13 +276,30 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
         }
     } else if (warp >= 9) {
         if (lane == 0) {
-            // ---- MMA issuer of group gq: S of tile i, then P V of tile i - 1; the two issuers never wait for each other
+            // ---- MMA issuer of group gq.  S has two buffers, so S of tiles i + 1 and i + 2 are issued before P V of tile
+            // i needs its P: the softmax threads never wait for S, and the tensor pipe has the other group's and the
+            // next tiles' products to run while a group computes its exponentials.  S of tile i + 2 overwrites the buffer
+            // that held S and P of tile i; it is issued after P V of tile i, and the pipe runs in issue order.
             const int gq = warp - 9;
             bool ok = true;
-            const uint32_t d_s = tmem + gq * 64, d_o = tmem + 128 + gq * 128, a_p = tmem + A_COL_P + gq * 32;
+            const uint32_t d_s0 = tmem + 128 * gq, d_o = tmem + 256 + 128 * gq;
             const uint64_t qdesc0 = a_desc(base + A_OFF_Q + (gq * 2) * A_QPLANE, 16), qdesc1 = a_desc(base + A_OFF_Q + (gq * 2 + 1) * A_QPLANE, 16);
+            auto issue_s = [&](int t) {                                  // S = Q K^T of tile t into buffer t & 1
+                const int s = t % A_STAGES;
+                if (!a_bar_wait(full0 + 8 * s, (t / A_STAGES) & 1)) { ok = false; return; }
+                a_fence_after();
+                const uint32_t st = base + s * A_STAGE_BYTES, d_s = d_s0 + 64 * (t & 1);
+                const uint64_t kdesc0 = a_desc(st, 16), kdesc1 = a_desc(st + A_PLANE, 16);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)                              // 16 of d per instruction, 32 bytes along the row
+                    a_umma(d_s, qdesc0 + (uint64_t)(j * 32 >> 4), kdesc0 + (uint64_t)(j * 32 >> 4), A_IDESC_S, j != 0);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    a_umma(d_s, qdesc1 + (uint64_t)(j * 32 >> 4), kdesc1 + (uint64_t)(j * 32 >> 4), A_IDESC_S, 1u);
+                a_commit(s_ready0 + 16 * gq + 8 * (t & 1));
+            };
             auto issue_pv = [&](int t) {                                 // O += P V of tile t
-                const uint32_t st = base + (t % A_STAGES) * A_STAGE_BYTES;
+                const uint32_t st = base + (t % A_STAGES) * A_STAGE_BYTES, a_p = d_s0 + 64 * (t & 1);
                 if (!a_bar_wait(p_ready0 + 8 * gq, t & 1)) { ok = false; return; }
                 a_fence_after();
                 const uint64_t vdesc = a_desc(st + 2 * A_PLANE, A_PLANE);         // the second 64 dims: one plane further
@@ -290,42 +309,29 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                 a_commit(pv_done0 + 8 * gq);
                 a_commit(empty0 + 8 * (t % A_STAGES));                   // this group is done with the stage
             };
+            issue_s(0);
+            if (ok && ntile > 1) issue_s(1);
             for (int i = 0; i < ntile && ok; ++i) {
-                const int s = i % A_STAGES;
-                if (!a_bar_wait(full0 + 8 * s, (i / A_STAGES) & 1)) { ok = false; break; }
-                if (i > 0 && !a_bar_wait(s_free0 + 8 * gq, (i - 1) & 1)) { ok = false; break; }
-                a_fence_after();
-                const uint32_t st = base + s * A_STAGE_BYTES;
-                const uint64_t kdesc0 = a_desc(st, 16), kdesc1 = a_desc(st + A_PLANE, 16);
-#pragma unroll
-                for (int j = 0; j < 4; ++j)                              // S = Q K^T: 16 of d per instruction, 32 bytes along the row
-                    a_umma(d_s, qdesc0 + (uint64_t)(j * 32 >> 4), kdesc0 + (uint64_t)(j * 32 >> 4), A_IDESC_S, j != 0);
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    a_umma(d_s, qdesc1 + (uint64_t)(j * 32 >> 4), kdesc1 + (uint64_t)(j * 32 >> 4), A_IDESC_S, 1u);
-                a_commit(s_ready0 + 8 * gq);
-                if (i > 0) issue_pv(i - 1);
+                issue_pv(i);
+                if (ok && i + 2 < ntile) issue_s(i + 2);
             }
-            if (ok) issue_pv(ntile - 1);
             if (!ok) *s_fail = 1;
         }
     } else {
         // ---- softmax warps
         const uint32_t lane_addr = tmem + ((uint32_t)(wl * 32) << 16);
-        const uint32_t s_col = (uint32_t)(grp * 64), o_col = (uint32_t)(128 + grp * 128);
+        const uint32_t s_col0 = (uint32_t)(128 * grp), o_col = (uint32_t)(256 + 128 * grp);
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < ntile; ++i) {
-            ok = __all_sync(0xffffffffu, a_bar_wait(s_ready0 + 8 * grp, i & 1));
+            ok = __all_sync(0xffffffffu, a_bar_wait(s_ready0 + 16 * grp + 8 * (i & 1), (i >> 1) & 1));
+            const uint32_t s_col = s_col0 + 64u * (uint32_t)(i & 1);
             if (!ok) break;
             a_fence_after();
             uint32_t sv[64];
             a_tmem_ld32(lane_addr + s_col, sv);
             a_tmem_ld32(lane_addr + s_col + 32, sv + 32);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            a_fence_before();
-            __syncwarp();
-            if (lane == 0) a_bar_arrive(s_free0 + 8 * grp);              // S may be overwritten by the next tile's product
             const int e0 = i * A_TILE;
             if (e0 + A_TILE > limit) {                                   // the tile crosses this row's causal limit
 #pragma unroll
@@ -374,7 +380,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                 sum = a0 + a1;
             }
             l = l * alpha + sum;
-            if (i > 0) {                                                 // P V of the previous tile: O complete, P buffer free
+            if (i > 0) {                                                 // P V of the previous tile: O complete (each phase is awaited once, in order)
                 ok = __all_sync(0xffffffffu, a_bar_wait(pv_done0 + 8 * grp, (i - 1) & 1));
                 if (!ok) break;
                 a_fence_after();
@@ -391,7 +397,7 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, CacheView cv,
                     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 }
             }
-            a_tmem_st32(lane_addr + A_COL_P + grp * 32, pk);             // P: the A operand of P V, two bf16 per column
+            a_tmem_st32(lane_addr + s_col, pk);                          // P over the first half of this tile's S: the A operand of P V
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             a_fence_before();
             __syncwarp();
