@@ -57,7 +57,7 @@ gate_fold_kernel(const float* __restrict__ W2, const float* __restrict__ b2, con
 // thread owns four consecutive hidden units, so a warp's weight load is 512 contiguous bytes, the x values of a dimension
 // are one broadcast read of shared memory for the whole warp, and every thread finishes its own sums (no shuffles).
 // GH_U dimensions are in flight per thread.  grid = (row tiles * chunks, ceil(dg / 512), layers).
-__global__ void __launch_bounds__(GH_THREADS)
+__global__ void __launch_bounds__(GH_THREADS, 4)
 gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1T, float* __restrict__ zpart, int layer0,
                    int R, int D, int dg, int nchunk) {
     __shared__ __align__(16) float xs[GH_DC][GH_RW];
