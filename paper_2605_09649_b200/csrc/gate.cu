@@ -17,7 +17,6 @@ namespace {
 
 constexpr int GH_THREADS = 128;  // threads per CTA of the hidden-layer kernel; a thread owns 4 consecutive hidden units
 constexpr int GH_DC = 128;       // input dimensions per CTA (its x tile lives in shared memory)
-constexpr int GH_RW = 8;         // rows per CTA
 constexpr int GH_U = 8;          // input dimensions (16-byte weight loads per lane) in flight
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -52,63 +51,114 @@ gate_fold_kernel(const float* __restrict__ W2, const float* __restrict__ b2, con
     }
 }
 
+// Two fp32 multiply-adds per instruction (each lane rounded as a scalar fmaf would).
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+// JT consecutive floats of read-once data.
+template <int JT>
+__device__ __forceinline__ void ld_stream_n(const float* p, float (&dst)[JT]) {
+    if constexpr (JT == 4) {
+        const float4 v = ld_stream(p);
+        dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    } else if constexpr (JT == 2) {
+        asm volatile("ld.global.nc.L1::no_allocate.v2.f32 {%0,%1}, [%2];" : "=f"(dst[0]), "=f"(dst[1]) : "l"(p));
+    } else {
+        asm volatile("ld.global.nc.L1::no_allocate.f32 %0, [%1];" : "=f"(dst[0]) : "l"(p));
+    }
+}
+
 // Partial pre-activations: zpart[lb][chunk][r][j] = sum over the chunk's input dimensions d of x[lb][r][d] W1[layer][j][d],
-// for GH_RW rows and one GH_DC-wide chunk of the input dimension per CTA.  W1 is kept transposed (W1T[layer][d][j]): a
-// thread owns four consecutive hidden units, so a warp's weight load is 512 contiguous bytes, the x values of a dimension
-// are one broadcast read of shared memory for the whole warp, and every thread finishes its own sums (no shuffles).
-// GH_U dimensions are in flight per thread.  grid = (row tiles * chunks, ceil(dg / 512), layers).
+// for RW rows and one GH_DC-wide chunk of the input dimension per CTA.  W1 is kept transposed (W1T[layer][d][j]): a
+// thread owns JT consecutive hidden units, so a warp's weight load is contiguous, the x values of a dimension are
+// broadcast reads of shared memory for the whole warp, and every thread finishes its own JT * RW = 32 sums (no
+// shuffles; the multiply-adds are packed fp32x2 over pairs of rows).  RW = 8 with JT = 4 serves up to 8 rows; larger
+// batches use RW = 16, JT = 2, which halves the number of times the weights are streamed (RW = 32, JT = 1 was slower: its
+// 4-byte weight loads quadruple the load instructions; measured at 32 rows: 0.254 against 0.164 ms).  U dimensions are in
+// flight per thread, and the next U are requested before the current ones are used.
+// grid = (row tiles * chunks, ceil(dg / (JT * GH_THREADS)), layers).
+template <int RW, int JT>
 __global__ void __launch_bounds__(GH_THREADS, 4)
 gate_hidden_kernel(const float* __restrict__ x, const float* __restrict__ W1T, float* __restrict__ zpart, int layer0,
                    int R, int D, int dg, int nchunk) {
-    __shared__ __align__(16) float xs[GH_DC][GH_RW];
+    constexpr int U = JT == 4 ? GH_U : 2 * GH_U;
+    __shared__ __align__(16) float xs[GH_DC][RW];
     const int lb = blockIdx.z;
     const int layer = layer0 + lb;
     const int chunk = blockIdx.x % nchunk;
-    const int r0 = (blockIdx.x / nchunk) * GH_RW;
-    const int nr = min(GH_RW, R - r0);
+    const int r0 = (blockIdx.x / nchunk) * RW;
+    const int nr = min(RW, R - r0);
     const int dbase = chunk * GH_DC;
     const int dn = min(GH_DC, D - dbase);
-    for (int i = threadIdx.x; i < GH_DC * GH_RW; i += blockDim.x) {
+    for (int i = threadIdx.x; i < GH_DC * RW; i += blockDim.x) {
         const int rr = i / GH_DC, dd = i % GH_DC;
         xs[dd][rr] = (rr < nr && dd < dn) ? __ldg(x + ((size_t)lb * R + r0 + rr) * D + dbase + dd) : 0.f;
     }
     __syncthreads();
-    const int j = (blockIdx.y * GH_THREADS + threadIdx.x) * 4;
+    const int j = (blockIdx.y * GH_THREADS + threadIdx.x) * JT;
     if (j >= dg) return;
     const float* Wp = W1T + ((size_t)layer * D + dbase) * dg + j;
-    float acc[4][GH_RW];
+    unsigned long long acc[JT][RW / 2];                                  // pairs of rows: packed fp32x2 multiply-adds
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
+    for (int q = 0; q < JT; ++q)
 #pragma unroll
-        for (int rr = 0; rr < GH_RW; ++rr) acc[q][rr] = 0.f;
-    // the weights of the next GH_U dimensions are requested before those of the current ones are used
-    float4 w[GH_U], wn[GH_U];
-    auto fetch = [&](float4 (&dst)[GH_U], int d0) {
+        for (int rr = 0; rr < RW / 2; ++rr) acc[q][rr] = 0ull;
+    float w[U][JT], wn[U][JT];
+    auto fetch = [&](float (&dst)[U][JT], int d0) {
 #pragma unroll
-        for (int u = 0; u < GH_U; ++u)
-            dst[u] = (d0 + u < dn) ? ld_stream(Wp + (size_t)(d0 + u) * dg) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int u = 0; u < U; ++u) {
+            if (d0 + u < dn) {
+                ld_stream_n<JT>(Wp + (size_t)(d0 + u) * dg, dst[u]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < JT; ++q) dst[u][q] = 0.f;
+            }
+        }
     };
     fetch(w, 0);
-    for (int d0 = 0; d0 < dn; d0 += GH_U) {
-        fetch(wn, d0 + GH_U);
+    for (int d0 = 0; d0 < dn; d0 += U) {
+        fetch(wn, d0 + U);
 #pragma unroll
-        for (int u = 0; u < GH_U; ++u) {
-            const float4 xa = *reinterpret_cast<const float4*>(&xs[d0 + u][0]);   // rows 0-3 (zero beyond dn)
-            const float4 xb = *reinterpret_cast<const float4*>(&xs[d0 + u][4]);   // rows 4-7
-            const float xr[GH_RW] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-            const float wq[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+        for (int u = 0; u < U; ++u) {
+            if (d0 + u < GH_DC) {                                        // (rows of xs beyond dn hold zeros)
+                unsigned long long w2[JT];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
+                for (int q = 0; q < JT; ++q) w2[q] = pack_f32x2(w[u][q], w[u][q]);
 #pragma unroll
-                for (int rr = 0; rr < GH_RW; ++rr) acc[q][rr] = fmaf(xr[rr], wq[q], acc[q][rr]);
+                for (int r4 = 0; r4 < RW / 4; ++r4) {
+                    const ulonglong2 xv = *reinterpret_cast<const ulonglong2*>(&xs[d0 + u][4 * r4]);   // rows 4 r4 .. 4 r4 + 3
+#pragma unroll
+                    for (int q = 0; q < JT; ++q) {
+                        acc[q][2 * r4] = fma_f32x2(xv.x, w2[q], acc[q][2 * r4]);
+                        acc[q][2 * r4 + 1] = fma_f32x2(xv.y, w2[q], acc[q][2 * r4 + 1]);
+                    }
+                }
+            }
         }
 #pragma unroll
-        for (int u = 0; u < GH_U; ++u) w[u] = wn[u];
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int q = 0; q < JT; ++q) w[u][q] = wn[u][q];
     }
     float* zp = zpart + (((size_t)lb * nchunk + chunk) * R + r0) * dg + j;
 #pragma unroll
-    for (int rr = 0; rr < GH_RW; ++rr)
-        if (rr < nr) *reinterpret_cast<float4*>(zp + (size_t)rr * dg) = make_float4(acc[0][rr], acc[1][rr], acc[2][rr], acc[3][rr]);
+    for (int rp = 0; rp < RW / 2; ++rp) {
+#pragma unroll
+        for (int q = 0; q < JT; ++q) {
+            float lo, hi;
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(acc[q][rp]));
+            if (2 * rp < nr) zp[(size_t)(2 * rp) * dg + q] = lo;
+            if (2 * rp + 1 < nr) zp[(size_t)(2 * rp + 1) * dg + q] = hi;
+        }
+    }
 }
 
 // W1T[d][j] = W1[j][d] for one layer (32 x 32 tiles through shared memory).  grid = (ceil(D / 32), ceil(dg / 32)).
@@ -221,8 +271,12 @@ void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, i
 void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
                  float* beta, float* lam, float* c, cudaStream_t st) {
     const int nchunk = gate_chunks(gp.D);
-    dim3 g1(((rows_per_layer + GH_RW - 1) / GH_RW) * nchunk, (gp.dg + 4 * GH_THREADS - 1) / (4 * GH_THREADS), nlayers);
-    gate_hidden_kernel<<<g1, GH_THREADS, 0, st>>>(x, gp.W1T, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
+    auto run = [&](auto kernel, int rw, int jt) {
+        dim3 g1(((rows_per_layer + rw - 1) / rw) * nchunk, (gp.dg + jt * GH_THREADS - 1) / (jt * GH_THREADS), nlayers);
+        kernel<<<g1, GH_THREADS, 0, st>>>(x, gp.W1T, z_scratch, layer0, rows_per_layer, gp.D, gp.dg, nchunk);
+    };
+    if (rows_per_layer <= 8) run(gate_hidden_kernel<8, 4>, 8, 4);
+    else run(gate_hidden_kernel<16, 2>, 16, 2);                 // row tiles of 16
     count_launch();
     launch_gate_out(gp, z_scratch, nchunk, layer0, nlayers, rows_per_layer, beta, lam, c, st);
 }
