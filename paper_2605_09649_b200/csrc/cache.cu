@@ -75,7 +75,7 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
     // rows: [lb][b][j][h][d]
     const int rc = cv.row_bytes / 16;                  // 16-byte chunks per row
     const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
-    const int total = n_new * rc * 2;
+    const int total = (mode & APPEND_ROWS_ELSEWHERE) ? 0 : n_new * rc * 2;   // (a chunk's rows are copied by append_rows_kernel)
     for (int w = threadIdx.x; w < total; w += blockDim.x) {
         const int ci = w % rc;
         const int part = (w / rc) & 1;
@@ -107,6 +107,37 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
         cv.owner[(size_t)b * cv.P_seq + bt[lp]] = make_int4(pool_local, lp, min(PAGE, n2 - lp * PAGE), 0);
     __syncthreads();
     if (threadIdx.x == 0) cv.len[pool] = n2;
+}
+
+// K/V rows of a chunk: the copy half of an append whose bookkeeping (pages, length) append_kernel has done.
+// grid = (pools of the call, blocks of APPEND_TOK tokens): a chunk's copy is spread over the whole GPU instead of one CTA
+// per pool.
+constexpr int APPEND_TOK = 32;
+__global__ void __launch_bounds__(256)
+append_rows_kernel(CacheView cv, int layer0, int n_new, const char* __restrict__ k_in, const char* __restrict__ v_in) {
+    const int h = blockIdx.x % cv.H;
+    const int b = (blockIdx.x / cv.H) % cv.B;
+    const int lb = blockIdx.x / (cv.H * cv.B);
+    const int pool_local = (layer0 + lb) * cv.H + h;
+    const long long pool = (long long)b * cv.L * cv.H + pool_local;
+    const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    const int old = cv.len[pool] - n_new;
+    if (old < 0) return;                               // the bookkeeping half failed (its error is latched)
+    const int rc = cv.row_bytes / 16;
+    const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
+    const int j0 = blockIdx.y * APPEND_TOK;
+    const int total = min(APPEND_TOK, n_new - j0) * rc * 2;
+    for (int w = threadIdx.x; w < total; w += blockDim.x) {
+        const int ci = w % rc;
+        const int part = (w / rc) & 1;
+        const int j = j0 + w / (2 * rc);
+        const int idx = old + j;
+        const int page = bt[idx / PAGE];
+        const int off = idx % PAGE;
+        const char* src = (part ? v_in : k_in) + (in_row0 + (size_t)j * cv.H) * cv.row_bytes + (size_t)ci * 16;
+        char* dst = cv.kv + kv_row_offset(cv, b, page, part, off) + (size_t)phys_chunk(cv, ci, off) * 16;
+        *reinterpret_cast<uint4*>(dst) = __ldg(reinterpret_cast<const uint4*>(src));
+    }
 }
 
 __device__ __forceinline__ u64 bits_below(int n) {   // mask with the lowest n bits set, n in [0, 64]
@@ -294,8 +325,15 @@ rehorizon_kernel(CacheView cv, int horizon) {
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st) {
     const int grid = nlayers * cv.B * cv.H;
-    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v, mode);
+    const bool split = (mode & APPEND_KV) && n_new >= 4 * APPEND_TOK;     // a chunk: copy its rows with a grid of their own
+    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v,
+                                        split ? (mode | APPEND_ROWS_ELSEWHERE) : mode);
     count_launch();
+    if (split) {
+        dim3 g2(grid, (n_new + APPEND_TOK - 1) / APPEND_TOK);
+        append_rows_kernel<<<g2, 256, 0, st>>>(cv, layer0, n_new, (const char*)k, (const char*)v);
+        count_launch();
+    }
 }
 
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max,

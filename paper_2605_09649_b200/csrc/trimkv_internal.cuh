@@ -140,6 +140,7 @@ void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int lay
                  float* beta, float* lam, float* c, cudaStream_t st);
 
 constexpr int APPEND_KV = 1, APPEND_META = 2;   // halves of an append; see append_kernel
+constexpr int APPEND_ROWS_ELSEWHERE = 4;        // (internal to launch_append: the K/V rows are copied by a second kernel)
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st);
 
