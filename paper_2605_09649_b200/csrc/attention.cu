@@ -681,8 +681,8 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         long long tpi = tiles_estimate / (workers * 2);
         // With at least half as many pools as workers and short pools (up to 4096 entries on average), whole pools are the
         // better items even when they are shorter than that: nothing is merged (the per-item fence weighs most on short
-        // items), and the warps that get no item are not missed (HBM is saturated by a third of them).  Measured: config 3
-        // 99 -> 94 us; longer pools (config 5: 8192 entries) do better cut in three.
+        // items), and the warps that get no item are not missed (HBM is saturated by a third of them).  Measured: workload
+        // qwen_vl_16k 99 -> 94 us; longer pools (stress_128k: 8192 entries) do better cut in three.
         if ((long long)n_scope * 2 >= workers) {
             const long long avg = tiles_estimate / n_scope;
             if (avg <= 128) tpi = std::max(tpi, avg + avg / 4 + 1);

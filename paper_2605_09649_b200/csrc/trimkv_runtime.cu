@@ -565,8 +565,8 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     // The side chain runs below the attention kernel's priority, unless the gate's weight stream is a sizeable part of
     // the step's traffic (above 15 % of the K/V bytes): a starved gate then ends together with the attention kernel and
     // the whole selection would follow it; at equal priority the gate finishes early and the selection hides under the
-    // rest of the attention kernel (measured: config 5 0.499 -> 0.480 ms, config 3 0.169 -> 0.155; config 2, where the
-    // gate is 7 % of the traffic, loses 9 us that way and keeps the low priority).
+    // rest of the attention kernel (measured on the named workloads: stress_128k 0.499 -> 0.480 ms per step, qwen_vl_16k
+    // 0.169 -> 0.155; llama8b_32k, where the gate is 7 % of the traffic, loses 9 us that way and keeps the low priority).
     const double kv_bytes = (double)(h->entries + (long long)h->L * h->H) * h->B * 2.0 * h->cv.row_bytes;
     const bool gate_heavy = x && (double)h->L * h->D * h->dg * 4.0 > 0.15 * kv_bytes;
     cudaStream_t sd = two ? (gate_heavy ? h->side_hi : h->side) : st, fs = two ? h->fast : st;
