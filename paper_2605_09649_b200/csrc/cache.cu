@@ -144,8 +144,9 @@ __device__ __forceinline__ u64 bits_below(int n) {   // mask with the lowest n b
     return n >= 64 ? ~0ull : ((1ull << n) - 1ull);
 }
 
-// Block-wide exclusive scan of a 64-bit value over 256 threads; returns the exclusive prefix and the total.
-__device__ __forceinline__ u64 block_exscan_256(u64 v, u64* total, u64* warp_tot /*[8] shared*/) {
+// Block-wide exclusive scan of a 64-bit value over NW warps; returns the exclusive prefix and the total.
+template <int NW>
+__device__ __forceinline__ u64 block_exscan(u64 v, u64* total, u64* warp_tot /*[NW] shared*/) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     u64 incl = v;
 #pragma unroll
@@ -158,7 +159,7 @@ __device__ __forceinline__ u64 block_exscan_256(u64 v, u64* total, u64* warp_tot
     __syncthreads();
     u64 off = 0, tot = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) {
+    for (int w = 0; w < NW; ++w) {
         const u64 t = warp_tot[w];
         if (w < warp) off += t;
         tot += t;
@@ -170,10 +171,13 @@ __device__ __forceinline__ u64 block_exscan_256(u64 v, u64* total, u64* warp_tot
 // One CTA per pool.  Entries flagged in evict_mask are removed: with n' = n - E survivors, the E' holes
 // at logical index < n' are filled, in ascending order, by the survivors at index >= n' (ascending), so
 // only as many rows move as there are holes.  Pages past the new end return to the free stack.
-__global__ void __launch_bounds__(256)
+// NT threads: 256 when many rows move (after a prefill chunk), 128 for the one or two evictions per pool of a decode
+// step (all CTAs of the launch are then resident at once).
+template <int NT>
+__global__ void __launch_bounds__(NT)
 compact_kernel(CacheView cv, int32_t* __restrict__ hole, int32_t* __restrict__ mover, int32_t* __restrict__ cursor,
                long long e_max) {
-    __shared__ u64 warp_tot[8];
+    __shared__ u64 warp_tot[NT / 32];
     __shared__ long long s_base;
     __shared__ int s_freebase;
     const long long pool = blockIdx.x;
@@ -191,7 +195,7 @@ compact_kernel(CacheView cv, int32_t* __restrict__ hole, int32_t* __restrict__ m
         e_local += __popcll(masks[bt[lp]] & valid);
     }
     u64 E;
-    block_exscan_256(e_local, &E, warp_tot);
+    block_exscan<NT / 32>(e_local, &E, warp_tot);
     if (E == 0) return;
     const int n2 = n - (int)E;
 
@@ -221,7 +225,7 @@ compact_kernel(CacheView cv, int32_t* __restrict__ hole, int32_t* __restrict__ m
         }
         const u64 packed = ((u64)__popcll(hb) << 32) | (u64)__popcll(mb);
         u64 tot;
-        const u64 ex = block_exscan_256(packed, &tot, warp_tot);
+        const u64 ex = block_exscan<NT / 32>(packed, &tot, warp_tot);
         long long ho = run_h + (long long)(ex >> 32), mo = run_m + (long long)(ex & 0xffffffffu);
         while (hb) {
             const int bit = __ffsll((long long)hb) - 1;
@@ -337,9 +341,12 @@ void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long
 }
 
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max,
-                    cudaStream_t st) {
+                    long long evictions_per_seq, cudaStream_t st) {
     const long long pools = (long long)cv.B * cv.L * cv.H;
-    compact_kernel<<<(unsigned)pools, 256, 0, st>>>(cv, hole, mover, cursor, e_max);
+    if (evictions_per_seq <= 4LL * cv.L * cv.H)
+        compact_kernel<128><<<(unsigned)pools, 128, 0, st>>>(cv, hole, mover, cursor, e_max);
+    else
+        compact_kernel<256><<<(unsigned)pools, 256, 0, st>>>(cv, hole, mover, cursor, e_max);
     count_launch();
 }
 

@@ -177,7 +177,9 @@ void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long
                               int32_t* compact_cursor, cudaStream_t st);
 // Fixed per-pool budget: every pool keeps its keep_per_pool best entries (masks as for launch_select_cache).
 void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st);
-void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max, cudaStream_t st);
+// evictions_per_seq: how many entries the selection just flagged per sequence (sizes the CTAs).
+void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max,
+                    long long evictions_per_seq, cudaStream_t st);
 
 void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,
                          int32_t* err, cudaStream_t st);

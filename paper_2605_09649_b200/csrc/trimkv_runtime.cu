@@ -220,7 +220,7 @@ trimkv_status select_impl(trimkv* h, long long k, cudaStream_t sel_st) {
 trimkv_status compact_impl(trimkv* h, cudaStream_t st) {
     PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
     if (pm) pm->mark(PH_COMPACT, 0, st);
-    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, st);
+    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, eviction_due(h), st);
     if (pm) pm->mark(PH_COMPACT, 1, st);
     h->entries -= eviction_due(h);
     CUDA_TRY(cudaGetLastError());
