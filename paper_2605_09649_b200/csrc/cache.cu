@@ -330,8 +330,9 @@ void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st) {
     const int grid = nlayers * cv.B * cv.H;
     const bool split = (mode & APPEND_KV) && n_new >= 4 * APPEND_TOK;     // a chunk: copy its rows with a grid of their own
-    append_kernel<<<grid, 256, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v,
-                                        split ? (mode | APPEND_ROWS_ELSEWHERE) : mode);
+    const int threads = n_new <= 2 ? 64 : 256;        // a decode step's row pair is 64 chunks: small CTAs, all resident at once
+    append_kernel<<<grid, threads, 0, st>>>(cv, layer0, n_new, pos0, lam, c, horizon, (const char*)k, (const char*)v,
+                                            split ? (mode | APPEND_ROWS_ELSEWHERE) : mode);
     count_launch();
     if (split) {
         dim3 g2(grid, (n_new + APPEND_TOK - 1) / APPEND_TOK);
