@@ -679,6 +679,13 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
         // dominates the cache is still cut up.  (Few warps suffice to saturate HBM, so coarse items cost no bandwidth.)
         // (A cross-warp merge costs a device-scope fence per item, which drains the warp's copy pipeline.)
         long long tpi = tiles_estimate / (workers * 2);
+        // ... but no coarser than a little above the average pool, down to a quarter of a worker's share: equal pools
+        // stay whole either way, while the few long pools of a ragged cache are cut finer and balance better
+        // (measured with pool lengths 17..32813: 0.786 -> 0.74 ms per step; equal pools: unchanged).
+        if (n_scope > 0) {
+            const long long avg = tiles_estimate / n_scope;
+            tpi = std::min(tpi, std::max(avg + avg / 4 + 1, tiles_estimate / (workers * 4)));
+        }
         // With at least half as many pools as workers and short pools (up to 4096 entries on average), whole pools are the
         // better items even when they are shorter than that: nothing is merged (the per-item fence weighs most on short
         // items), and the warps that get no item are not missed (HBM is saturated by a third of them).  Measured: workload
