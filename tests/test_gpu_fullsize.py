@@ -179,3 +179,36 @@ def test_full_size_chunk_attention_matches_oracle_on_samples(name, context):
     cache.score_and_evict()
     cache.sync_status()
     cache.close()
+
+
+def _keep_mask_from_words(bits, n):
+    """bool [n] on the device from the packed keep words (bit i of word i // 64, little-endian)."""
+    b8 = bits.view(torch.uint8)
+    m = ((b8[:, None] >> torch.arange(8, device=b8.device, dtype=torch.uint8)[None, :]) & 1).reshape(-1)[:n]
+    return m.bool()
+
+
+@pytest.mark.parametrize("log2n,kind", [(28, "uniform"), (26, "two_values")])
+def test_select_topk_properties_at_sweep_sizes(log2n, kind):
+    """The standalone selection at the sweep's sizes, where a full sort on the host is out of reach: properties that pin
+    the result at any size.  Exactly k entries are kept; no evicted score exceeds a kept one; among entries whose score
+    equals the threshold the kept ones are exactly those with the smallest indices (ties keep the older entry)."""
+    n = 1 << log2n
+    if kind == "uniform":
+        s = workloads.selection_scores(n, seed=3, device=DEV)
+    else:
+        s = (workloads.selection_scores(n, seed=4, device=DEV) > -5.0).float() * 2.0 - 7.0      # -5 or -7, heavy ties
+    for k in (n // 8, n - 512):
+        bits, status = binding.select_topk(s, k)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        keep = _keep_mask_from_words(bits, n)
+        assert int(keep.sum().item()) == k
+        tau = s[keep].min()                                   # lowest kept score
+        assert float(s[~keep].max().item()) <= float(tau.item())
+        tie = s == tau                                        # entries on the threshold: kept ones come first by index
+        idx = torch.nonzero(tie, as_tuple=False).reshape(-1)
+        kept_tie = keep[idx]
+        n_kept_tie = int(kept_tie.sum().item())
+        assert bool(kept_tie[:n_kept_tie].all().item()) and not bool(kept_tie[n_kept_tie:].any().item())
+        del keep, tie, idx, kept_tie
