@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_mma_kernel launch, from the ncu capture summarised in
 # profiles/attn_mma_kernel_llama8b_cache_at_budget.md (same kernel source as now; set to None when the kernel changes).
-NCU_TRAFFIC_BYTES = {"llama8b_32k": 4315471000 + 6803000}
+NCU_TRAFFIC_BYTES = {"llama8b_32k": 4315508000 + 2926000}
 
 METRIC = "decode tokens/s at fixed global KV budget (step time in ms_per_step, % of HBM peak in roofline)"
 UNIT = "tokens/s"
