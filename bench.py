@@ -412,7 +412,7 @@ def run_ours(args, w):
                    "earlier_turn_decode_ms_per_step": early_decode_ms / early_decode_steps if early_decode_steps else None},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if args.skew == 0 and args.context is None else None,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if args.skew == 0 and args.context is None and args.layers is None else None,
                      "algorithmic_bytes_per_launch": ab["kv"], "avg_launch_ms": attn_ms_per,
                      "note": "timed region: the kernel shares HBM with the gate and selection kernels running beside it",
                      "alone": {"avg_launch_ms": iso_ms, "achieved": iso_gbs, "frac": iso_gbs / peak},
