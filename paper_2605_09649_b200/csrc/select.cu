@@ -654,7 +654,7 @@ sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample
 // nearly empty and then takes the bin's outer edge, which only widens the range.
 __global__ void __launch_bounds__(1024)
 bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long long k_evict, long long n_total,
-               int distrust) {
+               int distrust, float sigmas) {
     constexpr int DB = 11, NBIN = 1 << DB, PER = SAMPLE_CAP / 1024;
     __shared__ unsigned hist[NBIN];
     __shared__ unsigned wtot[32];
@@ -744,7 +744,7 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
             r_lo = r_hi = k_evict;
         } else {
             const double mu = (double)k_evict * (double)ns / (double)n_total;   // expected sample rank of the k-th key
-            const double dev = 7.0 * sqrt(mu) + 8.0;
+            const double dev = (double)sigmas * sqrt(mu) + 8.0;  // margin in standard deviations of the sample rank
             r_lo = (long long)floor(mu - dev);
             r_hi = (long long)ceil(mu + dev) + 1;
         }
@@ -1271,7 +1271,8 @@ void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, lo
     const long long threads = cv.P_seq * (sub > 0 ? PAGE / sub : 1);
     dim3 gs((unsigned)((threads + 255) / 256), cv.B);
     sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, sub, thresh, seed, skip_newest);
-    bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample);
+    // 7 sigma: a miss costs the single-CTA exact redo of the whole sequence, so it must be next to impossible
+    bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample, 7.0f);
     count_launch(2);
 }
 
@@ -1309,7 +1310,9 @@ void launch_select_array(const float* scores, long long n, long long k_evict, u6
     src.err = err;
     u64* sample = reinterpret_cast<u64*>(sb.cand);        // the candidate buffer is idle until the filter pass
     flat_sample_kernel<<<SAMPLE_CAP / 1024, 1024, 0, st>>>(scores, n, sb.sel, sample);
-    bracket_kernel<<<1, 1024, 0, st>>>(sb.sel, sample, k_evict, n, 0);
+    // 4 sigma: here a miss (6e-5 per call) only costs one more histogram pass, and the narrower range keeps the
+    // candidate list of the last bin within what the resolution holds in registers
+    bracket_kernel<<<1, 1024, 0, st>>>(sb.sel, sample, k_evict, n, 0, 4.0f);
     flat_range_kernel<<<1, 1, 0, st>>>(sb.sel);
     count_launch(3);
     run_select_flat(src, sb, k_evict, 7, (unsigned)sb.cand_cap, evict_mask, err, st);
