@@ -71,8 +71,8 @@ def horizon_term(lam, horizon):
     if horizon == 0:
         with np.errstate(divide="ignore"):
             return -np.log(-np.expm1(lam))
-    acc = np.zeros_like(lam)
-    for k in range(int(horizon)):
+    acc = np.ones_like(lam)                      # k = 0: beta^0 = 1 for every beta, beta = 0 (lam = -inf) included
+    for k in range(1, int(horizon)):
         acc = acc + np.exp(k * lam)
     return np.log(acc)
 

@@ -71,6 +71,9 @@ def test_score_limits():
     # beta = 1: the sum has h unit terms; infinite horizon diverges
     assert orc.horizon_term(np.array([0.0]), 4)[0] == math.log(4)
     assert np.isposinf(orc.horizon_term(np.array([0.0]), 0)[0])
+    # beta = 0 (lambda = -inf): only the k = 0 term, beta^0 = 1, survives: c = ln 1 = 0 for every horizon
+    for h in (1, 2, 5, 0):
+        assert orc.horizon_term(np.array([-np.inf]), h)[0] == 0.0
 
 
 def test_score_is_two_separately_rounded_fp32_ops():
@@ -489,3 +492,18 @@ def test_set_horizon_rescoring_closed_forms():
     for l in range(L):
         for hh in range(H):
             np.testing.assert_array_equal(b.kept_positions(l, hh), np.arange(8, 13))
+
+
+def test_rounding_contract_case_discriminates_fused_and_fp64_scores():
+    """The inputs of the GPU score-rounding test: in EVERY sequence the kept set under the contract's score (fp32
+    multiply, then fp32 add) differs from the kept set under a fused multiply-add and under fp64 evaluation, so a kernel
+    that contracts the two operations, or scores in higher precision, cannot reproduce the oracle's sets."""
+    import util_parity as up
+    lam, c, budget = up.rounding_contract_case(seed=5, B=24, n=48, L=2, H=2)
+    want = up.rounding_contract_kept_sets(lam, c, budget, "contract")
+    fused = up.rounding_contract_kept_sets(lam, c, budget, "fused")
+    fp64 = up.rounding_contract_kept_sets(lam, c, budget, "fp64")
+    for b in range(lam.shape[1]):
+        assert len(want[b]) == budget
+        assert want[b] != fused[b] and want[b] != fp64[b]
+        assert len(want[b] ^ fused[b]) == 2 and len(want[b] ^ fp64[b]) == 2      # exactly the pair's two members swap
