@@ -72,8 +72,7 @@ typedef struct trimkv_config {
     int32_t horizon;        /* lookahead T - t (Sec. 5.1: 2); 0 = infinite horizon             */
     int32_t kv_dtype;       /* TRIMKV_DTYPE_BF16 or TRIMKV_DTYPE_F32 (K, V, q and out)         */
     int32_t max_chunk;      /* largest n_new of one append (1 for pure decode)                 */
-    int32_t reserved;       /* 0; bit 0 = testing aid: distrust the selection's key sample, so that the
-                               exact single-CTA redo of the selection runs in every eviction round  */
+    int32_t reserved;       /* must be 0                                                       */
     int64_t max_pool_pages; /* cap on pages of one (layer, head) pool; 0 = a pool may take all */
     int32_t retention_bias; /* 0: decode attention is the plain softmax over the retained set (Eq. (1));
                                1: retention-gated weights beta_i^(t-i) e^{z_i} of Sec. 2.2 (t = tokens seen) */
@@ -119,7 +118,11 @@ TRIMKV_API trimkv_status trimkv_gate(trimkv_t* h, int layer, int n_new, const fl
  * enters the cache, Sec. 3.2).  k, v: device [B, n_new, H, d] in kv_dtype.
  * Retention: x != NULL -> gate on x [B, n_new, D] fp32; else lambda [B, n_new, H] fp32 (<= 0) is
  * required and c [B, n_new, H] is optional (NULL -> derived from lambda on the device in fp32).
- * Token j of the call gets position tokens(layer) + j + 1.  n_new <= max_chunk. */
+ * Token j of the call gets position tokens(layer) + j + 1.  n_new <= max_chunk.
+ * Capacity rule: the cache has room for the budget plus ONE chunk of max_chunk tokens per layer, so an eviction round
+ * (trimkv_score_and_evict) must run before a sequence would hold more than budget_entries + max_chunk * layers *
+ * kv_heads entries (per_pool_budget > 0: per_pool_budget * layers * kv_heads in place of budget_entries).  An append
+ * that would exceed this is refused with TRIMKV_E_STATE and changes nothing. */
 TRIMKV_API trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, const float* lambda, const float* c,
                             const void* k, const void* v, void* stream);
 
@@ -201,6 +204,20 @@ TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);
 /* enable = 2 records the attention main kernel alone (two events per call: cheap enough for a timed run). */
 TRIMKV_API trimkv_status trimkv_profile(trimkv_t* h, int enable);
 TRIMKV_API trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host);
+
+/* ---- testing aids (not part of the method) ------------------------------------------------------
+ * Switches that make rarely taken paths run on demand, so that tests can reach them without a fault:
+ *   TRIMKV_TEST_DISTRUST_SAMPLE      the selection ignores its key sample; the exact fallback of the selection (cache:
+ *                                    the single-CTA redo; flat arrays: the histogram passes) then runs in every call.
+ *                                    Results are unchanged.
+ *   TRIMKV_TEST_ATTENTION_NO_COPY    the tensor-core decode attention kernel issues none of its asynchronous K/V copies
+ *                                    and uses a short limit for its waits: every wait runs out, the kernel latches
+ *                                    TRIMKV_E_TIMEOUT and returns with nothing in flight (its output is not written).
+ * h != NULL sets the switches of that handle; h == NULL those of the handle-less calls (trimkv_select_topk and
+ * trimkv_select_topk_static) for the whole process.  flags = 0 restores normal operation.  Synchronises. */
+#define TRIMKV_TEST_DISTRUST_SAMPLE 1
+#define TRIMKV_TEST_ATTENTION_NO_COPY 2
+TRIMKV_API trimkv_status trimkv_set_test_hooks(trimkv_t* h, int flags);
 
 /* Message of the calling thread's last failed call; never NULL. */
 TRIMKV_API const char* trimkv_last_error(void);

@@ -18,13 +18,14 @@ LIB_PATH = os.path.join(_HERE, "libtrimkv.so")
 OK, E_ARG, E_STATE, E_NOMEM, E_CUDA, E_NONFINITE, E_TIMEOUT, E_UNSUPPORTED = range(8)
 STATUS_NAMES = ["OK", "E_ARG", "E_STATE", "E_NOMEM", "E_CUDA", "E_NONFINITE", "E_TIMEOUT", "E_UNSUPPORTED"]
 DTYPE_BF16, DTYPE_F32 = 0, 1
+TEST_DISTRUST_SAMPLE, TEST_ATTENTION_NO_COPY = 1, 2     # testing aids, see trimkv_set_test_hooks
 
 EXPORTS = [
     "trimkv_default_config", "trimkv_create", "trimkv_create_ex", "trimkv_destroy", "trimkv_reset", "trimkv_set_gate",
     "trimkv_set_shared_projection", "trimkv_gate", "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention",
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
-    "trimkv_select_topk", "trimkv_select_topk_static",
+    "trimkv_select_topk", "trimkv_select_topk_static", "trimkv_set_test_hooks",
 ]
 
 
@@ -83,6 +84,7 @@ def lib() -> C.CDLL:
     L.trimkv_sync_status.argtypes = [vp]
     L.trimkv_profile.argtypes = [vp, i32]
     L.trimkv_set_overlap.argtypes = [vp, i32]
+    L.trimkv_set_test_hooks.argtypes = [vp, i32]
     L.trimkv_set_horizon.argtypes = [vp, i32, vp]
     L.trimkv_profile_read.argtypes = [vp, vp, vp]
     L.trimkv_last_error.argtypes = []
@@ -97,7 +99,7 @@ def lib() -> C.CDLL:
                  "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention", "trimkv_decode_step_all",
                  "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
                  "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_select_topk",
-                 "trimkv_select_topk_static", "trimkv_set_overlap", "trimkv_set_horizon"):
+                 "trimkv_select_topk_static", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_set_test_hooks"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -153,13 +155,15 @@ class TrimKV:
         cfg.max_pool_pages = max_pool_pages
         cfg.retention_bias = 1 if retention_bias else 0
         cfg.per_pool_budget = per_pool_budget
-        cfg.reserved = 1 if distrust_sample else 0     # testing aid: forces the selection's exact redo path
+        cfg.reserved = 0
         self.cfg = cfg
         self.torch_dtype = torch.bfloat16 if kv_dtype == "bf16" else torch.float32
         self.B, self.L, self.H, self.Hq, self.d, self.D = batch, layers, kv_heads, cfg.q_heads, head_dim, hidden
         h = C.c_void_p()
         _check(L.trimkv_create_ex(C.byref(cfg), C.byref(h)))
         self._h = h
+        if distrust_sample:                            # testing aid: forces the selection's exact redo path
+            self.set_test_hooks(TEST_DISTRUST_SAMPLE)
 
     @classmethod
     def from_workload(cls, w, **overrides) -> "TrimKV":
@@ -252,6 +256,10 @@ class TrimKV:
         """New horizon T - t for stored and future entries (0 = infinite)."""
         _check(lib().trimkv_set_horizon(self._h, int(horizon), _stream()))
 
+    def set_test_hooks(self, flags: int):
+        """Testing aids of this handle (TEST_* flags; 0 = normal operation)."""
+        _check(lib().trimkv_set_test_hooks(self._h, int(flags)))
+
     def set_overlap(self, enable: bool):
         _check(lib().trimkv_set_overlap(self._h, 1 if enable else 0))
 
@@ -292,6 +300,11 @@ class TrimKV:
         out = torch.empty(self.B, 4, dtype=torch.int64)
         _check(lib().trimkv_get_select_stats(self._h, C.c_void_p(out.data_ptr())))
         return out
+
+
+def set_global_test_hooks(flags: int):
+    """Testing aids of the handle-less calls (select_topk, select_topk_static); 0 = normal operation."""
+    _check(lib().trimkv_set_test_hooks(None, int(flags)))
 
 
 def select_workspace_bytes(n: int) -> int:

@@ -34,6 +34,7 @@ constexpr int ATT_META_OFF = (ATT_RING_OFF + ATT_WARPS * ATT_RING * 4 + 127) & ~
 constexpr int ATT_META_BYTES = 2 * TILE * 4;
 constexpr int ATT_SMEM = ATT_META_OFF + ATT_WARPS * ATT_STAGES * ATT_META_BYTES;
 constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
+constexpr unsigned WAIT_LIMIT_TEST = 1u << 8;  // the limit of the testing aid under which no copy is ever issued
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -55,8 +56,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Returns false if the wait gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    for (unsigned it = 0; it < WAIT_LIMIT; ++it)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, unsigned limit = WAIT_LIMIT) {
+    for (unsigned it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -127,7 +128,9 @@ __device__ __forceinline__ int tiles_per_item(int len, int items) {
 
 // NT = ceil(g / 8): column tiles of 8 query heads.  BIAS: retention-gated weights beta_i^(t-i) e^{z_i} (Sec. 2.2): the
 // entries' lambda and position travel with each tile and (t_now - pos) * lambda is added to the logit.
-template <int NT, bool BIAS>
+// NO_COPY (testing aid): the producer issues no asynchronous copy at all and the waits use a short limit, so every
+// wait runs out with nothing in flight: the kernel latches TRIMKV_E_TIMEOUT and returns; its output is not written.
+template <int NT, bool BIAS, bool NO_COPY = false>
 __global__ void __launch_bounds__(ATT_WARPS * 32, 1)
 attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, int Hq, int t_now, int32_t* __restrict__ pool_done,
                 int32_t* __restrict__ sched,
@@ -245,7 +248,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
         }
         const int page = __shfl_sync(0xffffffffu, prod.page_id, (tt >> 1) & 31);
         const int half = (prod.first_tile + tt) & 1;
-        if (lane == 0) {
+        if (lane == 0 && !NO_COPY) {
             const unsigned s = issued % ATT_STAGES;
             unsigned char* dst = wbuf + (size_t)s * STAGE_BYTES;
             const char* ksrc = cv.kv + kv_row_offset(cv, prod.b, page, 0, half * TILE);
@@ -310,7 +313,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
         for (int tt = 0; tt < cons.ntile; ++tt) {
             issue_one();    // refill the stage freed by the previous tile
             const unsigned s = consumed % ATT_STAGES;
-            if (!mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u)) { failed = true; break; }
+            if (!mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u, NO_COPY ? WAIT_LIMIT_TEST : WAIT_LIMIT)) { failed = true; break; }
             ++consumed;
             const uint32_t kbase = smem_u32(wbuf + (size_t)s * STAGE_BYTES);
             const uint32_t vbase = kbase + TILE * ROWB;
@@ -324,7 +327,10 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int r = mt * 16 + hh * 8 + (lane >> 2);
-                        rb[mt][hh] = (float)(t_now - mpos[r]) * mlam[r] * 1.4426950408889634f;
+                        // age 0 (the token of this step): beta^0 = 1 whatever lambda is; its stored lambda may not be
+                        // written yet, and 0 * -inf would be NaN
+                        const int age = t_now - mpos[r];
+                        rb[mt][hh] = age == 0 ? 0.f : (float)age * mlam[r] * 1.4426950408889634f;
                     }
             }
 
@@ -562,7 +568,7 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
     if (failed) {
         latch_error(cv.err, TRIMKV_E_TIMEOUT);
         // drain: wait (bounded) for the copies still in flight before leaving shared memory
-        while (consumed < issued) {
+        while (!NO_COPY && consumed < issued) {
             const unsigned s = consumed % ATT_STAGES;
             mbar_wait_bounded(bars + s, (consumed / ATT_STAGES) & 1u);
             ++consumed;
@@ -630,7 +636,8 @@ attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T*
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (bias) {                                       // retention-gated weights: + (t - i) * lambda_i
             const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + off;
-            s += (float)(t_now - cv.pos[slot]) * cv.lam[slot];
+            const int age = t_now - cv.pos[slot];
+            if (age != 0) s += (float)age * cv.lam[slot];     // age 0: beta^0 = 1 (and 0 * -inf would be NaN)
         }
         const float mn = fmaxf(m, s);
         const float f = __expf(m - mn), p = __expf(s - mn);
@@ -654,18 +661,17 @@ attn_plain_kernel(CacheView cv, int layer0, int n_scope, int g, int Hq, const T*
 
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
                       long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, int reserve_sms,
-                      const void* q, void* out, cudaStream_t st, PhaseMarker* pm) {
+                      bool test_no_copy, const void* q, void* out, cudaStream_t st, PhaseMarker* pm) {
     const int n_scope = nlayers * cv.B * cv.H;
     const int g = Hq / cv.H;
     const float scale = 1.0f / sqrtf((float)cv.d);
     if (is_bf16 && cv.d == 128 && g <= 16) {
-        static bool attr_set = false;
-        if (!attr_set) {
+        if (first_use_on_device(0)) {
             cudaFuncSetAttribute(attn_mma_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
             cudaFuncSetAttribute(attn_mma_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
             cudaFuncSetAttribute(attn_mma_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
             cudaFuncSetAttribute(attn_mma_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
-            attr_set = true;
+            cudaFuncSetAttribute(attn_mma_kernel<1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM);
         }
         int dev = 0, sms = 148;
         cudaGetDevice(&dev);
@@ -708,7 +714,8 @@ void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, in
                                                           (const __nv_bfloat16*)q, (__nv_bfloat16*)out, ab.part_o, ab.part_ml,
                                                           scale_log2, ab.max_items);
         };
-        if (g <= 8) { if (retention_bias) launch(attn_mma_kernel<1, true>); else launch(attn_mma_kernel<1, false>); }
+        if (test_no_copy) launch(attn_mma_kernel<1, false, true>);      // testing aid: every wait runs out (see the kernel)
+        else if (g <= 8) { if (retention_bias) launch(attn_mma_kernel<1, true>); else launch(attn_mma_kernel<1, false>); }
         else        { if (retention_bias) launch(attn_mma_kernel<2, true>); else launch(attn_mma_kernel<2, false>); }
         if (pm) pm->mark(PH_ATTN_MAIN, 1, st);
         count_launch(1);

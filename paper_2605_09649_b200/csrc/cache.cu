@@ -27,8 +27,9 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
     int32_t* bt = cv.block_table + pool * cv.maxpp;
 
     if (!(mode & APPEND_KV)) {
+        if (cv.append_failed[pool]) return;            // the K/V half of this append failed (its error is latched)
         const int old = cv.len[pool] - n_new;
-        if (old < 0) return;                           // the K/V half of this append failed (its error is latched)
+        if (old < 0) return;
         const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
         for (int j = threadIdx.x; j < n_new; j += blockDim.x) {
             const int idx = old + j;
@@ -65,6 +66,7 @@ append_kernel(CacheView cv, int layer0, int n_new, long long pos0, const float* 
             }
         }
         if (fail) latch_error(cv.err, TRIMKV_E_NOMEM);
+        cv.append_failed[pool] = fail;                 // read by the halves of this append that run later
         s_old = old;
         s_fail = fail;
     }
@@ -121,8 +123,9 @@ append_rows_kernel(CacheView cv, int layer0, int n_new, const char* __restrict__
     const int pool_local = (layer0 + lb) * cv.H + h;
     const long long pool = (long long)b * cv.L * cv.H + pool_local;
     const int32_t* bt = cv.block_table + pool * cv.maxpp;
+    if (cv.append_failed[pool]) return;                // the bookkeeping half failed (its error is latched)
     const int old = cv.len[pool] - n_new;
-    if (old < 0) return;                               // the bookkeeping half failed (its error is latched)
+    if (old < 0) return;
     const int rc = cv.row_bytes / 16;
     const size_t in_row0 = (((size_t)lb * cv.B + b) * n_new) * cv.H + h;
     const int j0 = blockIdx.y * APPEND_TOK;

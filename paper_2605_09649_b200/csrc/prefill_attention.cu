@@ -380,11 +380,8 @@ void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq,
     const int g = Hq / cv.H;
     const float scale = 1.0f / sqrtf((float)cv.d);
     if (is_bf16 && cv.d == 128 && g <= P_COLS) {
-        static bool attr_set = false;
-        if (!attr_set) {
+        if (first_use_on_device(1))
             cudaFuncSetAttribute(prefill_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P_SMEM);
-            attr_set = true;
-        }
         const int tc = P_WARPS * (P_COLS / g);
         dim3 grid((n_new + tc - 1) / tc, cv.B * cv.H);
         prefill_attn_mma_kernel<<<grid, P_WARPS * 32, P_SMEM, st>>>(cv, layer, n_new, g, Hq, (const __nv_bfloat16*)q,

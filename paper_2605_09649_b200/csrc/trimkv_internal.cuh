@@ -93,6 +93,7 @@ struct CacheView {
     int32_t* free_count;   // [B]
     u64* evict_mask;       // [B][P_seq]
     int32_t* err;          // latched device status
+    int32_t* append_failed; // [B*L*H] 1 if the bookkeeping half of the pool's last append failed (no page), else 0
     long long P_seq;       // pages per sequence
     long long maxpp;       // block-table row length
     int B, L, H, d;
@@ -206,7 +207,7 @@ struct PhaseMarker {
 // retention_bias != 0: retention-gated weights beta_i^(t_now - i) e^{z_i} instead of the plain softmax.
 void launch_attention(const CacheView& cv, const AttnBuffers& ab, int layer0, int nlayers, int Hq, int is_bf16,
                       long long tiles_estimate, long long tiles_upper, int retention_bias, long long t_now, int reserve_sms,
-                      const void* q, void* out, cudaStream_t st, PhaseMarker* pm);
+                      bool test_no_copy, const void* q, void* out, cudaStream_t st, PhaseMarker* pm);
 
 // Causal attention of the chunk of n_new tokens just appended to `layer`; q, out: [B, n_new, Hq, d].
 // tc: state of the tensor-core (tcgen05) form, or null; used when the chunk is large enough to fill its tiles.
@@ -227,6 +228,13 @@ void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32
                         void* v, int n, cudaStream_t st);
 
 void count_launch(int n = 1);
+
+// TRIMKV_TEST_* switches of the handle-less calls.
+int global_test_hooks();
+
+// True the first time it is called for (slot, current device): kernels with more than 48 KB of dynamic shared memory
+// need their opt-in attribute set once per device, not once per process.
+bool first_use_on_device(int slot);
 
 // Sets the calling thread's message returned by trimkv_last_error (printf format).
 void set_last_error(const char* fmt, ...);

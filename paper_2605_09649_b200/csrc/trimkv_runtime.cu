@@ -12,6 +12,15 @@
 namespace tkv {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+static std::atomic<int> g_test_hooks{0};   // testing aids of the handle-less calls (trimkv_set_test_hooks(NULL, ...))
+int global_test_hooks() { return g_test_hooks.load(std::memory_order_relaxed); }
+bool first_use_on_device(int slot) {
+    constexpr int MAX_DEV = 64, SLOTS = 8;
+    static std::atomic<bool> seen[SLOTS][MAX_DEV];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEV || slot < 0 || slot >= SLOTS) return true;
+    return !seen[slot][dev].exchange(true);
+}
 }  // namespace tkv
 
 using namespace tkv;
@@ -111,6 +120,9 @@ struct trimkv {
     cudaStream_t fast = nullptr, side = nullptr, side2 = nullptr;   // side2: the selection's sampling, beside the gate
     cudaStream_t side_hi = nullptr;                                 // `side` at the priority of `fast` (gate-heavy steps)
     bool overlap = true;
+    int test_hooks = 0;              // TRIMKV_TEST_* switches of this handle
+    char* pool_stage = nullptr;      // device staging of trimkv_get_pool, grown on demand
+    size_t pool_stage_bytes = 0;
     cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr, ev_sample = nullptr;
 };
 
@@ -146,6 +158,7 @@ trimkv_status init_cache_state(trimkv* h) {
     CUDA_TRY(cudaMemcpy(h->cv.owner, own.data(), own.size() * sizeof(int4), cudaMemcpyHostToDevice));
     CUDA_TRY(cudaMemset(h->cv.len, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->cv.err, 0, sizeof(int32_t)));
+    CUDA_TRY(cudaMemset(h->cv.append_failed, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->sb.hist, 0, (size_t)h->B * NB * sizeof(uint32_t)));
     CUDA_TRY(cudaMemset(h->sb.done, 0, (size_t)h->B * sizeof(unsigned)));
     CUDA_TRY(cudaMemset(h->sb.stats, 0, (size_t)h->B * 4 * sizeof(long long)));
@@ -205,6 +218,12 @@ long long eviction_due(const trimkv* h) {
     return h->entries - h->M;
 }
 
+// Entries per sequence the cache has room for between two eviction rounds: what survives a round plus one chunk.
+long long capacity_entries(const trimkv* h) {
+    const long long LH = (long long)h->L * h->H;
+    return (h->cfg.per_pool_budget > 0 ? (long long)h->cfg.per_pool_budget * LH : h->M) + h->e_max;
+}
+
 // Selection on `sel_st`, compaction on `st`; when the two differ the caller orders them with events.
 trimkv_status select_impl(trimkv* h, long long k, cudaStream_t sel_st) {
     PhaseMarker* pm = h->prof.on ? &h->prof : nullptr;
@@ -212,7 +231,7 @@ trimkv_status select_impl(trimkv* h, long long k, cudaStream_t sel_st) {
     if (h->cfg.per_pool_budget > 0)
         launch_select_pools(h->cv, h->tokens[0], h->cfg.per_pool_budget, h->cursor, sel_st);
     else
-        launch_select_cache(h->cv, h->sb, h->tokens[0], h->entries, k, h->cursor, h->cfg.reserved & 1, sel_st);
+        launch_select_cache(h->cv, h->sb, h->tokens[0], h->entries, k, h->cursor, h->test_hooks & TRIMKV_TEST_DISTRUST_SAMPLE, sel_st);
     if (pm) pm->mark(PH_SELECT, 1, sel_st);
     return TRIMKV_OK;
 }
@@ -241,7 +260,8 @@ trimkv_status attention_impl(trimkv* h, int layer0, int nlayers, const void* q, 
     const long long tiles = (h->entries * h->B / 32) * nlayers / h->L + (long long)nlayers * h->B * h->H;
     const long long tiles_upper = h->entries * h->B / 32 + (long long)nlayers * h->B * h->H;
     launch_attention(h->cv, h->ab, layer0, nlayers, h->Hq, h->cfg.kv_dtype == TRIMKV_DTYPE_BF16, tiles, tiles_upper,
-                     h->cfg.retention_bias, h->tokens[layer0], reserve_sms, q, out, st, h->prof.on ? &h->prof : nullptr);
+                     h->cfg.retention_bias, h->tokens[layer0], reserve_sms, (h->test_hooks & TRIMKV_TEST_ATTENTION_NO_COPY) != 0,
+                     q, out, st, h->prof.on ? &h->prof : nullptr);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
 }
@@ -284,6 +304,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
         cfg->max_chunk < 1)
         return fail(TRIMKV_E_ARG, "budget, layers, kv_heads, head_dim, max_batch and max_chunk must be positive");
     if (cfg->page_size != PAGE) return fail(TRIMKV_E_UNSUPPORTED, "page_size must be %d", PAGE);
+    if (cfg->reserved != 0) return fail(TRIMKV_E_ARG, "reserved must be 0");
     if (cfg->q_heads < cfg->kv_heads || cfg->q_heads % cfg->kv_heads) return fail(TRIMKV_E_ARG, "q_heads must be a multiple of kv_heads");
     if (cfg->kv_dtype != TRIMKV_DTYPE_BF16 && cfg->kv_dtype != TRIMKV_DTYPE_F32) return fail(TRIMKV_E_ARG, "unknown kv_dtype");
     if (cfg->head_dim % 8 || cfg->head_dim > 256) return fail(TRIMKV_E_UNSUPPORTED, "head_dim must be a multiple of 8, at most 256");
@@ -339,6 +360,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     A(dev_alloc(h, &cv.free_count, (size_t)h->B, false));
     A(dev_alloc(h, &cv.evict_mask, (size_t)h->B * h->P_seq, true));
     A(dev_alloc(h, &cv.err, 1, true));
+    A(dev_alloc(h, &cv.append_failed, pools, true));
     SelectBuffers& sb = h->sb;
     sb.cand_cap = h->n_max;
     A(dev_alloc(h, &sb.sel, (size_t)h->B, true));
@@ -426,6 +448,7 @@ void trimkv_destroy(trimkv_t* h) {
     if (h->side) cudaStreamDestroy(h->side);
     if (h->fast) cudaStreamDestroy(h->fast);
     for (void* p : h->allocs) cudaFree(p);
+    if (h->pool_stage) cudaFree(h->pool_stage);
     gate_tc_destroy(h->tc);
     prefill_tc_destroy(h->ptc);
     delete h;
@@ -487,6 +510,9 @@ trimkv_status trimkv_append(trimkv_t* h, int layer, int n_new, const float* x, c
     if (!k || !v || !aligned16(k) || !aligned16(v)) return fail(TRIMKV_E_ARG, "k and v must be non-NULL and 16-byte aligned");
     if (!x && !lambda) return fail(TRIMKV_E_ARG, "either x or lambda is required");
     if (h->tokens[layer] + n_new > h->max_pos) return fail(TRIMKV_E_UNSUPPORTED, "position limit %lld reached", h->max_pos);
+    if (h->entries + (long long)n_new * h->H > capacity_entries(h))
+        return fail(TRIMKV_E_STATE, "the cache holds %lld entries per sequence and has room for %lld: run trimkv_score_and_evict "
+                    "before appending more (at most max_chunk tokens per layer between eviction rounds)", h->entries, capacity_entries(h));
     cudaStream_t st = (cudaStream_t)stream;
     const float* lam = lambda;
     const float* cc = c;
@@ -551,6 +577,9 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layers hold different token counts");
     if (t + 1 > h->max_pos) return fail(TRIMKV_E_UNSUPPORTED, "position limit %lld reached", h->max_pos);
+    if (h->entries + (long long)h->L * h->H > capacity_entries(h))
+        return fail(TRIMKV_E_STATE, "the cache holds %lld entries per sequence and has room for %lld: run trimkv_score_and_evict first",
+                    h->entries, capacity_entries(h));
     cudaStream_t st = (cudaStream_t)stream;
     if (x) {
         if (trimkv_status s = gate_ready(h, 0, h->L)) return s;
@@ -614,7 +643,7 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     const bool early_sample = two && kev > 0 && h->cfg.per_pool_budget == 0 && side_critical;
     if (early_sample) {
         CUDA_TRY(cudaStreamWaitEvent(h->side2, h->ev_append, 0));
-        launch_select_cache_sample(h->cv, h->sb, h->tokens[0], h->entries, kev, 1, h->cfg.reserved & 1, h->side2);
+        launch_select_cache_sample(h->cv, h->sb, h->tokens[0], h->entries, kev, 1, h->test_hooks & TRIMKV_TEST_DISTRUST_SAMPLE, h->side2);
         CUDA_TRY(cudaEventRecord(h->ev_sample, h->side2));
     }
     if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
@@ -685,10 +714,18 @@ trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap
     if (len > cap) return fail(TRIMKV_E_ARG, "pool holds %d entries, capacity %d", len, cap);
     if (len == 0) return device_status(h);
     const size_t rb = (size_t)h->d * h->elt;
-    char* tmp = nullptr;
     const size_t meta = ((size_t)len * 4 + 255) / 256 * 256;
     const size_t kvb = ((size_t)len * rb + 255) / 256 * 256;
-    CUDA_TRY(cudaMalloc((void**)&tmp, 3 * meta + 2 * kvb));
+    const size_t need = 3 * meta + 2 * kvb;
+    if (need > h->pool_stage_bytes) {                 // the staging buffer only grows; most calls reuse it
+        if (h->pool_stage) cudaFree(h->pool_stage);
+        h->pool_stage = nullptr;
+        h->pool_stage_bytes = 0;
+        const size_t want = std::max(need, (size_t)1 << 20);
+        CUDA_TRY(cudaMalloc((void**)&h->pool_stage, want));
+        h->pool_stage_bytes = want;
+    }
+    char* tmp = h->pool_stage;
     int32_t* dpos = (int32_t*)tmp;
     float* dlam = (float*)(tmp + meta);
     float* dc = (float*)(tmp + 2 * meta);
@@ -701,7 +738,6 @@ trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap
     if (e == cudaSuccess && c_host) e = cudaMemcpy(c_host, dc, (size_t)len * 4, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && k_host) e = cudaMemcpy(k_host, dk, (size_t)len * rb, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess && v_host) e = cudaMemcpy(v_host, dv, (size_t)len * rb, cudaMemcpyDeviceToHost);
-    cudaFree(tmp);
     if (e != cudaSuccess) return fail(TRIMKV_E_CUDA, "get_pool: %s", cudaGetErrorString(e));
     return device_status(h);
 }
@@ -742,6 +778,14 @@ trimkv_status trimkv_set_horizon(trimkv_t* h, int horizon, void* stream) {
     h->cfg.horizon = horizon;
     launch_rehorizon(h->cv, horizon, (cudaStream_t)stream);
     CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_set_test_hooks(trimkv_t* h, int flags) {
+    if (flags & ~(TRIMKV_TEST_DISTRUST_SAMPLE | TRIMKV_TEST_ATTENTION_NO_COPY)) return fail(TRIMKV_E_ARG, "unknown test hook");
+    CUDA_TRY(cudaDeviceSynchronize());
+    if (h) h->test_hooks = flags;
+    else tkv::g_test_hooks.store(flags, std::memory_order_relaxed);
     return TRIMKV_OK;
 }
 

@@ -42,16 +42,25 @@ def _step_inputs(w, bank, seed, token):
 
 # context: enough tokens to fill the budget (the cache is then in the same state class as after the full prompt,
 # and the set-up stays short); the llama shape also runs its full 32K prompt
-CASES = [("llama8b_32k", 32768, 0), ("qwen_vl_16k", 4096, 2), ("stress_128k", 9216, 0), ("multiturn", 2048, 5)]
+# skew > 0: per-(layer, head) gate-logit offsets N(0, skew) (through b2, as `bench.py --skew` applies them): retention then
+# differs by orders of magnitude between heads, pool lengths run from 0 to tens of thousands of entries, long pools are
+# cut into many work items and the attention kernel's in-kernel merge is live
+CASES = [("llama8b_32k", 32768, 0, 0.0), ("qwen_vl_16k", 4096, 2, 0.0), ("stress_128k", 9216, 0, 0.0),
+         ("multiturn", 2048, 5, 0.0), ("llama8b_32k", 32768, 3, 3.0)]
 
 
-@pytest.mark.parametrize("name,context,seq", CASES)
-def test_full_size_step_matches_oracle_on_samples(name, context, seq):
+@pytest.mark.parametrize("name,context,seq,skew", CASES)
+def test_full_size_step_matches_oracle_on_samples(name, context, seq, skew):
     w = workloads.WORKLOADS[name]
     seed = 0
     LH = w.layers * w.kv_heads
     cache = binding.TrimKV.from_workload(w)
     per_layer, w_g = workloads.gate_params(w, seed, device=DEV)
+    if skew > 0:
+        off = workloads.head_logit_offsets(w, seed, skew, device=DEV)
+        wn = w_g / (w_g * w_g).sum()
+        per_layer = [(W1, b1, W2, (b2 + off[l][:, None] * wn[None, :]).contiguous())
+                     for l, (W1, b1, W2, b2) in enumerate(per_layer)]
     for l, p in enumerate(per_layer):
         cache.set_gate(l, *p)
     cache.set_shared_projection(w_g, w.b_g)
@@ -68,6 +77,11 @@ def test_full_size_step_matches_oracle_on_samples(name, context, seq):
 
     # ---- state of the sampled sequence before the step
     lens = cache.lengths()[seq].numpy()
+    if skew > 0:                                         # ragged pools: also the longest and the shortest non-empty pool
+        assert lens.max() > 8 * max(int(lens[lens > 0].min()), 1) and lens.max() > 16384
+        longest = np.unravel_index(np.argmax(lens), lens.shape)
+        shortest = np.unravel_index(np.argmin(np.where(lens > 0, lens, 1 << 30)), lens.shape)
+        sample_pools += [(int(longest[0]), int(longest[1])), (int(shortest[0]), int(shortest[1]))]
     cap = int(lens.max()) + 2
     before = {}
     for l in range(w.layers):
@@ -212,3 +226,86 @@ def test_select_topk_properties_at_sweep_sizes(log2n, kind):
         n_kept_tie = int(kept_tie.sum().item())
         assert bool(kept_tie[:n_kept_tie].all().item()) and not bool(kept_tie[n_kept_tie:].any().item())
         del keep, tie, idx, kept_tie
+
+
+def test_multi_turn_flow_at_full_shape():
+    """The multi-turn workload at its full shape (32 layers, 8 KV heads, batch 32, budget 524,288 entries per sequence),
+    two turns: each turn appends 2048 user tokens in 512-token chunks with an eviction round after every chunk (up to
+    131,072 evictions per sequence and round) and then decodes 8 tokens through trimkv_decode_step_all; positions and
+    the budget persist across the turns.  One sampled sequence is mirrored by the oracle through the whole flow (fed
+    the device's fp32 retention terms): pool lengths after every eviction round, the kept set of every one of its pools
+    after each turn's prompt and each turn's decode steps, bit for bit; the budget invariant for every sequence; and
+    the attention output of sampled pools in each turn's last decode step."""
+    w = workloads.WORKLOADS["multiturn"]
+    seed, seq = 0, 11
+    LH = w.layers * w.kv_heads
+    cache = binding.TrimKV.from_workload(w)
+    per_layer, w_g = workloads.gate_params(w, seed, device=DEV)
+    for l, p in enumerate(per_layer):
+        cache.set_gate(l, *p)
+    cache.set_shared_projection(w_g, w.b_g)
+    bank = workloads.ProjectionBank(w, seed, device=DEV)
+    oc = orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, 0, w.horizon)
+    empty = lambda n: np.zeros((n, w.kv_heads, 0))
+    rng = np.random.default_rng(3)
+    g = w.group
+
+    def check_lengths():
+        lens = cache.lengths().numpy()
+        np.testing.assert_array_equal(lens[seq], oc.lengths())
+        want = min(w.budget_entries, oc.tokens[0] * LH)
+        assert (lens.reshape(w.batch, -1).sum(1) == want).all()          # budget invariant, every sequence
+
+    def check_sets():
+        for l in range(w.layers):
+            for h in range(w.kv_heads):
+                want = oc.kept_positions(l, h)
+                got = cache.kept(seq, l, h, len(want) + 2).numpy()
+                np.testing.assert_array_equal(got, want, err_msg=f"kept set differs in pool ({seq},{l},{h})")
+
+    tokens = 0
+    for turn in range(2):
+        for ch in range(w.context // w.chunk):
+            for l in range(w.layers):
+                x = workloads.hidden_states(w, seed, l, tokens, w.chunk, device=DEV)
+                _, k, v = workloads.project_qkv(w, bank, l, x)
+                cache.append(l, k, v, x=x)
+                _, lam, c = cache.gate(l, x)                         # the terms the append computed (same kernels)
+                oc.append(l, empty(w.chunk), empty(w.chunk), lam=to_np(lam[seq]), c=to_np(c[seq]))
+            cache.score_and_evict()
+            oc.score_and_evict()
+            tokens += w.chunk
+            check_lengths()
+        check_sets()
+        for step in range(8):
+            X, K, V, Q = _step_inputs(w, bank, seed, tokens)
+            last = step == 7
+            if last:                                                   # sampled pools before the step, with their rows
+                pools = [(int(rng.integers(w.layers)), int(rng.integers(w.kv_heads))) for _ in range(3)]
+                rows = {}
+                for (l, h) in pools:
+                    n_old = len(oc.kept_positions(l, h))
+                    _, _, _, kk, vv = cache.pool(seq, l, h, n_old + 2, with_kv=True)
+                    rows[(l, h)] = (to_np(kk).astype(np.float64), to_np(vv).astype(np.float64))
+            out = torch.empty_like(Q)
+            cache.decode_step_all(K, V, Q, out, x=X)
+            for l in range(w.layers):
+                _, lam, c = cache.gate(l, X[l][:, None].contiguous())
+                oc.append(l, empty(1), empty(1), lam=to_np(lam[seq]), c=to_np(c[seq]))
+            oc.score_and_evict()
+            tokens += 1
+            check_lengths()
+            if last:
+                for (l, h), (kk, vv) in rows.items():
+                    Kp = np.concatenate([kk, to_np(K[l, seq, h])[None].astype(np.float64)])
+                    Vp = np.concatenate([vv, to_np(V[l, seq, h])[None].astype(np.float64)])
+                    for j in range(h * g, (h + 1) * g):
+                        err = np.abs(to_np(out[l, seq, j]) - orc.attention(to_np(Q[l, seq, j]), Kp, Vp)).max()
+                        assert err <= 2e-2, f"attention error {err} in pool ({seq},{l},{h}), head {j}, turn {turn}"
+        check_sets()
+    # positions kept counting across the turns: the newest kept position is the last token of the second turn
+    assert max(int(oc.kept_positions(l, h).max()) for l in range(w.layers) for h in range(w.kv_heads)
+               if len(oc.kept_positions(l, h))) == tokens
+    assert (cache.select_stats()[:, 0] == 0).all()
+    cache.sync_status()
+    cache.close()

@@ -739,3 +739,111 @@ def test_set_horizon_rescores_stored_entries():
         pair.gpu.set_horizon(65)
     pair.gpu.sync_status()
     pair.close()
+
+
+# ------------------------------------------------------------------------------------------- score rounding contract
+def test_score_rounding_contract_decides_kept_sets():
+    """The score is one fp32 multiply and one fp32 add, each rounded, never fused (Eq. (global_score) in log space).
+    Every sequence holds one pair of entries whose order under that contract differs from their order under a fused
+    multiply-add and under fp64 evaluation, and a budget that keeps exactly one member of the pair: the kept sets equal
+    the oracle's only if the device rounds as the contract says.  The discriminating power of the inputs is asserted
+    here on the host (fused and fp64 evaluations give other sets in every sequence); no kernel is altered."""
+    from util_parity import rounding_contract_case, rounding_contract_kept_sets
+    B, n, L, H = 320, 48, 2, 2
+    lam, c, budget = rounding_contract_case(seed=9, B=B, n=n, L=L, H=H)
+    want = rounding_contract_kept_sets(lam, c, budget, "contract")
+    fused = rounding_contract_kept_sets(lam, c, budget, "fused")
+    fp64 = rounding_contract_kept_sets(lam, c, budget, "fp64")
+    assert all(want[b] != fused[b] and want[b] != fp64[b] for b in range(B))
+    w = workloads.Workload("round", L, H, H, 128, 0, B, budget, "bf16", 0, 0, n)
+    pair = Pair(w, oracle_kv=False)
+    k = torch.zeros(B, n, H, 128, device=DEV, dtype=torch.bfloat16)
+    for l in range(L):
+        pair.append(l, k, k, lam[l], c[l])
+    pair.evict()
+    pair.check_sets()
+    for b in range(B):
+        got = {(l, int(p) - 1, h) for l in range(L) for h in range(H) for p in pair.gpu.kept(b, l, h, n).tolist()}
+        assert got == want[b], f"sequence {b}: the device's kept set is not the contract's"
+    pair.close()
+
+
+def test_bounded_wait_runs_out_and_the_handle_recovers():
+    """A device-side wait that can never be satisfied gives up: under the testing aid the attention kernel issues none
+    of its asynchronous copies (nothing is in flight) and waits with a short limit; it latches E_TIMEOUT and returns.
+    trimkv_sync_status reports it; after trimkv_reset the handle computes the same attention as before."""
+    w = BF16_SMALL.replace(budget_entries=4000, layers=1, batch=2)
+    cache = binding.TrimKV.from_workload(w)
+    g = torch.Generator(device=DEV); g.manual_seed(3)
+    k = torch.randn(w.batch, 150, w.kv_heads, 128, generator=g, device=DEV).to(torch.bfloat16)
+    v = torch.randn(w.batch, 150, w.kv_heads, 128, generator=g, device=DEV).to(torch.bfloat16)
+    q = torch.randn(w.batch, w.q_heads, 128, generator=g, device=DEV).to(torch.bfloat16)
+    lam = -torch.rand(w.batch, 150, w.kv_heads, generator=g, device=DEV) * 0.01
+    cache.append(0, k, v, lam=lam)
+    ref = cache.decode_attention(0, q).clone()
+    cache.sync_status()
+    cache.set_test_hooks(binding.TEST_ATTENTION_NO_COPY)
+    cache.decode_attention(0, q)
+    with pytest.raises(binding.TrimkvError) as e:
+        cache.sync_status()
+    assert e.value.status == binding.E_TIMEOUT
+    cache.set_test_hooks(0)
+    cache.reset()
+    cache.sync_status()                                   # the latch is cleared
+    cache.append(0, k, v, lam=lam)
+    assert torch.equal(cache.decode_attention(0, q), ref)
+    cache.sync_status()
+    cache.close()
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "f32"])
+def test_retention_gated_step_with_a_slot_that_held_zero_retention(kv_dtype):
+    """beta = 0 is legal (lambda = -inf): such entries are evicted first and leave lambda = -inf behind in their freed
+    slots.  The whole-step call writes the new token's K/V into such a slot before its lambda; the retention-gated
+    attention must give the new token the weight beta^0 = 1 whatever the slot still holds."""
+    d = 128 if kv_dtype == "bf16" else 64
+    dt = workloads.torch_dtype(kv_dtype)
+    atol = ATT_ATOL_BF16 if kv_dtype == "bf16" else ATT_ATOL_F32
+    w = workloads.Workload("stale", 1, 2, 8, d, 0, 1, 2 * 4, kv_dtype, 0, 0, 8)
+    pair = Pair(w, retention_bias=True)
+    g = torch.Generator(device=DEV); g.manual_seed(5)
+    k = torch.randn(1, 6, 2, d, generator=g, device=DEV).to(dt)
+    v = torch.randn(1, 6, 2, d, generator=g, device=DEV).to(dt)
+    lam = np.full((1, 6, 2), -0.01, np.float32)
+    lam[:, 4:, :] = -np.inf                                # the two newest tokens: never retained
+    pair.append(0, k, v, lam, oracle_retention(lam, w.horizon))
+    pair.evict()
+    pair.check_sets()
+    assert pair.gpu.lengths().tolist() == [[[4, 4]]]
+    K = torch.randn(1, 1, 2, d, generator=g, device=DEV).to(dt)
+    V = torch.randn(1, 1, 2, d, generator=g, device=DEV).to(dt)
+    Q = torch.randn(1, 1, 8, d, generator=g, device=DEV).to(dt)
+    nl = np.full((1, 1, 2), -0.02, np.float32)
+    out = torch.empty_like(Q)
+    pair.gpu.decode_step_all(K, V, Q, out, lam=torch.from_numpy(nl).to(DEV))
+    pair.gpu.sync_status()
+    pair.orc[0].append(0, to_np(K[0]), to_np(V[0]), lam=nl[0])
+    want = pair.orc[0].decode_attention(0, to_np(Q[0, 0]), retention_bias=True)
+    assert torch.isfinite(out.float()).all()
+    assert np.abs(to_np(out[0, 0]) - want).max() <= atol
+    pair.close()
+
+
+def test_append_beyond_capacity_is_refused_synchronously():
+    """The cache has room for the budget plus one chunk per layer: a further append before an eviction round is refused
+    with E_STATE at once and changes nothing."""
+    cache = binding.TrimKV(16, 2, 1, 64, kv_dtype="f32", max_chunk=4)
+    k = torch.zeros(1, 4, 1, 64, device=DEV)
+    lam = -torch.rand(1, 4, 1, device=DEV)
+    for _ in range(3):                                    # 24 entries = 16 + 4 * 2
+        cache.append(0, k, k, lam=lam)
+        cache.append(1, k, k, lam=lam)
+    with pytest.raises(binding.TrimkvError) as e:
+        cache.append(0, k, k, lam=lam)
+    assert e.value.status == binding.E_STATE
+    assert int(cache.lengths().sum()) == 24
+    cache.score_and_evict()
+    assert int(cache.lengths().sum()) == 16
+    cache.append(0, k, k, lam=lam)                        # room again
+    cache.sync_status()
+    cache.close()

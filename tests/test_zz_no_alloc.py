@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import trimkv_oracle as orc
 from paper_2605_09649_b200 import binding, workloads
 
 pytestmark = pytest.mark.gpu
@@ -57,3 +58,25 @@ def test_static_scratch_selection_edge_sizes_and_limit():
     got, st, want, _ = _both(at, binding.SELECT_STATIC_MAX_N // 8)
     assert st == 0
     np.testing.assert_array_equal(got, want)
+
+
+def test_static_scratch_selection_matches_the_oracle_and_allocates_nothing():
+    """Independent of the sibling entry point: the kept set equals the oracle's full sort (score descending, lower
+    index first among equals), and a warmed-up call leaves the device's free memory where it was."""
+    n = 300_001
+    s = (workloads.selection_scores(n, seed=9, device=DEV) * 8).round() / 8          # heavy ties
+    bits = torch.zeros((n + 63) // 64, dtype=torch.int64, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    binding.select_topk_static(s, n // 3, bits, status)                               # warm-up (first call: set-up)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for k in (n // 3, n - 512, 77):
+        binding.select_topk_static(s, k, bits, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        got = np.unpackbits(bits.cpu().numpy().view(np.uint8), bitorder="little")[:n].astype(bool)
+        z = np.zeros(n, np.int64)
+        want = np.zeros(n, bool)
+        want[orc.select_keep(s.cpu().numpy(), np.arange(n), z, z, k)] = True
+        np.testing.assert_array_equal(got, want)
+    assert torch.cuda.mem_get_info()[0] == free0
