@@ -9,10 +9,14 @@ selection + compaction (trimkv_decode_step_all).  At N = 1 the workload is the L
 its own batch of sequences (independent budgets, no data-path collective): weak scaling.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
+At N = 1 the line also carries `other_workloads`: the other named workloads (vision-language, multi-turn, long-context
+stress) and the standalone selection sweep, each timed the same way with its own clock record.
+`--gpus N` without a torchrun environment starts the N ranks itself (one process per GPU).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -25,9 +29,23 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_mma_kernel launch, from the ncu capture summarised in
-# profiles/attn_mma_kernel_llama8b_cache_at_budget.md (same kernel source as now; set to None when the kernel changes).
-NCU_TRAFFIC_BYTES = {"llama8b_32k": 4315508000 + 2926000}
+ATTENTION_SOURCE = os.path.join(ROOT, "paper_2605_09649_b200", "csrc", "attention.cu")
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "attn_mma_kernel_dram_traffic.txt")
+
+
+def recorded_traffic(workload: str):
+    """DRAM bytes (read + write) of one launch of the dominant kernel, as an ncu capture recorded them, or None.
+    Each record line is `<workload> <sha256 of the kernel's source file> <bytes per launch>`; a record counts only while
+    the source file still hashes to the same value, so a changed kernel reports no stale figure."""
+    try:
+        digest = hashlib.sha256(open(ATTENTION_SOURCE, "rb").read()).hexdigest()
+        for line in open(TRAFFIC_RECORD):
+            f = line.split()
+            if len(f) >= 3 and not line.startswith("#") and f[0] == workload and f[1] == digest:
+                return int(f[2])
+    except OSError:
+        pass
+    return None
 
 METRIC = "decode tokens/s at fixed global KV budget (step time in ms_per_step, % of HBM peak in roofline)"
 UNIT = "tokens/s"
@@ -115,18 +133,19 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------- CPU oracle arm
-def oracle_sample(w, steps, seed=0):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload: ONE sequence whose cache is at its
-    budget (M_global entries spread evenly over the pools, seeded N(0,1) K/V, seeded retention), running `steps`
-    whole decode steps (gate, append, attention over all pools, score + full sort + eviction).  Returns
-    (seconds per step, threads used, description)."""
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_synthetic_state(w, seed=0):
+    """One sequence of the workload with its cache at the budget (M_global entries spread evenly over the pools, seeded
+    N(0,1) K/V rows, seeded retention around the gate's bias) and seeded random-init gates, built on the host.
+    Returns (oracle cache, generator)."""
     import numpy as np
     from oracle import trimkv_oracle as orc
-    try:
-        from threadpoolctl import threadpool_info
-        threads = max([int(t.get("num_threads", 1)) for t in threadpool_info()] + [1])
-    except Exception:
-        threads = 1
     r = np.random.default_rng(seed)
     oc = orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, w.head_dim, w.horizon)
     per_pool = w.budget_entries // (w.layers * w.kv_heads)
@@ -147,59 +166,121 @@ def oracle_sample(w, steps, seed=0):
                        r.standard_normal((w.kv_heads, w.gate_embed, w.gate_hidden)) * 0.02,
                        np.zeros((w.kv_heads, w.gate_embed))))
     oc.set_gate(params, r.standard_normal(w.gate_embed) * 0.02, w.b_g)
+    return oc, r
+
+
+def oracle_synthetic_inputs(w, r, steps):
+    return [(r.standard_normal((w.layers, 1, w.hidden)), r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim)),
+             r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim)), r.standard_normal((w.layers, w.q_heads, w.head_dim)))
+            for _ in range(steps)]
+
+
+def oracle_time_steps(oc, w, inputs, threads):
+    """Runs the oracle, as it stands, through whole decode steps (gate, append, attention over all pools, score + full
+    sort + eviction) with its library routines limited to `threads` threads.  Returns seconds per step."""
+    try:
+        from threadpoolctl import threadpool_limits
+        limit = threadpool_limits(limits=threads)
+    except Exception:
+        limit = None
     times = []
-    for _ in range(steps):
-        x = r.standard_normal((w.layers, 1, w.hidden))
-        k = r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim))
-        v = r.standard_normal((w.layers, 1, w.kv_heads, w.head_dim))
-        q = r.standard_normal((w.layers, w.q_heads, w.head_dim))
-        a = time.perf_counter()
-        for l in range(w.layers):
-            oc.append(l, k[l], v[l], x=x[l])
-            oc.decode_attention(l, q[l])
-        oc.score_and_evict()
-        times.append(time.perf_counter() - a)
-    desc = (f"1 of {w.batch} sequences at budget ({w.budget_entries} entries), {steps} whole decode steps "
+    try:
+        for (x, k, v, q) in inputs:
+            a = time.perf_counter()
+            for l in range(w.layers):
+                oc.append(l, k[l], v[l], x=x[l])
+                oc.decode_attention(l, q[l])
+            oc.score_and_evict()
+            times.append(time.perf_counter() - a)
+    finally:
+        if limit is not None:
+            limit.restore_original_limits()
+    return sum(times) / len(times)
+
+
+def oracle_sample_desc(w, steps, source):
+    return (f"1 of {w.batch} sequences at budget ({w.budget_entries} entries; {source}), {steps} whole decode steps "
             f"(gate+append+attention over all {w.layers * w.kv_heads} pools+score+full sort)")
-    return sum(times) / len(times), threads, desc
 
 
 def run_reference(args, w):
     from paper_2605_09649_b200 import dist_util
     rank, _, world = dist_util.env_world()
     if rank != 0:
-        return
+        return                                   # under torchrun rank 0 alone runs the oracle; the others exit 0
     steps = max(1, min(args.steps, 8))
-    for _ in range(min(args.warmup, 1)):
-        oracle_sample(w, 1)
-    sec, threads, desc = oracle_sample(w, steps)
+    warm = min(args.warmup, 1)
+    cores = host_cores()
+    oc, r = oracle_synthetic_state(w, args.seed)
+    if warm:
+        oracle_time_steps(oc, w, oracle_synthetic_inputs(w, r, warm), cores)
+    sec = oracle_time_steps(oc, w, oracle_synthetic_inputs(w, r, steps), cores)
     value = 1.0 / sec                       # one sequence advances one token per oracle step
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded N(0,1) hidden states, K/V, random-init gates)",
         "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
-                   "head_dim": w.head_dim, "hidden": w.hidden, "batch": w.batch, "budget_entries_per_seq": w.budget_entries,
-                   "context": w.context},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+                   "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
+                   "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk, "b_g": w.b_g},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": oracle_sample_desc(w, steps, "state drawn on the host from the seed")},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
 
 
+def oracle_beside_gpu(cache, w, per_layer, w_g, step_inputs, first_token, seq=0):
+    """The CPU baseline of the CUDA arm: the oracle on the SAME tensors.  Sequence `seq` of the GPU run is read back
+    from the device (every pool: positions, fp32 retention terms, K/V rows) after the timed steps, and the oracle then
+    runs whole decode steps on the GPU run's next seeded step inputs, once with one thread and once with all host
+    cores.  Returns the cpu_baseline object."""
+    import numpy as np
+    from oracle import trimkv_oracle as orc
+    f64 = lambda t: t.detach().float().cpu().numpy().astype(np.float64)
+    oc = orc.OracleCache(w.budget_entries, w.layers, w.kv_heads, w.q_heads, w.head_dim, w.horizon)
+    lens = cache.lengths()[seq]
+    cap = int(lens.max()) + 1
+    for l in range(w.layers):
+        for h in range(w.kv_heads):
+            pos, lam, c, k, v = cache.pool(seq, l, h, cap, with_kv=True)
+            order = np.argsort(pos.numpy(), kind="stable")
+            oc.pos[l][h] = pos.numpy().astype(np.int64)[order]
+            oc.lam[l][h] = lam.numpy()[order]
+            oc.c[l][h] = c.numpy()[order]
+            oc.K[l][h] = f64(k)[order]
+            oc.V[l][h] = f64(v)[order]
+        oc.tokens[l] = first_token
+    oc.set_gate([tuple(f64(t) for t in p) for p in per_layer], f64(w_g), w.b_g)
+    big = w.budget_entries > 100000
+    n1, nc = (2, 3) if big else (4, 8)
+    ins = []
+    for i in range(n1 + nc):
+        X, Kt, Vt, Q = step_inputs(i)
+        ins.append((f64(X[:, seq])[:, None], f64(Kt[:, seq])[:, None], f64(Vt[:, seq])[:, None], f64(Q[:, seq])))
+    cores = host_cores()
+    sec1 = oracle_time_steps(oc, w, ins[:n1], 1)
+    secc = oracle_time_steps(oc, w, ins[n1:], cores)
+    return {"value": 1.0 / secc, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": oracle_sample_desc(w, nc, f"sequence {seq} of the GPU run read back from the device, then the GPU run's "
+                                                "next seeded step inputs"),
+            "one_thread": {"value": 1.0 / sec1, "unit": UNIT, "cores": 1, "steps": n1}}
+
+
 # ------------------------------------------------------------------------------------------------- CUDA arm
-def run_ours(args, w):
+def measure_workload(args, w, K, W, rank, world, local_rank, main):
+    """Builds the workload's cache on this rank's GPU (chunked prefill with evictions, earlier turns of a dialogue), then
+    times K whole decode steps after W warm-up steps (device-resident inputs; CUDA events; barrier on both sides), the
+    per-phase times with the phases serialised, and the end-to-end form with host buffers.  main: the headline
+    workload (per-phase detail, CPU baseline); otherwise a compact record is enough."""
     import torch
     from paper_2605_09649_b200 import binding, dist_util, workloads
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    rank, local_rank, world = dist_util.init("nccl") if int(os.environ.get("WORLD_SIZE", "1")) > 1 else (0, 0, 1)
-    torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    seed = args.seed + 1000 * rank                      # every rank owns different sequences
-    K, W = args.steps, args.warmup
+    # weak scaling: the job holds world x batch independent sequences; this rank owns a contiguous block of them
+    seq_lo, seq_hi = workloads.shard_sequences(world * w.batch, rank, world)
+    seed = args.seed + 1000 * (seq_lo // w.batch)       # every rank draws different sequences
 
     per_pool = w.budget_entries // (w.layers * w.kv_heads) if args.fixed_budget else 0
     cache = binding.TrimKV.from_workload(w, retention_bias=args.retention_bias, per_pool_budget=per_pool)
@@ -298,9 +379,12 @@ def run_ours(args, w):
     out = torch.empty_like(inputs[0][3])
     torch.cuda.synchronize()
 
+    done_steps = [0]                             # decode steps this cache has taken since the prefill
+
     def step(i):
         X, Kt, Vt, Q = inputs[i % NSETS]
         cache.decode_step_all(Kt, Vt, Q, out, x=X)
+        done_steps[0] += 1
 
     for i in range(W):
         step(i)
@@ -324,13 +408,19 @@ def run_ours(args, w):
     ms_total = e0.elapsed_time(e1)
     live = cache.profile_read()["attn_main"]
     cache.profile(False)
+    if rank == 0:                            # a short timed region: keep the GPU under the same load until nvidia-smi has sampled it
+        t_load = time.perf_counter()
+        while K * ms_total / max(K, 1) < 600.0 and time.perf_counter() - t_load < 0.6 - ms_total * 1e-3:
+            for i in range(16):
+                step(W + K + i)
+            torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     cache.sync_status()
     ms_step = dist_util.max_over_ranks(ms_total / K, device=dev)
     tokens_per_step = dist_util.sum_over_ranks(w.batch, device=dev)
     value = tokens_per_step / (ms_step * 1e-3)
 
-    # ---- per-phase device time over K more steps with the phases run back to back on one stream (no overlap), CUDA
+    # ---- per-phase device time over more steps with the phases run back to back on one stream (no overlap), CUDA
     # events around each phase: what each kernel takes when it has the memory system to itself
     KP = min(K, 32)
     cache.set_overlap(False)
@@ -347,28 +437,48 @@ def run_ours(args, w):
     host_out = torch.empty_like(out, device="cpu").pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in host_in[0])
     d2h = host_out.numel() * host_out.element_size()
+
+    def e2e_loop(n):
+        for i in range(n):
+            hX, hK, hV, hQ = host_in[i % len(host_in)]
+            cache.decode_step_all_host(hK, hV, hQ, host_out, x=hX)   # the C-ABI call with host buffers: copies inside
+            torch.cuda.current_stream().synchronize()         # the caller needs the step's result before the next token
+            done_steps[0] += 1
+
+    e2e_loop(2)
     torch.cuda.synchronize()
     dist_util.barrier()
     e0.record()
-    for i in range(KE):
-        hX, hK, hV, hQ = host_in[i % len(host_in)]
-        cache.decode_step_all_host(hK, hV, hQ, host_out, x=hX)   # the C-ABI call with host buffers: copies inside
-        torch.cuda.current_stream().synchronize()         # the caller needs the step's result before the next token
+    e2e_loop(KE)
     e1.record()
     torch.cuda.synchronize()
     dist_util.barrier()
     e2e_ms = dist_util.max_over_ranks(e0.elapsed_time(e1) / KE, device=dev)
     e2e_value = tokens_per_step / (e2e_ms * 1e-3)
+    # where the end-to-end step's time goes: the same loop with events around the copies and the kernels (the events
+    # themselves cost a little, so this loop is not the one that is reported as the end-to-end number)
+    cache.profile(True)
+    t0 = time.perf_counter()
+    e2e_loop(KE)
+    torch.cuda.synchronize()
+    wall_prof = (time.perf_counter() - t0) / KE * 1e3
+    eph = cache.profile_read()
+    cache.profile(False)
+    per = lambda name: eph[name][0] / max(eph[name][1], 1)
+    breakdown = {"h2d_kvq_ms": per("h2d_kvq"), "h2d_x_ms": per("h2d_x"), "append_ms": per("append"), "attention_ms": per("attn_main"),
+                 "gate_ms": per("gate"), "select_ms": per("select"), "compact_ms": per("compact"), "d2h_out_ms": per("d2h_out"),
+                 "what": "device time of each part of trimkv_decode_step_all_host (gate, x copy and selection run beside the "
+                         "attention kernel); critical path = h2d_kvq + append + attention + compact + d2h_out; the rest of "
+                         "ms_per_step is host launch and synchronisation latency"}
+    breakdown["critical_path_ms"] = sum(breakdown[k] for k in ("h2d_kvq_ms", "append_ms", "attention_ms", "compact_ms", "d2h_out_ms"))
+    breakdown["host_latency_ms"] = max(0.0, e2e_ms - breakdown["critical_path_ms"])
+    breakdown["wall_ms_per_step_with_events"] = wall_prof
     cache.sync_status()
     lens = cache.lengths()
     assert int(lens[0].sum()) == min(w.budget_entries, entries), "budget invariant violated"
     assert per_pool == 0 or int(lens.max()) <= per_pool
 
-    if rank != 0:
-        cache.close()
-        return
     peak, peak_kind = load_peaks()
-    tpk = load_tensor_peaks()
     ab = algorithmic_bytes(w, entries + w.layers * w.kv_heads)
     if args.retention_bias:                                        # lambda and position of every entry ride along
         extra_b = w.batch * (entries + w.layers * w.kv_heads) * 8
@@ -378,24 +488,55 @@ def run_ours(args, w):
     iso_ms = phases["attn_main"][0] / max(phases["attn_main"][1], 1)
     iso_gbs = ab["kv"] / (iso_ms * 1e-3) / 1e9 if iso_ms > 0 else 0.0
     step_gbs = ab["total"] / (ms_step * 1e-3) / 1e9
-    cpu = None
-    if not args.no_cpu_baseline:
-        sec, threads, desc = oracle_sample(w, 3 if w.budget_entries > 100000 else 8)
-        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+    res = {"w": w, "K": K, "W": W, "value": value, "ms_step": ms_step, "launches": launches, "clocks": clocks, "entries": entries,
+           "lens_min_max": [int(lens[0].min()), int(lens[0].max())], "t_setup": t_setup, "tokens_seen": tokens_seen,
+           "prefill_ms": prefill_ms, "prefill_chunks": prefill_chunks, "attn_stats": attn_stats,
+           "early_decode": early_decode_ms / early_decode_steps if early_decode_steps else None,
+           "ab": ab, "attn_ms_per": attn_ms_per, "achieved": achieved, "iso_ms": iso_ms, "iso_gbs": iso_gbs, "step_gbs": step_gbs,
+           "phases": {k: v[0] / KP for k, v in phases.items() if v[1]}, "peak": peak, "peak_kind": peak_kind,
+           "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "steps": KE, "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "breakdown": breakdown},
+           "per_pool": per_pool, "seqs": [seq_lo, seq_hi], "cpu": None}
+    if main and rank == 0 and not args.no_cpu_baseline:
+        res["cpu"] = oracle_beside_gpu(cache, w, per_layer, w_g, lambda i: step_inputs(done_steps[0] + i),
+                                       tokens_seen + done_steps[0])
+    cache.close()
+    del cache, inputs, host_in
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args, w):
+    import torch
+    from paper_2605_09649_b200 import dist_util
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = dist_util.init("nccl") if int(os.environ.get("WORLD_SIZE", "1")) > 1 else (0, 0, 1)
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank} needs CUDA device {local_rank}; {torch.cuda.device_count()} present")
+    torch.cuda.set_device(local_rank)
+    K, W = args.steps, args.warmup
+    r = measure_workload(args, w, K, W, rank, world, local_rank, main=True)
+    if rank != 0:
+        return
+    tpk = load_tensor_peaks()
+    ab, peak, peak_kind, attn_stats = r["ab"], r["peak"], r["peak_kind"], r["attn_stats"]
+    default_config = args.skew == 0 and args.context is None and args.layers is None and not args.retention_bias
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "f32",
+        "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": r["ms_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "f32",
         "data": "synthetic (seeded N(0,1) hidden states; K/V/Q from random-init projections; random-init gates)",
         "config": {"workload": w.name, "layers": w.layers, "kv_heads": w.kv_heads, "q_heads": w.q_heads,
                    "head_dim": w.head_dim, "hidden": w.hidden, "batch_per_gpu": w.batch,
                    "budget_entries_per_seq": w.budget_entries, "context": w.context, "prefill_chunk": w.chunk,
-                   "entries_per_seq_during_step": entries + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew, "retention_bias": bool(args.retention_bias), "fixed_per_pool_budget": per_pool,
-                   "pool_len_min_max": [int(lens[0].min()), int(lens[0].max())],
-                   "parallelism": f"sequences sharded over {world} rank(s), no collective",
-                   "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(t_setup, 1),
-                   "turns": w.turns, "tokens_before_timed_region": tokens_seen,
-                   "prefill": {"chunks": prefill_chunks, "ms_per_chunk": prefill_ms / max(prefill_chunks, 1),
-                               "tokens_per_s": w.batch * w.chunk / (prefill_ms / max(prefill_chunks, 1) * 1e-3) if prefill_ms > 0 else None,
+                   "entries_per_seq_during_step": r["entries"] + w.layers * w.kv_heads, "b_g": w.b_g, "skew": args.skew, "retention_bias": bool(args.retention_bias), "fixed_per_pool_budget": r["per_pool"],
+                   "pool_len_min_max": r["lens_min_max"],
+                   "parallelism": f"{world * w.batch} independent sequences sharded over {world} rank(s) (rank 0: {r['seqs']}), no collective",
+                   "l2": "inputs larger than L2 (each step streams the whole cache)", "setup_s": round(r["t_setup"], 1),
+                   "turns": w.turns, "tokens_before_timed_region": r["tokens_seen"],
+                   "prefill": {"chunks": r["prefill_chunks"], "ms_per_chunk": r["prefill_ms"] / max(r["prefill_chunks"], 1),
+                               "tokens_per_s": w.batch * w.chunk / (r["prefill_ms"] / max(r["prefill_chunks"], 1) * 1e-3) if r["prefill_ms"] > 0 else None,
                                "what": "gate + append of every layer and one eviction per chunk" +
                                        (", with the chunk's causal attention" if args.prefill_attention else " (no chunk attention)"),
                                "chunk_attention": None if not args.prefill_attention else {
@@ -409,41 +550,64 @@ def run_ours(args, w):
                                    "frac_of_sustained": (attn_stats["last_flops"] / (attn_stats["last_ms"] * 1e-3) / 1e12 / tpk["sustained"])
                                                         if attn_stats["last_ms"] > 0 else None,
                                    "flops": "causal: 4 d per (query head, visible entry); masked tile parts not counted"}},
-                   "earlier_turn_decode_ms_per_step": early_decode_ms / early_decode_steps if early_decode_steps else None},
-        "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name) if args.skew == 0 and args.context is None and args.layers is None else None,
-                     "algorithmic_bytes_per_launch": ab["kv"], "avg_launch_ms": attn_ms_per,
+                   "earlier_turn_decode_ms_per_step": r["early_decode"]},
+        "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": r["achieved"], "peak": peak, "unit": "GB/s",
+                     "frac": r["achieved"] / peak, "peak_kind": f"of {peak_kind} (a copy's read + write rate: a read-only stream can exceed it)",
+                     "traffic": recorded_traffic(w.name) if default_config else None,
+                     "traffic_source": "ncu capture recorded under profiles/, valid while the kernel's source hashes to the recorded value",
+                     "algorithmic_bytes_per_launch": ab["kv"], "avg_launch_ms": r["attn_ms_per"],
                      "note": "timed region: the kernel shares HBM with the gate and selection kernels running beside it",
-                     "alone": {"avg_launch_ms": iso_ms, "achieved": iso_gbs, "frac": iso_gbs / peak},
-                     "step": {"algorithmic_bytes": ab, "achieved_gbs": step_gbs, "frac_of_peak": step_gbs / peak,
-                              "frac_of_8tbs_nominal": step_gbs / 8000.0},
-                     "phase_ms_per_step_serial": {k: v[0] / KP for k, v in phases.items() if v[1]}},
-        "cpu_baseline": cpu,
-        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "steps": KE, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches,
-        "clocks": clocks,
+                     "alone": {"avg_launch_ms": r["iso_ms"], "achieved": r["iso_gbs"], "frac": r["iso_gbs"] / peak},
+                     "step": {"algorithmic_bytes": ab, "achieved_gbs": r["step_gbs"], "frac_of_peak": r["step_gbs"] / peak,
+                              "frac_of_8tbs_nominal": r["step_gbs"] / 8000.0},
+                     "phase_ms_per_step_serial": r["phases"]},
+        "cpu_baseline": r["cpu"],
+        "e2e": r["e2e"],
+        "gpu_launches": r["launches"],
+        "clocks": r["clocks"],
     }
+    if world == 1 and args.workload == "llama8b_32k" and default_config and not args.no_other_workloads:
+        line["other_workloads"] = other_workloads(args)
     print(json.dumps(line), flush=True)
-    cache.close()
+
+
+def other_workloads(args):
+    """The other named workloads at their full shapes and the standalone selection sweep, each timed like the headline
+    workload (device-resident inputs, CUDA events, its own clock record): compact records for the one JSON line."""
+    from paper_2605_09649_b200 import workloads
+    out = {}
+    for name in ("qwen_vl_16k", "stress_128k", "multiturn"):
+        w = workloads.WORKLOADS[name]
+        r = measure_workload(args, w, 32, 3, 0, 1, 0, main=False)
+        out[name] = {"ms_per_step": r["ms_step"], "tokens_per_s": r["value"], "steps": r["K"], "warmup": r["W"],
+                     "batch": w.batch, "entries_per_seq_during_step": r["entries"] + w.layers * w.kv_heads,
+                     "algorithmic_bytes": r["ab"], "step_gbs": r["step_gbs"], "frac_of_measured_hbm": r["step_gbs"] / r["peak"],
+                     "frac_of_8tbs_nominal": r["step_gbs"] / 8000.0,
+                     "attention_kernel": {"avg_launch_ms": r["attn_ms_per"], "achieved_gbs": r["achieved"], "frac": r["achieved"] / r["peak"]},
+                     "e2e_ms_per_step": r["e2e"]["ms_per_step"], "e2e_tokens_per_s": r["e2e"]["value"],
+                     "gpu_launches": r["launches"], "clocks": r["clocks"], "setup_s": round(r["t_setup"], 1),
+                     "earlier_turn_decode_ms_per_step": r["early_decode"]}
+    rows, clocks = select_sweep_rows(args, (20, 24, 28), 5, 3)
+    out["select_sweep"] = {"rows": rows, "clocks": clocks, "l2": "flushed between timed calls",
+                           "what": "trimkv_select_topk over n fp32 scores uniform in [-8, 0]; gbs counts one pass of 4 n bytes per call"}
+    return out
 
 
 # ------------------------------------------------------------------------------------------------- selection sweep
-def run_select_sweep(args):
-    """Standalone global selection over flat fp32 score arrays (uniform in [-8, 0]), N = 2^20 .. 2^28, timed alone.
-    Reported per (N, k): milliseconds per call and GB/s of score bytes (4 N) per call.  One JSON line."""
+def select_sweep_rows(args, exps, K, W):
+    """Times trimkv_select_topk over flat fp32 score arrays (uniform in [-8, 0]) of 2^p scores for p in exps, k in
+    {n/8, n/2, n - 512}: median of K calls after W warm-up calls, L2 flushed before each timed call.  Returns
+    (rows, clock record)."""
     import numpy as np
     import torch
     from paper_2605_09649_b200 import binding, workloads
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the selection has no CPU fallback")
-    dev = "cuda:0"
-    torch.cuda.set_device(0)
-    peak, peak_kind = load_peaks()
-    K, W = min(max(args.steps, 1), 10), max(args.warmup, 3)
+    dev = f"cuda:{torch.cuda.current_device()}"
+    peak, _ = load_peaks()
     flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev)            # larger than L2
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     rows = []
-    for p in range(args.sweep_min, args.sweep_max + 1):
+    for p in exps:
         n = 1 << p
         s = workloads.selection_scores(n, seed=args.seed, device=dev)
         bits = torch.empty((n + 63) // 64, dtype=torch.int64, device=dev)
@@ -453,6 +617,7 @@ def run_select_sweep(args):
             for _ in range(W):
                 binding.select_topk(s, k, bits, ws, status)
             ms = []
+            launches0 = binding.kernel_launches()
             for _ in range(K):
                 flush.zero_()                                                 # L2 flush between timed calls
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -463,17 +628,54 @@ def run_select_sweep(args):
                 ms.append(e0.elapsed_time(e1))
             assert int(status.item()) == 0
             m = float(np.median(ms))
-            rows.append({"n": n, "k_keep": k, "ms": m, "gbs": 4.0 * n / (m * 1e-3) / 1e9})
+            gbs = 4.0 * n / (m * 1e-3) / 1e9
+            rows.append({"n": n, "k_keep": k, "ms": m, "gbs": gbs, "frac_of_measured_hbm": gbs / peak,
+                         "launches_per_call": (binding.kernel_launches() - launches0) // K})
         del s, bits, ws
+    torch.cuda.synchronize()
+    return rows, sampler.stop()
+
+
+def run_select_sweep(args):
+    """Standalone global selection, N = 2^sweep_min .. 2^sweep_max, timed alone.  One JSON line."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the selection has no CPU fallback")
+    torch.cuda.set_device(0)
+    peak, peak_kind = load_peaks()
+    K, W = min(max(args.steps, 1), 10), max(args.warmup, 3)
+    rows, clocks = select_sweep_rows(args, range(args.sweep_min, args.sweep_max + 1), K, W)
     best = max(r["gbs"] for r in rows if r["n"] == rows[-1]["n"])
     line = {"metric": "standalone global selection, GB/s of score bytes per call", "unit": "GB/s", "value": best, "n_gpus": 1,
             "steps": K, "warmup": W, "higher_is_better": True, "dtype": "f32", "data": "synthetic (uniform log-retention in [-8, 0])",
             "config": {"workload": "select_sweep", "n": [1 << args.sweep_min, 1 << args.sweep_max], "l2": "flushed between timed calls"},
-            "roofline": {"bound": "hbm", "kernel": "hist_kernel + filter_kernel", "achieved": best, "peak": peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": "flat selection (whole call)", "achieved": best, "peak": peak, "unit": "GB/s",
                          "frac": best / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
-                         "note": "achieved counts ONE pass of 4 N bytes per call; the method reads the scores 2-3 times"},
-            "sweep": rows}
+                         "note": "achieved counts ONE pass of 4 N bytes per call"},
+            "sweep": rows, "clocks": clocks}
     print(json.dumps(line), flush=True)
+
+
+def spawn_ranks(args):
+    """`--gpus N` outside a torchrun environment: start the N ranks here, one process per GPU (torch.distributed.run on
+    this node, rendezvous on 127.0.0.1).  Returns the launcher's exit code."""
+    import socket
+    import torch
+    have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+    if have < args.gpus:
+        sys.stderr.write(f"bench.py --gpus {args.gpus}: needs {args.gpus} CUDA devices, found {have}\n")
+        return 2
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")                   # the communicator's set-up lines, on stderr: stdout carries the JSON line
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env, cwd=ROOT)
 
 
 def main():
@@ -496,12 +698,21 @@ def main():
     ap.add_argument("--layers", type=int, default=None,
                     help="override the layer count, budget scaled with it (development and small profiling captures only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="leave out the other named workloads and the selection sweep (they add about half a minute)")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
     ap.add_argument("--sweep-max", type=int, default=28)
     ap.add_argument("--sweep-min", type=int, default=20)
     args = ap.parse_args()
     if args.select_sweep:
         return run_select_sweep(args)
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be at least 1")
+    in_torchrun = "WORLD_SIZE" in os.environ and "RANK" in os.environ
+    if in_torchrun and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={os.environ['WORLD_SIZE']}")
+    if args.impl == "ours" and args.gpus > 1 and not in_torchrun:
+        sys.exit(spawn_ranks(args))
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2605_09649_b200 import workloads
     w = workloads.WORKLOADS[args.workload]

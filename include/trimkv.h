@@ -199,8 +199,10 @@ TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);
  * decode_attention, decode_step_all and score_and_evict).  trimkv_profile(h, 1) starts recording,
  * trimkv_profile(h, 0) stops; both synchronise and discard earlier records.  trimkv_profile_read
  * synchronises, writes to host ms[8] the summed milliseconds and to count[8] the number of recorded
- * intervals per phase {0 gate, 1 append, 2 unused, 3 attention kernel, 4 unused, 5 score+select, 6 compact,
- * 7 unused}, and clears the records.  Phases that run on different internal streams overlap in time. */
+ * intervals per phase {0 gate, 1 append, 2 host-to-device copies of K, V and q (host-buffer entry point), 3 attention
+ * kernel, 4 device-to-host copy of the output (host-buffer entry point), 5 score+select, 6 compact, 7 host-to-device
+ * copy of x or lambda (host-buffer entry point)}, and clears the records.  Phases that run on different internal
+ * streams overlap in time. */
 /* enable = 2 records the attention main kernel alone (two events per call: cheap enough for a timed run). */
 TRIMKV_API trimkv_status trimkv_profile(trimkv_t* h, int enable);
 TRIMKV_API trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host);

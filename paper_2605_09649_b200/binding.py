@@ -246,7 +246,7 @@ class TrimKV:
     def sync_status(self):
         _check(lib().trimkv_sync_status(self._h))
 
-    PHASES = ["gate", "append", "attn_plan", "attn_main", "attn_merge", "select", "compact"]
+    PHASES = ["gate", "append", "h2d_kvq", "attn_main", "d2h_out", "select", "compact", "h2d_x"]
 
     def profile(self, enable):
         """False/0 off, True/1 every phase, 2 the attention kernel alone."""

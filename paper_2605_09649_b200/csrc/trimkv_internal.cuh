@@ -196,8 +196,8 @@ struct AttnBuffers {
 };
 
 // Optional per-phase timing: mark(phase, 0) before and mark(phase, 1) after a phase's launches.
-enum Phase { PH_GATE = 0, PH_APPEND = 1, PH_ATTN_PLAN = 2, PH_ATTN_MAIN = 3, PH_ATTN_MERGE = 4, PH_SELECT = 5,
-             PH_COMPACT = 6, PH_COUNT = 8 };
+enum Phase { PH_GATE = 0, PH_APPEND = 1, PH_H2D = 2, PH_ATTN_MAIN = 3, PH_D2H = 4, PH_SELECT = 5,
+             PH_COMPACT = 6, PH_H2D_SIDE = 7, PH_COUNT = 8 };
 struct PhaseMarker {
     virtual void mark(int phase, int end, cudaStream_t st) = 0;
     virtual ~PhaseMarker() {}

@@ -606,11 +606,15 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     }
     if (host) {
         const size_t kvb = (size_t)h->L * h->B * h->H * h->d * h->elt, qb = (size_t)h->L * h->B * h->Hq * h->d * h->elt;
+        if (h->prof.on) h->prof.mark(PH_H2D, 0, fs);
         CUDA_TRY(cudaMemcpyAsync(h->st_k, host->k, kvb, cudaMemcpyHostToDevice, fs));
         CUDA_TRY(cudaMemcpyAsync(h->st_v, host->v, kvb, cudaMemcpyHostToDevice, fs));
         CUDA_TRY(cudaMemcpyAsync(h->st_q, host->q, qb, cudaMemcpyHostToDevice, fs));
+        if (h->prof.on) h->prof.mark(PH_H2D, 1, fs);
+        if (h->prof.on) h->prof.mark(PH_H2D_SIDE, 0, sd);
         if (host->x) CUDA_TRY(cudaMemcpyAsync(h->st_x, host->x, (size_t)h->L * h->B * h->D * 4, cudaMemcpyHostToDevice, sd));
         else CUDA_TRY(cudaMemcpyAsync(h->st_x, host->lambda, (size_t)h->L * h->B * h->H * 4, cudaMemcpyHostToDevice, sd));
+        if (h->prof.on) h->prof.mark(PH_H2D_SIDE, 1, sd);
     }
     if (h->prof.on) h->prof.mark(PH_APPEND, 0, fs);
     launch_append(h->cv, 0, h->L, 1, t, nullptr, nullptr, h->cfg.horizon, k, v, APPEND_KV, fs);
@@ -661,7 +665,11 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
         CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_side, 0));
     }
     if (s == TRIMKV_OK && kev > 0) s = compact_impl(h, fs);
-    if (host) CUDA_TRY(cudaMemcpyAsync(host->out, out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, cudaMemcpyDeviceToHost, fs));
+    if (host) {
+        if (h->prof.on) h->prof.mark(PH_D2H, 0, fs);
+        CUDA_TRY(cudaMemcpyAsync(host->out, out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, cudaMemcpyDeviceToHost, fs));
+        if (h->prof.on) h->prof.mark(PH_D2H, 1, fs);
+    }
     if (two) {
         CUDA_TRY(cudaEventRecord(h->ev_done, fs));
         CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));

@@ -37,3 +37,51 @@ def test_cuda_arm_fails_loudly_without_a_gpu():
     p = _run(["--workload", "tiny", "--steps", "1"])
     assert p.returncode != 0
     assert "CUDA" in (p.stderr + p.stdout)
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="needs a machine without a GPU")
+def test_gpus_flag_starts_ranks_itself_and_refuses_without_enough_devices():
+    """`--gpus 2` outside a torchrun environment takes the self-spawn path; with fewer than 2 devices it exits non-zero
+    with a message instead of running one rank and calling it two."""
+    p = _run(["--gpus", "2", "--workload", "tiny", "--steps", "1"])
+    assert p.returncode != 0
+    assert "needs 2 CUDA devices" in p.stderr
+
+
+def test_reference_arm_under_two_ranks_prints_one_line_from_rank_zero():
+    """Launched the way the scaling run launches it (torch.distributed.run, 2 processes, 127.0.0.1): rank 0 alone runs
+    the oracle and prints the line with n_gpus = 2; rank 1 exits 0 without output."""
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--workload", "tiny",
+           "--steps", "1", "--warmup", "0"]
+    p = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
+    assert lines[0]["cpu_baseline"]["cores"] == len(os.sched_getaffinity(0))
+
+
+def test_world_size_must_match_the_gpus_flag():
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "4", "--workload", "tiny"],
+                       cwd=ROOT, capture_output=True, text=True, timeout=120, env=env)
+    assert p.returncode != 0 and "WORLD_SIZE" in (p.stderr + p.stdout)
+
+
+def test_recorded_traffic_counts_only_for_the_recorded_kernel_source(tmp_path, monkeypatch):
+    """The roofline's `traffic` figure comes from a record keyed on the hash of the kernel's source file: a record made
+    for other source text is ignored (null) rather than reported stale."""
+    import hashlib
+    sys.path.insert(0, ROOT)
+    import bench
+    digest = hashlib.sha256(open(bench.ATTENTION_SOURCE, "rb").read()).hexdigest()
+    rec = tmp_path / "traffic.txt"
+    rec.write_text(f"# comment\nllama8b_32k {'0' * 64} 111\nllama8b_32k {digest} 4318434000\n")
+    monkeypatch.setattr(bench, "TRAFFIC_RECORD", str(rec))
+    assert bench.recorded_traffic("llama8b_32k") == 4318434000
+    assert bench.recorded_traffic("qwen_vl_16k") is None
+    rec.write_text(f"llama8b_32k {'0' * 64} 111\n")
+    assert bench.recorded_traffic("llama8b_32k") is None
