@@ -232,7 +232,12 @@ TRIMKV_API int64_t trimkv_kernel_launches(void);
  * uint64 [(n + 63) / 64], bit (i % 64) of word i / 64 set iff score i is kept.  workspace: device
  * scratch of at least trimkv_select_workspace_bytes(n) bytes, 256-byte aligned, contents ignored.
  * NaN scores are not allowed (latched as TRIMKV_E_NONFINITE in the status word).
- * status_out: device int32, set to a trimkv_status by the kernels (may be NULL). */
+ * status_out: device int32, set to a trimkv_status by the kernels (may be NULL).
+ * The scores are read once: a sampled bracket of the threshold, one pass that writes the keep bits and a short list of
+ * keys near the threshold, exact ranking of that list.  If the bracket misses (about one call in 10^4) an exact
+ * multi-pass fallback runs instead; the result is the same either way.  After the call, int64 workspace[64 .. 68)
+ * (byte offset 512) holds counters for tests and tuning: {fallback taken: 0 none, 1 exact over the candidate list,
+ * 2 exact over all scores; keys in the sampled bracket; keys ranked exactly; keys sampled}. */
 TRIMKV_API size_t trimkv_select_workspace_bytes(int64_t n);
 TRIMKV_API trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
                                  size_t workspace_bytes, int32_t* status_out, void* stream);
@@ -247,14 +252,16 @@ TRIMKV_API trimkv_status trimkv_select_topk(const float* scores, int64_t n, int6
  * cudaMalloc, cudaFree or any other allocating routine.  The caller still passes scores, keep_bits
  * and status_out (device memory, as for trimkv_select_topk).
  *   - Limit: n <= TRIMKV_SELECT_STATIC_MAX_N scores; a larger n is refused with
- *     TRIMKV_E_UNSUPPORTED and a message in trimkv_last_error.  The array takes about 274 KB of
+ *     TRIMKV_E_UNSUPPORTED and a message in trimkv_last_error.  The array takes about 2.4 MB of
  *     device memory on every GPU that loads the library, until the process exits.
- *   - The first call on each device looks up the array's device address (with that device current);
- *     make that first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current;
+ *     the CUDA runtime may load the library's device code at that moment, which is the driver's
+ *     business, not an allocation of this call); make that first call outside any stream capture.
+ *     The address is cached per device; after a cudaDeviceReset it is looked up again.
  *   - All calls share the one array, which keeps whatever the last call left in it; each call
  *     clears, on `stream`, the part that must start at zero.  Two calls whose GPU work may overlap
  *     (different streams, or different threads or handles on one device) race on it: serialise them. */
-#define TRIMKV_SELECT_STATIC_MAX_N (1 << 24)
+#define TRIMKV_SELECT_STATIC_MAX_N (1 << 22)
 TRIMKV_API trimkv_status trimkv_select_topk_static(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits,
                                         int32_t* status_out, void* stream);
 

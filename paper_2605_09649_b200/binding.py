@@ -328,7 +328,7 @@ def select_topk(scores: torch.Tensor, k_keep: int, keep_bits: Optional[torch.Ten
     return keep_bits, status
 
 
-SELECT_STATIC_MAX_N = 1 << 24
+SELECT_STATIC_MAX_N = 1 << 22
 
 
 def select_topk_static(scores: torch.Tensor, k_keep: int, keep_bits: torch.Tensor, status: torch.Tensor):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtrimkv.so")
-SOURCES = ["trimkv_runtime.cu", "gate.cu", "gate_tc.cu", "cache.cu", "select.cu", "select_static.cu", "attention.cu", "prefill_attention.cu", "prefill_attention_tc.cu"]
+SOURCES = ["trimkv_runtime.cu", "gate.cu", "gate_tc.cu", "cache.cu", "select.cu", "select_flat.cu", "select_static.cu", "attention.cu", "prefill_attention.cu", "prefill_attention_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
@@ -33,7 +33,7 @@ def _stale(target: str, deps) -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu to an object and link libtrimkv.so next to this file.  Returns the library path."""
     nvcc = _nvcc()
-    headers = [os.path.join(CSRC, "trimkv_internal.cuh"), os.path.join(ROOT, "include", "trimkv.h"), __file__]
+    headers = [os.path.join(CSRC, "trimkv_internal.cuh"), os.path.join(CSRC, "async_copy.cuh"), os.path.join(ROOT, "include", "trimkv.h"), __file__]
     objs = []
     procs = []
     for src in SOURCES:

@@ -13,6 +13,7 @@
 // Any other shape / fp32 uses a plain one-warp-per-query-head kernel.
 #include <algorithm>
 
+#include "async_copy.cuh"
 #include "trimkv_internal.cuh"
 
 namespace tkv {
@@ -33,40 +34,8 @@ constexpr int ATT_RING_OFF = ATT_GRP_OFF + (ATT_GROUPS + 1) * 4 + 12;
 constexpr int ATT_META_OFF = (ATT_RING_OFF + ATT_WARPS * ATT_RING * 4 + 127) & ~127;   // per warp and stage: lambda[32], pos[32]
 constexpr int ATT_META_BYTES = 2 * TILE * 4;
 constexpr int ATT_SMEM = ATT_META_OFF + ATT_WARPS * ATT_STAGES * ATT_META_BYTES;
-constexpr unsigned WAIT_LIMIT = 1u << 24;      // bounded mbarrier wait (each try may suspend briefly)
 constexpr unsigned WAIT_LIMIT_TEST = 1u << 8;  // the limit of the testing aid under which no copy is ever issued
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Returns false if the wait gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, unsigned limit = WAIT_LIMIT) {
-    for (unsigned it = 0; it < limit; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])

@@ -10,8 +10,7 @@
 // warp votes) and collects the keys inside it; one CTA per sequence verifies the bracket and ranks the collected
 // keys exactly (radix select on the differing bits).  A bracket that missed (probability below 1e-9) is redone
 // exactly by a single-CTA radix select over the whole sequence.
-// Flat-array path (standalone selection over fp32 scores): shared-memory histogram passes (4094 equal-width bins,
-// first centred on a small sample, then narrowed to the bin that holds the k-th key), filter, exact ranking.
+// (The standalone selection over a flat score array lives in select_flat.cu.)
 // Fixed per-pool budgets: one CTA per pool ranks that pool's keys exactly.
 #include <algorithm>
 
@@ -55,302 +54,6 @@ struct CacheSrc {
         return vm;
     }
 };
-
-struct ArraySrc {
-    static constexpr bool FLAT = true;
-    const float* s;
-    long long n;
-    int32_t* err;
-    __device__ long long pages() const { return (n + PAGE - 1) / PAGE; }
-    __device__ int4 info(int, long long) const { return make_int4(0, 0, PAGE, 0); }
-    __device__ unsigned load4(int, long long p, int e0, const int4&, uint32_t (&sc)[4], uint32_t (&tie)[4]) const {
-        const long long i0 = p * PAGE + e0;
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        unsigned vm = 0;
-        if (i0 + 3 < n) {
-            const float4 f = *reinterpret_cast<const float4*>(s + i0);
-            v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
-            vm = 0xFu;
-        } else {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (i0 + j < n) { v[j] = s[i0 + j]; vm |= 1u << j; }
-        }
-        bool bad = false;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            bad |= (v[j] != v[j]) && (vm & (1u << j));
-            sc[j] = orderable_key(v[j]);
-            tie[j] = (uint32_t)(i0 + j);
-        }
-        if (bad) latch_error(err, TRIMKV_E_NONFINITE);
-        return vm;
-    }
-};
-
-__device__ __forceinline__ u64 compose_key(uint32_t sc, uint32_t tie) { return ((u64)sc << 32) | (u64)(~tie); }
-
-// Float-domain forms of 32-bit key comparisons, for any non-NaN x:
-//   x <  key_float_lt(k)  iff  orderable_key(x) <  k        x <= key_float_le(k)  iff  orderable_key(x) <= k
-// Keys at or below that of -inf / at or above that of +inf (NaN bit patterns) clamp to -inf / +inf.  No float has the
-// key 0x7fffffff (it would be -0, which is folded onto +0): "<" there means "< -0", "<=" means "<= the key before it".
-__device__ __forceinline__ float key_float_lt(uint32_t key) {
-    if (key <= 0x007fffffu) return __uint_as_float(0xff800000u);         // at or below key(-inf)
-    if (key >= 0xff800000u) return __uint_as_float(0x7f800000u);         // at or above key(+inf)
-    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
-}
-__device__ __forceinline__ float key_float_le(uint32_t key) { return key_float_lt(key == 0x7fffffffu ? 0x7ffffffeu : key); }
-
-// ------------------------------------------------------------------ threshold search (one CTA, 256 threads)
-__device__ void threshold_scan(SelState* st, uint32_t* hist_b, long long k, long long n_total, bool last_pass,
-                               unsigned cand_target) {
-    __shared__ u64 warp_tot[8];
-    __shared__ int s_bin;
-    __shared__ u64 s_below;
-    __shared__ unsigned s_cnt;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int PER = NB / 256;
-    uint32_t v[PER];
-    u64 local = 0;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        const int bin = tid * PER + i;
-        v[i] = (bin < NB - 1) ? __ldcg(hist_b + bin) : 0u;
-        local += v[i];
-    }
-    u64 incl = local;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const u64 t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (tid == 0) s_bin = -1;
-    if (lane == 31) warp_tot[warp] = incl;
-    __syncthreads();
-    u64 off = 0, total = 0;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const u64 t = warp_tot[w];
-        if (w < warp) off += t;
-        total += t;
-    }
-    const u64 excl = off + incl - local;
-    const u64 kk = (u64)k;
-    if (kk > excl && kk <= excl + local) {
-        u64 cum = excl;
-#pragma unroll
-        for (int i = 0; i < PER; ++i) {
-            if (kk > cum && kk <= cum + v[i]) { s_bin = tid * PER + i; s_below = cum; s_cnt = v[i]; }
-            cum += v[i];
-        }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < PER; ++i) hist_b[tid * PER + i] = 0u;     // clean for the next pass / call
-    if (tid == 0) {
-        const u64 lo = st->lo;
-        const int shift = st->shift;
-        u64 c_lo, c_hi, below, cnt;
-        if (s_bin == 0) {                       // k-th key lies below the binned range
-            c_lo = 0; c_hi = lo - 1; below = 0; cnt = s_cnt;
-        } else if (s_bin > 0) {
-            c_lo = lo + ((u64)(s_bin - 1) << shift);
-            const u64 width_m1 = (shift >= 64) ? ~0ull : ((1ull << shift) - 1ull);
-            c_hi = (c_lo + width_m1 < c_lo) ? ~0ull : c_lo + width_m1;
-            below = s_below; cnt = s_cnt;
-        } else {                                // above the binned range
-            c_lo = lo + ((u64)REG_BINS << shift);
-            c_hi = ~0ull; below = total; cnt = (u64)n_total - total;
-        }
-        const u64 kmin = __ldcg(&st->kmin), kmax = __ldcg(&st->kmax);   // written by other CTAs' atomics
-        if (c_lo < kmin) c_lo = kmin;           // no key lies in [c_lo, kmin): the count below is unchanged
-        if (c_hi > kmax) c_hi = kmax;
-        st->cand_lo = c_lo;
-        st->cand_hi = c_hi;
-        st->n_below = (long long)below;
-        st->cand_expected = (unsigned)(cnt > 0xffffffffull ? 0xffffffffull : cnt);
-        st->passes += 1;
-        if (cnt <= (u64)cand_target || c_lo >= c_hi || last_pass) {
-            st->resolved = 1;
-        } else {
-            u64 nlo = c_lo;
-            int bits = 64 - __clzll((long long)(c_hi - nlo));
-            int nshift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
-            if (nshift >= 32) {                 // bins then depend on the score word alone: start them on a score boundary
-                nlo &= ~0xffffffffull;
-                bits = 64 - __clzll((long long)(c_hi - nlo));
-                nshift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
-            }
-            st->lo = nlo;
-            st->shift = nshift;
-        }
-        st->kmin = ~0ull;
-        st->kmax = 0ull;
-    }
-}
-
-// ------------------------------------------------------------------ pass 1..n: histogram
-template <class Src>
-__global__ void __launch_bounds__(256)
-hist_kernel(Src src, SelState* __restrict__ sel, uint32_t* __restrict__ hist, unsigned int* __restrict__ done,
-            long long k, long long n_total, int last_pass, unsigned cand_target) {
-    __shared__ uint32_t sh[NB];
-    __shared__ u64 s_min[8], s_max[8];
-    __shared__ int s_last;
-    const int b = blockIdx.y;
-    SelState* st = sel + b;
-    if (st->resolved) return;
-    const u64 lo = st->lo;
-    const int shift = st->shift;
-    for (int i = threadIdx.x; i < NB; i += blockDim.x) sh[i] = 0u;
-    __syncthreads();
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sub = lane >> 4, e0 = (lane & 15) * 4;
-    const long long P = src.pages();
-    const long long chunk = (P + gridDim.x - 1) / gridDim.x;
-    const long long p0 = (long long)blockIdx.x * chunk;
-    const long long p1 = min(P, p0 + chunk);
-
-    u64 kmin = ~0ull, kmax = 0ull;
-    unsigned under = 0;
-    int cur_bin = -1;
-    unsigned cur_cnt = 0;
-    auto tally = [&](const uint32_t (&sc)[4], const uint32_t (&tie)[4], unsigned vm) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (vm & (1u << j)) {
-                const u64 key = compose_key(sc[j], tie[j]);
-                kmin = key < kmin ? key : kmin;
-                kmax = key > kmax ? key : kmax;
-                const int bin = bin_of(key, lo, shift);
-                if (bin == 0) {
-                    ++under;
-                } else if (bin < NB - 1) {
-                    if (bin == cur_bin) {
-                        ++cur_cnt;
-                    } else {
-                        if (cur_cnt) atomicAdd(&sh[cur_bin], cur_cnt);
-                        cur_bin = bin;
-                        cur_cnt = 1;
-                    }
-                }
-            }
-        }
-    };
-    bool fast_done = false;
-    if constexpr (Src::FLAT) {
-        // Flat arrays, bins at least one score step wide and starting on a score boundary: the bin of a key depends on
-        // its 32-bit score word alone.  Grid-stride over 16-byte groups, four groups in flight per thread.
-        if (shift >= 32 && (lo & 0xffffffffull) == 0ull) {
-            const uint32_t lo32 = (uint32_t)(lo >> 32);
-            const int sh32 = shift - 32;
-            // Most scores fall outside the binned range (it brackets the k-th key): two float compares settle those.
-            const u64 end64 = (u64)lo32 + ((u64)REG_BINS << sh32) - 1ull;
-            const float lo_f = key_float_lt(lo32);
-            const float hi_f = end64 >= 0xffffffffull ? __uint_as_float(0x7f800000u) : key_float_le((uint32_t)end64);
-            float fmin_ = __uint_as_float(0x7f800000u), fmax_ = __uint_as_float(0xff800000u);
-            bool bad = false;
-            // Straight-line per score (no divergent branches: with a sixth of the scores inside the range nearly every
-            // warp would run both sides of one anyway): the in-range work is predicated.
-            auto one = [&](float x) {
-                bad |= (x != x);
-                fmin_ = fminf(fmin_, x);
-                fmax_ = fmaxf(fmax_, x);
-                const bool below = x < lo_f;
-                under += below ? 1u : 0u;
-                const uint32_t sc = orderable_key(x);
-                const uint32_t bi = (sc - lo32) >> sh32;
-                if (!below && x <= hi_f && bi < (uint32_t)REG_BINS) atomicAdd(&sh[bi + 1], 1u);
-            };
-            const long long n4 = src.n >> 2;
-            const float4* s4 = reinterpret_cast<const float4*>(src.s);
-            const long long T = (long long)gridDim.x * blockDim.x;
-            long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-            for (; i + 3 * T < n4; i += 4 * T) {                         // four 16-byte groups in flight per thread
-                float4 v[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = __ldg(s4 + i + u * T);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) { one(v[u].x); one(v[u].y); one(v[u].z); one(v[u].w); }
-            }
-            for (; i < n4; i += T) {
-                const float4 v = __ldg(s4 + i);
-                one(v.x); one(v.y); one(v.z); one(v.w);
-            }
-            if (blockIdx.x == 0 && threadIdx.x < (int)(src.n & 3)) one(src.s[(n4 << 2) + threadIdx.x]);
-            if (bad) latch_error(src.err, TRIMKV_E_NONFINITE);
-            if (fmin_ <= fmax_) {
-                kmin = (u64)orderable_key(fmin_) << 32;
-                kmax = ((u64)orderable_key(fmax_) << 32) | 0xffffffffull;
-            }
-            fast_done = true;
-        }
-    }
-    // Each half-warp takes two pages per trip; the page records of the next trip are fetched one trip ahead,
-    // so the metadata loads of a trip depend on nothing that is still in flight.
-    const long long stride = (long long)(blockDim.x >> 5) * 4;
-    long long pp = fast_done ? p1 : p0 + warp * 4;
-    int4 infA = make_int4(-1, 0, 0, 0), infB = infA;
-    if (pp + sub < p1) infA = src.info(b, pp + sub);
-    if (pp + 2 + sub < p1) infB = src.info(b, pp + 2 + sub);
-    for (; pp < p1; pp += stride) {
-        const long long pgA = pp + sub, pgB = pp + 2 + sub, nx = pp + stride;
-        int4 nA = make_int4(-1, 0, 0, 0), nB = nA;
-        if (nx + sub < p1) nA = src.info(b, nx + sub);
-        if (nx + 2 + sub < p1) nB = src.info(b, nx + 2 + sub);
-        uint32_t scA[4], scB[4], tiA[4], tiB[4];
-        unsigned vmA = 0, vmB = 0;
-        if (pgA < p1) vmA = src.load4(b, pgA, e0, infA, scA, tiA);
-        if (pgB < p1) vmB = src.load4(b, pgB, e0, infB, scB, tiB);
-        tally(scA, tiA, vmA);
-        tally(scB, tiB, vmB);
-        infA = nA;
-        infB = nB;
-    }
-    if (cur_cnt) atomicAdd(&sh[cur_bin], cur_cnt);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        under += __shfl_xor_sync(0xffffffffu, under, o);
-        const u64 a = __shfl_xor_sync(0xffffffffu, kmin, o);
-        const u64 c = __shfl_xor_sync(0xffffffffu, kmax, o);
-        kmin = a < kmin ? a : kmin;
-        kmax = c > kmax ? c : kmax;
-    }
-    if (lane == 0) {
-        if (under) atomicAdd(&sh[0], under);
-        s_min[warp] = kmin;
-        s_max[warp] = kmax;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) {
-            kmin = s_min[w] < kmin ? s_min[w] : kmin;
-            kmax = s_max[w] > kmax ? s_max[w] : kmax;
-        }
-        if (kmin <= kmax) {
-            atomicMin(&st->kmin, kmin);
-            atomicMax(&st->kmax, kmax);
-        }
-    }
-    uint32_t* hb = hist + (size_t)b * NB;
-    for (int i = threadIdx.x; i < NB - 1; i += blockDim.x) {
-        const uint32_t v = sh[i];
-        if (v) atomicAdd(hb + i, v);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned ticket = atomicAdd(done + b, 1u);
-        s_last = (ticket == gridDim.x - 1);
-        if (s_last) done[b] = 0u;
-    }
-    __syncthreads();
-    if (s_last) {
-        __threadfence();
-        threshold_scan(st, hb, k, n_total, last_pass != 0, cand_target);
-    }
-}
 
 // ------------------------------------------------------------------ filter: evict masks + candidates
 // COUNT_BELOW: also count the keys below the candidate range into st->n_below (the sample-bracket path, where
@@ -432,8 +135,7 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
         }
         if (l16 == 0 && page < p1 && inf.x >= 0) evict_mask[(size_t)b * mask_stride + page] = ((u64)whi << 32) | (u64)wlo;
     };
-    // Pages are visited from the end of the CTA's range backwards: the histogram pass went forwards, so the
-    // most recently read metadata (the likeliest to still sit in L2) comes first.  Warp-uniform trip count.
+    // Pages are visited from the end of the CTA's range backwards (warp-uniform trip count).
     const long long stride = (long long)(blockDim.x >> 5) * 4;
     long long pp = p0 + warp * 4;
     const long long span = p1 - p0;
@@ -465,135 +167,6 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
 
 
 
-// Filter pass for flat arrays.  A warp takes 512 consecutive scores per trip; lane l reads elements 32 j + l, so the
-// ballot over the lanes for a given j is already 32 consecutive bits of the eviction mask.
-constexpr int FBUF = 64;                                 // candidates a warp stages before it takes a slice of the global list
-
-// Appends the warp's staged candidates to the global list (one atomic per flush).
-__device__ __noinline__ void flat_flush(Cand* wb, int nbuf, SelState* st, Cand* cb, long long cand_cap, int32_t* err) {
-    const int lane = threadIdx.x & 31;
-    unsigned wbase = 0;
-    if (lane == 0) wbase = atomicAdd(&st->cand_count, (unsigned)nbuf);
-    wbase = __shfl_sync(0xffffffffu, wbase, 0);
-    for (int i = lane; i < nbuf; i += 32) {
-        if ((long long)wbase + i < cand_cap) cb[(long long)wbase + i] = wb[i];
-        else latch_error(err, TRIMKV_E_NOMEM);
-    }
-    __syncwarp();
-}
-
-// Stages the candidates of one ballot (cdb: lanes whose score at flat index idx is a candidate); returns the new fill.
-__device__ __noinline__ int flat_stage(Cand* wb, int nbuf, unsigned cdb, float x, long long idx, SelState* st, Cand* cb,
-                                       long long cand_cap, int32_t* err) {
-    const int lane = threadIdx.x & 31;
-    const int cnt = __popc(cdb);
-    if (nbuf + cnt > FBUF) {
-        flat_flush(wb, nbuf, st, cb, cand_cap, err);
-        nbuf = 0;
-    }
-    if (cdb & (1u << lane)) {
-        Cand cnd;
-        cnd.key = compose_key(orderable_key(x), (uint32_t)idx);
-        cnd.slot = (u64)idx;
-        wb[nbuf + __popc(cdb & ((1u << lane) - 1u))] = cnd;
-    }
-    __syncwarp();
-    return nbuf + cnt;
-}
-
-// WHOLE: the candidate range is made of whole score values (its ends carry no index tie-break), the usual case after
-// histogram passes over score words: two float compares decide an entry (a NaN is neither evicted nor a candidate; the
-// histogram pass has flagged it).  Otherwise the 64-bit keys are compared.
-template <bool WHOLE>
-__device__ __forceinline__ void flat_filter_body(const float* __restrict__ s, long long n, SelState* __restrict__ st,
-                                                 Cand* __restrict__ cb, long long cand_cap, u64* __restrict__ evict_mask,
-                                                 int32_t* err, Cand* wb) {
-    constexpr int J = 16;
-    const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
-    const uint32_t lo32 = (uint32_t)(c_lo >> 32), hi32 = (uint32_t)(c_hi >> 32);
-    const float lo_f = key_float_lt(lo32), hi_f = key_float_le(hi32);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long words = (n + 63) / 64;
-    const long long nchunk = (n + 32 * J - 1) / (32 * J);
-    const long long W = (long long)gridDim.x * (blockDim.x >> 5);
-    int nbuf = 0;                                        // warp-uniform
-    auto decide = [&](float x, long long idx, bool& ev, bool& cd) {
-        if (WHOLE) {
-            ev = x < lo_f;
-            cd = !ev && x <= hi_f;
-        } else {
-            const uint32_t sc = orderable_key(x);
-            // one 32-bit compare settles an entry unless its score word equals that of a range end
-            ev = sc < lo32;
-            cd = !ev && sc <= hi32;
-            if (cd && (sc == lo32 || sc == hi32)) {
-                const u64 key = compose_key(sc, (uint32_t)idx);
-                ev = key < c_lo;
-                cd = !ev && key <= c_hi;
-            }
-        }
-    };
-    for (long long c = (long long)blockIdx.x * (blockDim.x >> 5) + warp; c < nchunk; c += W) {
-        const long long base = c * (32 * J);
-        const long long rem = n - base;                  // elements left from the start of this chunk
-        const float* p = s + base + lane;
-        float x[J];
-        unsigned evb[J];
-        if (rem >= 32 * J) {
-#pragma unroll
-            for (int j = 0; j < J; ++j) x[j] = __ldg(p + 32 * j);
-#pragma unroll
-            for (int j = 0; j < J; ++j) {
-                bool ev, cd;
-                decide(x[j], base + 32 * j + lane, ev, cd);
-                evb[j] = __ballot_sync(0xffffffffu, ev);
-                const unsigned cdb = __ballot_sync(0xffffffffu, cd);
-                if (cdb) nbuf = flat_stage(wb, nbuf, cdb, x[j], base + 32 * j + lane, st, cb, cand_cap, err);
-            }
-        } else {                                         // the ragged last chunk
-#pragma unroll 1
-            for (int j = 0; j < J; ++j) {
-                const bool live = 32 * j + lane < rem;
-                const float xv = live ? __ldg(p + 32 * j) : 0.0f;
-                bool ev, cd;
-                decide(xv, base + 32 * j + lane, ev, cd);
-                ev = ev && live;
-                cd = cd && live;
-                const unsigned e = __ballot_sync(0xffffffffu, ev);
-#pragma unroll
-                for (int q = 0; q < J; ++q)
-                    if (q == j) evb[q] = e;
-                const unsigned cdb = __ballot_sync(0xffffffffu, cd);
-                if (cdb) nbuf = flat_stage(wb, nbuf, cdb, xv, base + 32 * j + lane, st, cb, cand_cap, err);
-            }
-        }
-        if (lane < J / 2) {
-            // word `lane` of this chunk = ballots 2 * lane (low half) and 2 * lane + 1 (high half)
-            u64 wv = 0ull;
-#pragma unroll
-            for (int j = 0; j < J / 2; ++j)
-                if (lane == j) wv = (u64)evb[2 * j] | ((u64)evb[2 * j + 1] << 32);
-            const long long wi = c * (J / 2) + lane;
-            if (wi < words) evict_mask[wi] = wv;
-        }
-    }
-    if (nbuf > 0) flat_flush(wb, nbuf, st, cb, cand_cap, err);
-}
-
-__global__ void __launch_bounds__(256, 4)                // the grid is sized for four CTAs per SM
-flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, Cand* __restrict__ cb,
-                   long long cand_cap, u64* __restrict__ evict_mask, int32_t* err) {
-    // Candidates go through a per-warp buffer so that the single global counter sees one atomic per ~50 candidates
-    // (a quarter of a million same-address atomics would serialise the whole pass).
-    __shared__ Cand sbuf[8][FBUF];
-    Cand* wb = sbuf[threadIdx.x >> 5];
-    const u64 c_lo = st->cand_lo, c_hi = st->cand_hi;
-    if ((c_lo & 0xffffffffull) == 0ull && (c_hi & 0xffffffffull) == 0xffffffffull)
-        flat_filter_body<true>(s, n, st, cb, cand_cap, evict_mask, err, wb);
-    else
-        flat_filter_body<false>(s, n, st, cb, cand_cap, evict_mask, err, wb);
-}
-
 // ------------------------------------------------------------------ sample bracket (cache path)
 // One full pass suffices when a candidate range that surely holds the k-th smallest key is known beforehand.
 // A Bernoulli sample of the sequence's keys (a hash of the slot decides, about SAMPLE_MEAN keys) is sorted by one
@@ -602,11 +175,6 @@ flat_filter_kernel(const float* __restrict__ s, long long n, SelState* __restric
 // not (probability below 1e-9 per call), a single-CTA exact selection redoes the sequence.
 constexpr int SAMPLE_CAP = 4096;
 constexpr int SAMPLE_MEAN = 3072;
-
-__device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: spreads slot indices over 32 bits
-    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
-    return x;
-}
 
 // Bernoulli sample of the live slots with probability p each.  sub = 0: every live slot is taken (small sequences).
 // Otherwise a thread owns a block of `sub` consecutive slots of a page (sub a power of two, sub * p <= 1/2): it takes
@@ -1044,48 +612,6 @@ redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_ma
     if (tid == 0) st->resolved = 1;
 }
 
-// Flat arrays: centres the first histogram pass on the threshold.  4096 evenly spaced scores are sampled and ranked by
-// bracket_kernel exactly as for the cache path; the bracket of the k-th key (a tenth of the key range or less) becomes
-// the binned range of the first pass, whose bins are then fine enough to settle the selection at once.  Any range is
-// correct: keys outside it fall into the catch-all bins and cost a further pass at worst.
-__global__ void __launch_bounds__(1024)
-flat_sample_kernel(const float* __restrict__ s, long long n, SelState* __restrict__ st, u64* __restrict__ sample) {
-    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
-    if (gid >= SAMPLE_CAP) return;
-    const long long step = n / SAMPLE_CAP > 0 ? n / SAMPLE_CAP : 1;
-    const long long idx = (long long)gid * step;
-    if (idx >= n) return;
-    const float x = s[idx];
-    if (x != x) return;                                   // NaN is reported by the histogram pass
-    const unsigned w = atomicAdd(&st->sample_count, 1u);
-    const u64 key = compose_key(orderable_key(x), (uint32_t)idx);
-    if (w < SAMPLE_CAP) sample[w] = key;
-    atomicMin(&st->kmin, key);                            // smallest sampled key: lower end when the bracket has none
-}
-
-__global__ void flat_range_kernel(SelState* __restrict__ st) {
-    u64 c_lo = st->cand_lo;
-    const u64 c_hi = st->cand_hi, smin = st->kmin;
-    st->passes = 0;
-    st->sample_count = 0;
-    st->kmin = ~0ull;                                     // as the histogram pass expects it
-    if (c_lo == 0ull && smin < c_hi) {                    // bracket open below: start a little under the sampled minimum
-        const u64 pad = (c_hi - smin) / 8 + 1;
-        c_lo = smin > pad ? smin - pad : 0ull;
-    }
-    if (c_hi <= c_lo) return;                             // keep the full-range default
-    u64 lo = c_lo;
-    int bits = 64 - __clzll((long long)(c_hi - lo));
-    int shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
-    if (shift >= 32) {                                    // bins depend on the score word alone: start on a score boundary
-        lo &= ~0xffffffffull;
-        bits = 64 - __clzll((long long)(c_hi - lo));
-        shift = bits > ZOOM_BITS ? bits - ZOOM_BITS : 0;
-    }
-    st->lo = lo;
-    st->shift = shift;
-}
-
 // ------------------------------------------------------------------ fixed per-pool budget (TrimKV arm)
 // One CTA per pool: the pool keeps its `keep` best entries on its own.  The keys of the pool (up to 8192; longer pools
 // re-read their metadata every sweep) sit in registers; a radix descent over the bits in which they differ finds the
@@ -1215,36 +741,12 @@ __global__ void state_init_kernel(SelState* sel, int B) {
     sel[b] = s;
 }
 
-__global__ void invert_mask_kernel(const u64* __restrict__ ev, u64* __restrict__ keep, long long n) {
-    const long long words = (n + 63) / 64;
-    for (long long w = blockIdx.x * (long long)blockDim.x + threadIdx.x; w < words;
-         w += (long long)gridDim.x * blockDim.x) {
-        const long long rem = n - w * 64;
-        const u64 valid = rem >= 64 ? ~0ull : ((1ull << rem) - 1ull);
-        keep[w] = ~ev[w] & valid;
-    }
-}
-
 int grid_x_for(long long pages, int B) {
     long long g = (pages + 31) / 32;              // at least ~32 pages per CTA
     long long cap = (592 + B - 1) / B;            // ~4 CTAs per SM over the whole grid
     if (g > cap) g = cap;
     if (g < 1) g = 1;
     return (int)g;
-}
-
-// Histogram path (flat arrays): up to max_passes histogram passes, filter, exact resolve.
-void run_select_flat(const ArraySrc& src, const SelectBuffers& sb, long long k_evict, int max_passes, unsigned cand_target,
-                     u64* evict_mask, int32_t* err, cudaStream_t st) {
-    const long long pages = (src.n + PAGE - 1) / PAGE;
-    dim3 grid(grid_x_for(pages, 1), 1);
-    for (int p = 0; p < max_passes; ++p)
-        hist_kernel<ArraySrc><<<grid, 256, 0, st>>>(src, sb.sel, sb.hist, sb.done, k_evict, src.n, p == max_passes - 1,
-                                                    cand_target);
-    flat_filter_kernel<<<grid, 256, 0, st>>>(src.s, src.n, sb.sel, sb.cand, sb.cand_cap, evict_mask, err);
-    resolve_kernel<true><<<1, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, evict_mask, pages, k_evict,
-                                             max(cand_target / 8u, 1u), sb.stats, nullptr, err);
-    count_launch(max_passes + 2);
 }
 
 }  // namespace
@@ -1299,31 +801,6 @@ void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, in
     const long long pools = (long long)cv.B * cv.L * cv.H;
     cudaMemsetAsync(compact_cursor, 0, (size_t)cv.B * sizeof(int32_t), st);
     pool_select_kernel<<<(unsigned)pools, 256, 0, st>>>(cv, t + 1, keep_per_pool);
-    count_launch();
-}
-
-void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,
-                         int32_t* err, cudaStream_t st) {
-    ArraySrc src;
-    src.s = scores;
-    src.n = n;
-    src.err = err;
-    u64* sample = reinterpret_cast<u64*>(sb.cand);        // the candidate buffer is idle until the filter pass
-    flat_sample_kernel<<<SAMPLE_CAP / 1024, 1024, 0, st>>>(scores, n, sb.sel, sample);
-    // 4 sigma: here a miss (6e-5 per call) only costs one more histogram pass, and the narrower range keeps the
-    // candidate list of the last bin within what the resolution holds in registers
-    bracket_kernel<<<1, 1024, 0, st>>>(sb.sel, sample, k_evict, n, 0, 4.0f);
-    flat_range_kernel<<<1, 1, 0, st>>>(sb.sel);
-    count_launch(3);
-    run_select_flat(src, sb, k_evict, 7, (unsigned)sb.cand_cap, evict_mask, err, st);
-}
-
-void launch_invert_mask(const u64* evict_mask, u64* keep_bits, long long n, cudaStream_t st) {
-    const long long words = (n + 63) / 64;
-    int grid = (int)((words + 255) / 256);
-    if (grid > 1184) grid = 1184;
-    if (grid < 1) grid = 1;
-    invert_mask_kernel<<<grid, 256, 0, st>>>(evict_mask, keep_bits, n);
     count_launch();
 }
 

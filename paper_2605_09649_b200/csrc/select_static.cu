@@ -10,9 +10,10 @@
 
 namespace {
 
-// Scratch needed by the selection for n <= TRIMKV_SELECT_STATIC_MAX_N scores: 1 KB of state, the
-// 4096-bin histogram and 16384 candidate records of 16 bytes, plus alignment slack.
-constexpr size_t STATIC_SCRATCH_BYTES = 1024 + (size_t)tkv::NB * sizeof(uint32_t) + 16384 * sizeof(tkv::Cand) + 256;
+// Scratch needed by the selection for n <= TRIMKV_SELECT_STATIC_MAX_N scores: the same layout and size formula as the
+// workspace of trimkv_select_topk (state, histograms, the candidate list of n / 16 + 16384 keys): about 2.4 MB.
+constexpr size_t STATIC_SCRATCH_BYTES = tkv::flat_select_workspace_bytes(TRIMKV_SELECT_STATIC_MAX_N);
+static_assert(STATIC_SCRATCH_BYTES < (3u << 20), "the built-in scratch array is meant to stay small");
 
 static __device__ __align__(256) unsigned char g_select_scratch[STATIC_SCRATCH_BYTES];
 
@@ -27,6 +28,15 @@ cudaError_t scratch_address(void** out) {
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> guard(g_setup_lock);
+    if (g_scratch_addr[dev]) {
+        // a cudaDeviceReset since the look-up would have destroyed the context the address belongs to: check it still
+        // names device memory (a query, no allocation) and look it up again if not
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, g_scratch_addr[dev]) != cudaSuccess || attr.type != cudaMemoryTypeDevice) {
+            cudaGetLastError();
+            g_scratch_addr[dev] = nullptr;
+        }
+    }
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_select_scratch);
@@ -57,7 +67,7 @@ extern "C" TRIMKV_API trimkv_status trimkv_select_topk_static(const float* score
         tkv::set_last_error("cudaGetSymbolAddress of the built-in scratch array failed: %s", cudaGetErrorString(e));
         return TRIMKV_E_CUDA;
     }
-    // The selection clears the state words and the histogram it needs at zero on `stream` before its
-    // kernels run; the candidate records are written before they are read.
+    // The selection's first kernel clears, on `stream`, every counter and histogram that must start at zero; the
+    // candidate lists are written before they are read.
     return trimkv_select_topk(scores, n, k_keep, keep_bits, scratch, STATIC_SCRATCH_BYTES, status_out, stream);
 }

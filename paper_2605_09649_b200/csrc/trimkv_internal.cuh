@@ -61,6 +61,24 @@ __device__ __forceinline__ u64 make_key(float score, uint32_t tie) {
     return ((u64)orderable_key(score) << 32) | (u64)(~tie);
 }
 
+__device__ __forceinline__ u64 compose_key(uint32_t sc, uint32_t tie) { return ((u64)sc << 32) | (u64)(~tie); }
+
+// Float-domain forms of 32-bit key comparisons, for any non-NaN x:
+//   x <  key_float_lt(k)  iff  orderable_key(x) <  k        x <= key_float_le(k)  iff  orderable_key(x) <= k
+// Keys at or below that of -inf / at or above that of +inf (NaN bit patterns) clamp to -inf / +inf.  No float has the
+// key 0x7fffffff (it would be -0, which is folded onto +0): "<" there means "< -0", "<=" means "<= the key before it".
+__device__ __forceinline__ float key_float_lt(uint32_t key) {
+    if (key <= 0x007fffffu) return __uint_as_float(0xff800000u);         // at or below key(-inf)
+    if (key >= 0xff800000u) return __uint_as_float(0x7f800000u);         // at or above key(+inf)
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+__device__ __forceinline__ float key_float_le(uint32_t key) { return key_float_lt(key == 0x7fffffffu ? 0x7ffffffeu : key); }
+
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {   // integer finaliser: spreads slot indices over 32 bits
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
 // c = ln sum_{k<horizon} exp(k * lambda): the beta-only factor of the retention score (horizon 0 = infinite).
 __device__ __forceinline__ float horizon_term_f32(float lam, int horizon) {
     if (horizon == 1) return 0.0f;
@@ -182,9 +200,18 @@ void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, in
 void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t* cursor, long long e_max,
                     long long evictions_per_seq, cudaStream_t st);
 
-void launch_select_array(const float* scores, long long n, long long k_evict, u64* evict_mask, const SelectBuffers& sb,
-                         int32_t* err, cudaStream_t st);
-void launch_invert_mask(const u64* evict_mask, u64* keep_bits, long long n, cudaStream_t st);
+// Standalone selection over a flat score array (select_flat.cu).  Workspace layout: 1 KB of state and counters, the
+// candidate histogram (in several copies; the exact fallback's histograms reuse the space), the keys ranked exactly,
+// then the candidate list.
+constexpr int FLAT_HIST_BINS = 4096, FLAT_HIST_REPLICAS = 8, FLAT_X_BINS = 2048, FLAT_X_PASSES = 6, FLAT_CAND2_CAP = 16384;
+constexpr size_t FLAT_FIXED_BYTES = 1024 + (size_t)FLAT_HIST_REPLICAS * FLAT_HIST_BINS * 4 + (size_t)FLAT_CAND2_CAP * 8;
+constexpr long long flat_select_cand_cap(long long n) { return n / 16 + 16384; }   // keys inside the sampled bracket, with margin
+constexpr size_t flat_select_workspace_bytes(long long n) {
+    return FLAT_FIXED_BYTES + (size_t)flat_select_cand_cap(n) * 8 + 256;
+}
+// Keeps the k_keep largest of n scores: keep_bits words are written in full.  status (may be null) is set by the kernels.
+cudaError_t launch_select_flat(const float* scores, long long n, long long k_keep, u64* keep_bits, void* workspace,
+                               size_t workspace_bytes, int32_t* status, int distrust, cudaStream_t stream);
 void launch_select_state_init(SelState* sel, int B, cudaStream_t st);
 
 struct AttnBuffers {

@@ -825,16 +825,9 @@ const char* trimkv_last_error(void) { return g_err; }
 int64_t trimkv_kernel_launches(void) { return (int64_t)tkv::g_launches.load(std::memory_order_relaxed); }
 
 // ---- standalone selection ---------------------------------------------------------------------------
-static long long select_cand_cap(int64_t n) {
-    long long cap = n / 1024;
-    if (cap < 16384) cap = 16384;
-    return cap;
-}
-static const size_t SEL_HDR = 1024;   // SelState, done counter, stats
-
 size_t trimkv_select_workspace_bytes(int64_t n) {
     if (n < 0) return 0;
-    return SEL_HDR + (size_t)NB * sizeof(uint32_t) + (size_t)select_cand_cap(n) * sizeof(Cand) + 256;
+    return flat_select_workspace_bytes(n);
 }
 
 trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
@@ -844,30 +837,9 @@ trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep,
     if (!scores || !keep_bits || !workspace || !aligned16(scores) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return fail(TRIMKV_E_ARG, "NULL or misaligned buffer (scores 16 B, workspace 256 B)");
     if (workspace_bytes < trimkv_select_workspace_bytes(n)) return fail(TRIMKV_E_ARG, "workspace too small");
-    cudaStream_t st = (cudaStream_t)stream;
-    const long long words = (n + 63) / 64;
-    if (status_out) CUDA_TRY(cudaMemsetAsync(status_out, 0, sizeof(int32_t), st));
-    const long long k_evict = n - std::min<long long>(k_keep, n);
-    if (k_evict == 0 || k_evict == n) {
-        CUDA_TRY(cudaMemsetAsync(keep_bits, k_evict == 0 ? 0x00 : 0xFF, (size_t)words * 8, st));
-        launch_invert_mask((const u64*)keep_bits, (u64*)keep_bits, n, st);   // 0 -> all kept, 1s -> none kept
-        CUDA_TRY(cudaGetLastError());
-        return TRIMKV_OK;
-    }
-    char* ws = (char*)workspace;
-    SelectBuffers sb;
-    sb.sel = (SelState*)ws;
-    sb.done = (unsigned*)(ws + 256);
-    sb.stats = (long long*)(ws + 512);
-    sb.hist = (uint32_t*)(ws + SEL_HDR);
-    sb.cand = (Cand*)(ws + SEL_HDR + (size_t)NB * sizeof(uint32_t));
-    sb.cand_cap = select_cand_cap(n);
-    sb.sample = nullptr;
-    CUDA_TRY(cudaMemsetAsync(ws, 0, SEL_HDR + (size_t)NB * sizeof(uint32_t), st));
-    launch_select_state_init(sb.sel, 1, st);
-    launch_select_array(scores, n, k_evict, (u64*)keep_bits, sb, status_out, st);
-    launch_invert_mask((const u64*)keep_bits, (u64*)keep_bits, n, st);
-    CUDA_TRY(cudaGetLastError());
+    const cudaError_t e = launch_select_flat(scores, n, k_keep, (u64*)keep_bits, workspace, workspace_bytes, status_out,
+                                             tkv::global_test_hooks() & TRIMKV_TEST_DISTRUST_SAMPLE, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(TRIMKV_E_CUDA, "selection launch failed: %s", cudaGetErrorString(e));
     return TRIMKV_OK;
 }
 

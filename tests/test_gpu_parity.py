@@ -625,6 +625,55 @@ def test_select_topk_matches_full_sort(n):
             np.testing.assert_array_equal(got, _oracle_keep_bits(s_np, k), err_msg=f"{kind} n={n} k={k}")
 
 
+def _select_with_stats(s, k):
+    n = s.numel()
+    ws = torch.zeros(binding.select_workspace_bytes(n), dtype=torch.uint8, device=DEV)
+    bits, status = binding.select_topk(s, k, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    stats = ws[512:512 + 32].view(torch.int64).cpu().tolist()      # {fallback taken, bracket keys, ranked keys, sampled}
+    return _unpack(bits, n), stats
+
+
+def test_select_topk_reads_the_scores_once_in_the_normal_case():
+    """Uniform scores: the sampled bracket holds the threshold, a few percent of the keys go to the candidate list and a
+    few hundred are ranked exactly; no fallback."""
+    n = (1 << 22) + 12345
+    s = workloads.selection_scores(n, seed=2, device=DEV)
+    for k in (n // 8, n // 2, n - 512):
+        got, stats = _select_with_stats(s, k)
+        np.testing.assert_array_equal(got, _oracle_keep_bits(s.cpu().numpy(), k))
+        assert stats[0] == 0 and 4096 < stats[3] <= 8192
+        assert 0 < stats[1] < n // 10 and 0 < stats[2] <= 16384, stats
+
+
+def test_select_topk_exact_fallbacks_match_full_sort():
+    """The two exact fallbacks on demand.  (1) With the sample distrusted (testing aid) the bracket cannot hold the
+    threshold and the exact radix select over all scores runs.  (2) Two score values with the threshold just beside the
+    boundary between them: the bracket straddles the two values, all candidates of one value fall into one histogram bin,
+    more than the final ranking holds, and the exact radix select over the candidate list runs."""
+    try:
+        binding.set_global_test_hooks(binding.TEST_DISTRUST_SAMPLE)
+        for n in (1000, 4097, (1 << 20) + 3):
+            for kind in ("uniform", "two"):
+                s = workloads.selection_scores(n, seed=n + 5, device=DEV)
+                if kind == "two":
+                    s = (s > -4.0).float() * -3.0 - 1.0
+                for k in (1, n // 3, n - 1):
+                    got, stats = _select_with_stats(s, k)
+                    assert stats[0] == 2, stats
+                    np.testing.assert_array_equal(got, _oracle_keep_bits(s.cpu().numpy(), k), err_msg=f"{kind} n={n} k={k}")
+    finally:
+        binding.set_global_test_hooks(0)
+    n = 1 << 21
+    s = (workloads.selection_scores(n, seed=77, device=DEV) > -4.0).float() * 2.0 - 7.0          # -7 or -5, about half each
+    low = int((s == -7.0).sum().item())
+    for k_evict in (low - 1000, low + 1000):
+        got, stats = _select_with_stats(s, n - k_evict)
+        assert stats[0] == 1 and stats[2] > 16384, stats
+        np.testing.assert_array_equal(got, _oracle_keep_bits(s.cpu().numpy(), n - k_evict))
+
+
 def test_select_topk_rejects_nan_and_bad_args():
     s = torch.tensor([0.0, float("nan"), -1.0, -2.0] * 64, device=DEV)
     bits, status = binding.select_topk(s, 100)
