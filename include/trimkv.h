@@ -79,6 +79,12 @@ typedef struct trimkv_config {
     int32_t per_pool_budget; /* 0: one global budget per sequence (the paper's method).  > 0: the fixed-budget variant it is
                                compared with (TrimKV): every (layer, head) pool keeps its own per_pool_budget best
                                entries; budget_entries (>= per_pool_budget x layers x kv_heads) then only sizes the cache */
+    int32_t shard_total_layers; /* 0: the handle holds whole sequences.  > 0: it holds `layers` consecutive layers, starting
+                               at shard_layer0, of sequences whose shard_total_layers layers are spread over several
+                               handles (ranks) that share ONE global budget (see the trimkv_shard_* calls).
+                               budget_entries is then this handle's CAPACITY: the most entries per sequence its layers
+                               may keep after an eviction round                                                      */
+    int32_t shard_layer0;   /* first layer of the slice (layer arguments of the other calls stay local: 0 .. layers-1) */
 } trimkv_config;
 
 /* Fill *cfg with defaults (batch 1, q_heads = kv_heads, bf16, no gate, page 64, d_g 512,
@@ -206,6 +212,45 @@ TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);
 /* enable = 2 records the attention main kernel alone (two events per call: cheap enough for a timed run). */
 TRIMKV_API trimkv_status trimkv_profile(trimkv_t* h, int enable);
 TRIMKV_API trimkv_status trimkv_profile_read(trimkv_t* h, double* ms_host, int64_t* count_host);
+
+/* ---- one sequence sharded by layer over several handles (ranks) ------------------------------------
+ * The global eviction rule ranks the entries of ALL layers and heads of a sequence under one budget (Sec. 4.2).  When
+ * the layers of a sequence live on several GPUs, each rank creates a handle for its slice (shard_total_layers > 0) and
+ * uses append / decode_attention as usual; an eviction round is then run in stages, with three small exchanges between
+ * them that the caller performs (an all-gather, an all-reduce, an all-gather: NCCL through torch.distributed, or any
+ * other transport).  After each exchange every rank computes the same result from the same data, so all reach the same
+ * threshold and each flags its own entries.  Per sequence, with W ranks and B sequences:
+ *   1. trimkv_shard_sample     local key sample (Bernoulli, rate from the GLOBAL entry count) -> keys [B][cap], counts [B]
+ *      exchange: all-gather keys and counts                          (cap = trimkv_shard_sample_cap() keys of 8 bytes)
+ *   2. trimkv_shard_bracket    gathered samples [W][B][cap], [W][B] -> the bracket of the k-th smallest key (same on all ranks)
+ *   3. trimkv_shard_filter     one pass over the local metadata: keys below the bracket are flagged and counted, keys
+ *                              inside it listed -> n_below [B] (int64), cand_count [B] (int32; -1 = the local list overflowed)
+ *      exchange: all-reduce (sum) n_below, all-gather cand_count, then all-gather the candidate records
+ *   4. trimkv_shard_candidates local candidate records (16 bytes each: key, slot) -> [B][cand_cap_x]
+ *   5. trimkv_shard_resolve    gathered records [W][B][cand_cap_x], counts [W][B], global n_below [B] -> exact threshold;
+ *                              this rank's candidates up to it are flagged; resolved [B] (int32) = 0 where the bracket
+ *                              missed the threshold or a list overflowed (same on every rank)
+ *   6. only if some sequence is unresolved (all ranks see the same flags): exact radix select, 6 rounds of
+ *      trimkv_shard_hist (local digit histogram [B][2048], uint32) -> exchange: all-reduce (sum) -> trimkv_shard_digit
+ *      (prefix [B] uint64 and rank [B] int64 move one digit down; start: prefix 0, rank k_evict, top 64, then
+ *      top = 53, 42, 31, 20, 9), then trimkv_shard_mark with tau = prefix
+ *   7. trimkv_shard_compact    compaction of the local pools; returns this rank's entries per sequence (synchronises)
+ * t, n_total and k_evict are GLOBAL: tokens seen, entries of one sequence over all ranks, entries to evict.  All
+ * pointers are device memory unless the name says host; calls are asynchronous on `stream` except the last one. */
+TRIMKV_API int32_t trimkv_shard_sample_cap(void);
+TRIMKV_API trimkv_status trimkv_shard_sample(trimkv_t* h, int64_t n_total, int64_t k_evict, uint64_t* keys_out, int32_t* counts_out,
+                                  void* stream);
+TRIMKV_API trimkv_status trimkv_shard_bracket(trimkv_t* h, int world, const uint64_t* gathered_keys, const int32_t* gathered_counts,
+                                   int64_t n_total, int64_t k_evict, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_filter(trimkv_t* h, int64_t* n_below_out, int32_t* cand_count_out, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_candidates(trimkv_t* h, int64_t cap, void* cand_out, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_resolve(trimkv_t* h, int world, int rank, int64_t cap, const void* gathered_cand,
+                                   const int32_t* gathered_counts, const int64_t* n_below_global, int64_t k_evict,
+                                   int32_t* resolved_out, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_hist(trimkv_t* h, const uint64_t* prefix, int top, uint32_t* hist_out, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_digit(trimkv_t* h, const uint32_t* hist, uint64_t* prefix, int64_t* rank, int top, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_mark(trimkv_t* h, const uint64_t* tau, void* stream);
+TRIMKV_API trimkv_status trimkv_shard_compact(trimkv_t* h, int64_t* local_entries_out_host, void* stream);
 
 /* ---- testing aids (not part of the method) ------------------------------------------------------
  * Switches that make rarely taken paths run on demand, so that tests can reach them without a fault:

@@ -26,6 +26,8 @@ EXPORTS = [
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static", "trimkv_set_test_hooks",
+    "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
+    "trimkv_shard_resolve", "trimkv_shard_hist", "trimkv_shard_digit", "trimkv_shard_mark", "trimkv_shard_compact",
 ]
 
 
@@ -42,6 +44,7 @@ class Config(C.Structure):
         ("gate_hidden", C.c_int32), ("gate_embed", C.c_int32), ("horizon", C.c_int32), ("kv_dtype", C.c_int32),
         ("max_chunk", C.c_int32), ("reserved", C.c_int32), ("max_pool_pages", C.c_int64),
         ("retention_bias", C.c_int32), ("per_pool_budget", C.c_int32),
+        ("shard_total_layers", C.c_int32), ("shard_layer0", C.c_int32),
     ]
 
 
@@ -85,6 +88,16 @@ def lib() -> C.CDLL:
     L.trimkv_profile.argtypes = [vp, i32]
     L.trimkv_set_overlap.argtypes = [vp, i32]
     L.trimkv_set_test_hooks.argtypes = [vp, i32]
+    L.trimkv_shard_sample_cap.argtypes = []
+    L.trimkv_shard_sample.argtypes = [vp, i64, i64, vp, vp, vp]
+    L.trimkv_shard_bracket.argtypes = [vp, i32, vp, vp, i64, i64, vp]
+    L.trimkv_shard_filter.argtypes = [vp, vp, vp, vp]
+    L.trimkv_shard_candidates.argtypes = [vp, i64, vp, vp]
+    L.trimkv_shard_resolve.argtypes = [vp, i32, i32, i64, vp, vp, vp, i64, vp, vp]
+    L.trimkv_shard_hist.argtypes = [vp, vp, i32, vp, vp]
+    L.trimkv_shard_digit.argtypes = [vp, vp, vp, vp, i32, vp]
+    L.trimkv_shard_mark.argtypes = [vp, vp, vp]
+    L.trimkv_shard_compact.argtypes = [vp, vp, vp]
     L.trimkv_set_horizon.argtypes = [vp, i32, vp]
     L.trimkv_profile_read.argtypes = [vp, vp, vp]
     L.trimkv_last_error.argtypes = []
@@ -99,7 +112,10 @@ def lib() -> C.CDLL:
                  "trimkv_append", "trimkv_score_and_evict", "trimkv_decode_attention", "trimkv_decode_step_all",
                  "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
                  "trimkv_sync_status", "trimkv_profile", "trimkv_profile_read", "trimkv_select_topk",
-                 "trimkv_select_topk_static", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_set_test_hooks"):
+                 "trimkv_select_topk_static", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_set_test_hooks",
+                 "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter",
+                 "trimkv_shard_candidates", "trimkv_shard_resolve", "trimkv_shard_hist", "trimkv_shard_digit",
+                 "trimkv_shard_mark", "trimkv_shard_compact"):
         getattr(L, name).restype = i32
     _lib = L
     return L
@@ -140,7 +156,7 @@ class TrimKV:
     def __init__(self, budget_entries: int, layers: int, kv_heads: int, head_dim: int, *, q_heads: Optional[int] = None,
                  hidden: int = 0, batch: int = 1, gate_hidden: int = 512, gate_embed: int = 64, horizon: int = 2,
                  kv_dtype: str = "bf16", max_chunk: int = 512, max_pool_pages: int = 0, distrust_sample: bool = False,
-                 retention_bias: bool = False, per_pool_budget: int = 0):
+                 retention_bias: bool = False, per_pool_budget: int = 0, shard_total_layers: int = 0, shard_layer0: int = 0):
         L = lib()
         cfg = Config()
         L.trimkv_default_config(C.byref(cfg), budget_entries, layers, kv_heads, head_dim)
@@ -155,6 +171,8 @@ class TrimKV:
         cfg.max_pool_pages = max_pool_pages
         cfg.retention_bias = 1 if retention_bias else 0
         cfg.per_pool_budget = per_pool_budget
+        cfg.shard_total_layers = shard_total_layers
+        cfg.shard_layer0 = shard_layer0
         cfg.reserved = 0
         self.cfg = cfg
         self.torch_dtype = torch.bfloat16 if kv_dtype == "bf16" else torch.float32

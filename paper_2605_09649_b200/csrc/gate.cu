@@ -177,10 +177,12 @@ gate_transpose_kernel(const float* __restrict__ W1, float* __restrict__ W1T, int
 constexpr int GO_RT = 2;  // rows per CTA of the output kernel (few: at decode the kernel is a chain of dependent loads per thread)
 
 // s[lb][r][h] = v[layer][h] . u[lb][r] + s0[layer][h]; then beta / lambda / c.   grid = (row tiles, layers).
+// to_cache (a decode step: row r is sequence r's new token, whose K/V half of the append has run): the retention terms
+// also go straight to the token's slot, the newest entry of pool (r, layer, h).
 __global__ void __launch_bounds__(256)
 gate_out_kernel(const float* __restrict__ zpart, const float* __restrict__ b1, const float* __restrict__ v,
                 const float* __restrict__ s0, int layer0, int R, int dg, int nchunk, int H, int horizon,
-                float* __restrict__ beta, float* __restrict__ lam, float* __restrict__ cterm) {
+                float* __restrict__ beta, float* __restrict__ lam, float* __restrict__ cterm, int to_cache, CacheView cv) {
     extern __shared__ float su[];           // [GO_RT][dg] rows of u = SiLU(sum of the chunk partials + b1)
     const int lb = blockIdx.y;
     const int layer = layer0 + lb;
@@ -237,7 +239,20 @@ gate_out_kernel(const float* __restrict__ zpart, const float* __restrict__ b1, c
                 const size_t o = ((size_t)lb * R + r0 + rr) * H + h;
                 if (beta) beta[o] = bt;
                 if (lam) lam[o] = lm;
-                if (cterm) cterm[o] = horizon_term_f32(lm, horizon);
+                const float ct = horizon_term_f32(lm, horizon);
+                if (cterm) cterm[o] = ct;
+                if (to_cache) {
+                    const int b = r0 + rr;
+                    const long long pool = ((long long)b * cv.L + layer) * cv.H + h;
+                    const int idx = cv.len[pool] - 1;
+                    if (!cv.append_failed[pool] && idx >= 0) {
+                        const int page = cv.block_table[pool * cv.maxpp + idx / PAGE];
+                        const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + idx % PAGE;
+                        if (lm != lm || ct != ct) latch_error(cv.err, TRIMKV_E_NONFINITE);
+                        cv.lam[slot] = lm;
+                        cv.c[slot] = ct;
+                    }
+                }
             }
         }
     }
@@ -260,16 +275,17 @@ void launch_gate_transpose(const float* W1, float* W1T, int dg, int D, cudaStrea
 }
 
 void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, int layer0, int nlayers, int rows_per_layer,
-                     float* beta, float* lam, float* c, cudaStream_t st) {
+                     float* beta, float* lam, float* c, cudaStream_t st, const CacheView* to_cache) {
     dim3 g2((rows_per_layer + GO_RT - 1) / GO_RT, nlayers);
     const size_t smem = (size_t)GO_RT * gp.dg * sizeof(float);
+    CacheView none{};
     gate_out_kernel<<<g2, 256, smem, st>>>(z_scratch, gp.b1, gp.v, gp.s0, layer0, rows_per_layer, gp.dg, nchunk, gp.H,
-                                           gp.horizon, beta, lam, c);
+                                           gp.horizon, beta, lam, c, to_cache ? 1 : 0, to_cache ? *to_cache : none);
     count_launch();
 }
 
-void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
-                 float* beta, float* lam, float* c, cudaStream_t st) {
+void launch_gate_hidden(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
+                        cudaStream_t st) {
     const int nchunk = gate_chunks(gp.D);
     auto run = [&](auto kernel, int rw, int jt) {
         dim3 g1(((rows_per_layer + rw - 1) / rw) * nchunk, (gp.dg + jt * GH_THREADS - 1) / (jt * GH_THREADS), nlayers);
@@ -278,7 +294,12 @@ void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int lay
     if (rows_per_layer <= 8) run(gate_hidden_kernel<8, 4>, 8, 4);
     else run(gate_hidden_kernel<16, 2>, 16, 2);                 // row tiles of 16
     count_launch();
-    launch_gate_out(gp, z_scratch, nchunk, layer0, nlayers, rows_per_layer, beta, lam, c, st);
+}
+
+void launch_gate(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
+                 float* beta, float* lam, float* c, cudaStream_t st) {
+    launch_gate_hidden(gp, x, z_scratch, layer0, nlayers, rows_per_layer, st);
+    launch_gate_out(gp, z_scratch, gate_chunks(gp.D), layer0, nlayers, rows_per_layer, beta, lam, c, st, nullptr);
 }
 
 }  // namespace tkv

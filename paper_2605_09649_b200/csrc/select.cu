@@ -47,7 +47,7 @@ struct CacheSrc {
             const float S = retention_score(l4[j], c4[j], (float)(t1i - p4[j]));
             bad |= (S != S) && (e0 + j < inf.z);
             sc[j] = orderable_key(S);
-            tie[j] = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)inf.x;
+            tie[j] = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)(inf.x + cv.pool_offset);
             if (e0 + j < inf.z) vm |= 1u << j;
         }
         if (bad) latch_error(cv.err, TRIMKV_E_NONFINITE);
@@ -200,7 +200,7 @@ sample_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ sample
         const size_t s = ((size_t)b * cv.P_seq + page) * PAGE + off;
         const int pos = cv.pos[s];
         const float S = retention_score(cv.lam[s], cv.c[s], (float)(src.t1 - (long long)pos));
-        const uint32_t tie = ((uint32_t)pos << cv.pool_bits) | (uint32_t)inf.x;
+        const uint32_t tie = ((uint32_t)pos << cv.pool_bits) | (uint32_t)(inf.x + cv.pool_offset);
         const unsigned w = atomicAdd(&st->sample_count, 1u);
         if (w < SAMPLE_CAP) sample[(size_t)b * SAMPLE_CAP + w] = make_key(S, tie);
     };
@@ -332,15 +332,20 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
     }
 }
 
+constexpr int SHARD_TAG_SHIFT = 56;      // a sharded selection tags a candidate's slot with its rank above this bit
+
 // ------------------------------------------------------------------ exact ranking of the candidates
 // One CTA per sequence.  STRICT (histogram path): the candidate range is known to hold the k-th key; any
 // inconsistency is an internal error.  Otherwise (sample-bracket path): an inconsistent count means the range
-// missed; resolved stays 0 and the exact redo kernel takes over.
+// missed; resolved stays 0 and (redo_inline) this CTA redoes its sequence exactly, or the caller runs its own fallback.
+__device__ void redo_body(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_mask, long long mask_stride,
+                          long long k_evict, int32_t* err);
+
 template <bool STRICT>
 __global__ void __launch_bounds__(1024)
 resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap, u64* __restrict__ evict_mask,
                long long mask_stride, long long k_evict, unsigned next_aim, long long* __restrict__ stats,
-               int32_t* __restrict__ cursor, int32_t* err) {
+               int32_t* __restrict__ cursor, int32_t* err, CacheSrc src, int redo_inline, int my_rank = -1) {
     constexpr int DB = 11, NBIN = 1 << DB;
     __shared__ unsigned hist[NBIN];
     __shared__ unsigned wtot[32];
@@ -367,6 +372,10 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
                 if (stats) { stats[b * 4 + 0] = 1; stats[b * 4 + 1] = C; stats[b * 4 + 2] = k_evict; stats[b * 4 + 3] = sample_n; }
                 if (cursor) cursor[b] = 0;
             }
+            // the bracket missed (next to never): this CTA redoes its sequence exactly, at once, instead of a further
+            // kernel that every call would have to launch just to find nothing to do
+            __syncthreads();
+            if (redo_inline) redo_body(src, sel, evict_mask, mask_stride, k_evict, err);
             return;
         }
     }
@@ -475,8 +484,12 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
         tau = prefix;   // the r-th smallest candidate key: everything <= tau is evicted
         for (long long i = tid; i < C; i += blockDim.x) {
             const Cand cnd = cb[i];
-            if (cnd.key <= tau)
-                atomicOr(evict_mask + (size_t)b * mask_stride + (cnd.slot >> 6), 1ull << (cnd.slot & 63));
+            // my_rank >= 0 (a sequence sharded over ranks): the list holds every rank's candidates, tagged with their
+            // rank in the slot's top byte; only this rank's own slots exist here
+            if (cnd.key <= tau && (my_rank < 0 || (int)(cnd.slot >> SHARD_TAG_SHIFT) == my_rank)) {
+                const u64 slot = cnd.slot & ((1ull << SHARD_TAG_SHIFT) - 1ull);
+                atomicOr(evict_mask + (size_t)b * mask_stride + (slot >> 6), 1ull << (slot & 63));
+            }
         }
     } else {
         tau = st->cand_lo;
@@ -512,11 +525,11 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
     }
 }
 
-// Exact redo for a sequence whose sample bracket missed: one CTA radix-selects the k-th smallest key over all of
-// the sequence's entries (DB bits per sweep) and rewrites every eviction mask.  Slow and rare.
-__global__ void __launch_bounds__(1024)
-redo_kernel(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_mask, long long mask_stride,
-            long long k_evict, int32_t* err) {
+// Exact redo for a sequence whose sample bracket missed (called by the ranking kernel's CTA of that sequence): the CTA
+// radix-selects the k-th smallest key over all of the sequence's entries (DB bits per sweep) and rewrites every eviction
+// mask.  Slow and rare.
+__device__ void redo_body(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_mask, long long mask_stride,
+                          long long k_evict, int32_t* err) {
     constexpr int DB = 11, NBIN = 1 << DB;
     __shared__ unsigned hist[NBIN];
     __shared__ unsigned wtot[32];
@@ -642,7 +655,7 @@ pool_select_kernel(CacheView cv, long long t1, int keep) {
         const int pos = cv.pos[slot];
         const float S = retention_score(cv.lam[slot], cv.c[slot], (float)(t1i - pos));
         if (S != S) latch_error(cv.err, TRIMKV_E_NONFINITE);
-        return make_key(S, ((uint32_t)pos << cv.pool_bits) | (uint32_t)pool_local);
+        return make_key(S, ((uint32_t)pos << cv.pool_bits) | (uint32_t)(pool_local + cv.pool_offset));
     };
     const bool inreg = n <= PER * 256;
     u64 kr[PER];
@@ -749,15 +762,266 @@ int grid_x_for(long long pages, int B) {
     return (int)g;
 }
 
+// ------------------------------------------------------------------ one sequence sharded by layer over ranks
+// Every rank holds the pools of a slice of the layers; the budget is global over all of them (Sec. 4.2).  The selection
+// is the same as on one GPU (sample -> bracket -> filter -> exact ranking), with three small exchanges between the
+// stages: the ranks' sample keys, their counts of keys below the bracket, and their candidates.  After each exchange
+// every rank computes the same thing from the same data, so all reach the same threshold and each flags its own slots.
+// The kernels below are the rank-local pieces; the exchanges are the caller's (NCCL through torch.distributed).
+
+// Sample keys and their count out of the handle (one CTA per sequence).
+__global__ void shard_export_sample_kernel(const SelState* __restrict__ sel, const u64* __restrict__ sample,
+                                           u64* __restrict__ keys_out, int32_t* __restrict__ counts_out) {
+    const int b = blockIdx.x;
+    const unsigned raw = sel[b].sample_count;
+    const int ns = (int)min(raw, (unsigned)SAMPLE_CAP);
+    for (int i = threadIdx.x; i < ns; i += blockDim.x) keys_out[(size_t)b * SAMPLE_CAP + i] = sample[(size_t)b * SAMPLE_CAP + i];
+    if (threadIdx.x == 0) counts_out[b] = ns;
+}
+
+// The ranks' samples, concatenated in rank order, become the handle's sample (gkeys [W][B][SAMPLE_CAP], gcounts [W][B]).
+__global__ void shard_merge_sample_kernel(const u64* __restrict__ gkeys, const int32_t* __restrict__ gcounts, int W, int B,
+                                          SelState* __restrict__ sel, u64* __restrict__ sample) {
+    const int b = blockIdx.x;
+    long long off = 0;
+    for (int w = 0; w < W; ++w) {
+        const int cnt = gcounts[(size_t)w * B + b];
+        const u64* src = gkeys + ((size_t)w * B + b) * SAMPLE_CAP;
+        for (int i = threadIdx.x; i < cnt; i += blockDim.x)
+            if (off + i < SAMPLE_CAP) sample[(size_t)b * SAMPLE_CAP + off + i] = src[i];
+        off += cnt;
+    }
+    if (threadIdx.x == 0) sel[b].sample_count = (unsigned)off;
+}
+
+__global__ void shard_export_filter_kernel(const SelState* __restrict__ sel, long long cand_cap, long long* __restrict__ n_below_out,
+                                           int32_t* __restrict__ cand_count_out, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    n_below_out[b] = sel[b].n_below;
+    const long long cc = (long long)sel[b].cand_count;
+    cand_count_out[b] = cc > cand_cap ? -1 : (int32_t)cc;                            // -1: the local list overflowed
+}
+
+__global__ void shard_export_cands_kernel(const SelState* __restrict__ sel, const Cand* __restrict__ cand, long long cand_cap,
+                                          Cand* __restrict__ out, long long cap) {
+    const int b = blockIdx.y;
+    const long long cnt = min(min((long long)sel[b].cand_count, cand_cap), cap);
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < cnt; i += (long long)gridDim.x * blockDim.x)
+        out[(size_t)b * cap + i] = cand[(size_t)b * cand_cap + i];
+}
+
+// All ranks' candidates (gcand [W][B][cap], gcounts [W][B]) become the handle's candidate list, each slot tagged with its
+// rank; the global count of keys below the bracket replaces the local one.  A list that does not fit, or a rank whose
+// own list overflowed, makes the count inconsistent on purpose: the exact ranking then reports a miss.
+__global__ void shard_merge_cands_kernel(const Cand* __restrict__ gcand, const int32_t* __restrict__ gcounts,
+                                         const long long* __restrict__ n_below_global, int W, int B, long long cap,
+                                         SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap) {
+    const int b = blockIdx.y;
+    long long off = 0;
+    bool bad = false;
+    for (int w = 0; w < W; ++w) {
+        const long long cnt = gcounts[(size_t)w * B + b];
+        if (cnt < 0 || cnt > cap) { bad = true; continue; }
+        const Cand* src = gcand + ((size_t)w * B + b) * cap;
+        for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < cnt; i += (long long)gridDim.x * blockDim.x) {
+            if (off + i < cand_cap) {
+                Cand c = src[i];
+                c.slot |= (u64)w << SHARD_TAG_SHIFT;
+                cand[(size_t)b * cand_cap + off + i] = c;
+            }
+        }
+        off += cnt;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        sel[b].cand_count = (bad || off > cand_cap) ? 0xffffffffu : (unsigned)off;
+        sel[b].n_below = n_below_global[b];
+    }
+}
+
+__global__ void shard_export_resolved_kernel(const SelState* __restrict__ sel, int32_t* __restrict__ out, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) out[b] = sel[b].resolved;
+}
+
+// Exact fallback, one radix digit per round: local histogram of the digit below `top` over the keys whose bits above
+// `top` equal prefix[b] (sequences already resolved contribute nothing).  hist_out [B][2048], zeroed here.
+__global__ void __launch_bounds__(1024)
+shard_hist_kernel(CacheSrc src, const SelState* __restrict__ sel, const u64* __restrict__ prefix, int top,
+                  unsigned* __restrict__ hist_out) {
+    constexpr int DB = 11, NBIN = 1 << DB;
+    __shared__ unsigned hist[NBIN];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    hist[tid] = 0u;
+    hist[tid + 1024] = 0u;
+    __syncthreads();
+    if (!sel[b].resolved) {
+        const int dbits = top < DB ? top : DB, sh = top - dbits;
+        const u64 pfx = prefix[b];
+        const int sub = lane >> 4, e0 = (lane & 15) * 4;
+        const long long P = src.pages();
+        for (long long pp = warp * 2; pp < P; pp += 64) {
+            const long long page = pp + sub;
+            if (page < P) {
+                const int4 inf = src.info(b, page);
+                uint32_t sc[4], tie[4];
+                const unsigned vm = src.load4(b, page, e0, inf, sc, tie);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (vm & (1u << j)) {
+                        const u64 key = compose_key(sc[j], tie[j]);
+                        if (top >= 64 || (key >> top) == pfx) atomicAdd(&hist[(unsigned)((key >> sh) & ((1u << dbits) - 1u))], 1u);
+                    }
+                }
+            }
+        }
+    }
+    __syncthreads();
+    hist_out[(size_t)b * NBIN + tid] = hist[tid];
+    hist_out[(size_t)b * NBIN + tid + 1024] = hist[tid + 1024];
+}
+
+// From the histogram summed over the ranks: the digit that holds rank r[b]; prefix and rank move one digit down.
+__global__ void __launch_bounds__(1024)
+shard_digit_kernel(const unsigned* __restrict__ hist, u64* __restrict__ prefix, long long* __restrict__ rank, int top) {
+    constexpr int DB = 11, NBIN = 1 << DB;
+    __shared__ unsigned wtot[32];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int dbits = top < DB ? top : DB;
+    const unsigned h0 = hist[(size_t)b * NBIN + 2 * tid], h1 = hist[(size_t)b * NBIN + 2 * tid + 1];
+    unsigned incl = h0 + h1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) wtot[warp] = incl;
+    __syncthreads();
+    unsigned off = 0;
+    for (int w = 0; w < warp; ++w) off += wtot[w];
+    const long long excl = (long long)off + incl - (h0 + h1);
+    const long long r = rank[b];
+    const u64 p = top >= 64 ? 0ull : (prefix[b] << dbits);
+    __syncthreads();
+    if (r > excl && r <= excl + h0) { prefix[b] = p | (u64)(2 * tid); rank[b] = r - excl; }
+    else if (r > excl + h0 && r <= excl + h0 + h1) { prefix[b] = p | (u64)(2 * tid + 1); rank[b] = r - excl - h0; }
+}
+
+// Exact fallback, last step: every local key up to tau[b] is evicted (sequences already resolved keep their masks).
+__global__ void __launch_bounds__(1024)
+shard_mark_kernel(CacheSrc src, SelState* __restrict__ sel, const u64* __restrict__ tau, u64* __restrict__ evict_mask,
+                  long long mask_stride, int32_t* __restrict__ cursor) {
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (sel[b].resolved) return;
+    const u64 t = tau[b];
+    const int sub = lane >> 4, l16 = lane & 15, e0 = l16 * 4;
+    const long long P = src.pages();
+    for (long long pp = warp * 2; pp < P; pp += 64) {          // warp-uniform trip count
+        const long long page = pp + sub;
+        int4 inf = make_int4(-1, 0, 0, 0);
+        uint32_t sc[4], tie[4];
+        unsigned vm = 0;
+        if (page < P) {
+            inf = src.info(b, page);
+            vm = src.load4(b, page, e0, inf, sc, tie);
+        }
+        unsigned ev = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if ((vm & (1u << j)) && compose_key(sc[j], tie[j]) <= t) ev |= 1u << j;
+        const unsigned nib = ev << (4 * (l16 & 7));
+        unsigned wlo = (l16 < 8) ? nib : 0u, whi = (l16 >= 8) ? nib : 0u;
+#pragma unroll
+        for (int o = 1; o < 16; o <<= 1) {
+            wlo |= __shfl_xor_sync(0xffffffffu, wlo, o);
+            whi |= __shfl_xor_sync(0xffffffffu, whi, o);
+        }
+        if (l16 == 0 && page < P && inf.x >= 0) evict_mask[(size_t)b * mask_stride + page] = ((u64)whi << 32) | (u64)wlo;
+    }
+    __syncthreads();
+    if (tid == 0) { sel[b].resolved = 1; sel[b].cand_count = 0; sel[b].sample_count = 0; if (cursor) cursor[b] = 0; }
+}
+
 }  // namespace
+
+// ---- launchers of the sharded selection's rank-local stages
+int shard_sample_cap() { return SAMPLE_CAP; }
+
+void launch_shard_export_sample(const CacheView& cv, const SelectBuffers& sb, u64* keys_out, int32_t* counts_out, cudaStream_t st) {
+    shard_export_sample_kernel<<<cv.B, 256, 0, st>>>(sb.sel, sb.sample, keys_out, counts_out);
+    count_launch();
+}
+
+void launch_shard_bracket(const CacheView& cv, const SelectBuffers& sb, const u64* gkeys, const int32_t* gcounts, int world,
+                          long long n_total, long long k_evict, int distrust, cudaStream_t st) {
+    shard_merge_sample_kernel<<<cv.B, 256, 0, st>>>(gkeys, gcounts, world, cv.B, sb.sel, sb.sample);
+    bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust, 7.0f);
+    count_launch(2);
+}
+
+void launch_shard_filter(const CacheView& cv, const SelectBuffers& sb, long long t, long long* n_below_out,
+                         int32_t* cand_count_out, cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
+    dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
+    filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, nullptr);
+    shard_export_filter_kernel<<<(cv.B + 127) / 128, 128, 0, st>>>(sb.sel, sb.cand_cap, n_below_out, cand_count_out, cv.B);
+    count_launch(2);
+}
+
+void launch_shard_export_cands(const CacheView& cv, const SelectBuffers& sb, void* out, long long cap, cudaStream_t st) {
+    dim3 grid(8, cv.B);
+    shard_export_cands_kernel<<<grid, 256, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, (Cand*)out, cap);
+    count_launch();
+}
+
+void launch_shard_resolve(const CacheView& cv, const SelectBuffers& sb, const void* gcand, const int32_t* gcounts,
+                          const long long* n_below_global, int world, int rank, long long cap, long long k_evict,
+                          int32_t* compact_cursor, int32_t* resolved_out, cudaStream_t st) {
+    dim3 grid(8, cv.B);
+    shard_merge_cands_kernel<<<grid, 256, 0, st>>>((const Cand*)gcand, gcounts, n_below_global, world, cv.B, cap, sb.sel, sb.cand,
+                                                   sb.cand_cap);
+    CacheSrc none;
+    none.cv = cv;
+    none.t1 = 0;
+    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u, sb.stats,
+                                                 compact_cursor, cv.err, none, 0, rank);
+    shard_export_resolved_kernel<<<(cv.B + 127) / 128, 128, 0, st>>>(sb.sel, resolved_out, cv.B);
+    count_launch(3);
+}
+
+void launch_shard_hist(const CacheView& cv, const SelectBuffers& sb, long long t, const u64* prefix, int top, unsigned* hist_out,
+                       cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
+    shard_hist_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, prefix, top, hist_out);
+    count_launch();
+}
+
+void launch_shard_digit(int B, const unsigned* hist, u64* prefix, long long* rank, int top, cudaStream_t st) {
+    shard_digit_kernel<<<B, 1024, 0, st>>>(hist, prefix, rank, top);
+    count_launch();
+}
+
+void launch_shard_mark(const CacheView& cv, const SelectBuffers& sb, long long t, const u64* tau, int32_t* compact_cursor,
+                       cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
+    shard_mark_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, tau, cv.evict_mask, cv.P_seq, compact_cursor);
+    count_launch();
+}
 
 void launch_select_state_init(SelState* sel, int B, cudaStream_t st) {
     state_init_kernel<<<(B + 127) / 128, 128, 0, st>>>(sel, B);
     count_launch();
 }
 
-void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
-                                long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st) {
+// The sampling pass alone (n_total: the entry count the sampling rate is derived from).
+static void launch_sample_only(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, int skip_newest,
+                               cudaStream_t st) {
     CacheSrc src;
     src.cv = cv;
     src.t1 = t + 1;
@@ -769,13 +1033,25 @@ void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, lo
         while (sub > 1 && p * sub > 0.5) sub >>= 1;
         thresh = (uint32_t)(4294967296.0 * std::min(p * sub, 0.999999));
     }
-    const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u;
+    const uint32_t seed = (uint32_t)t * 0x9E3779B1u + 0x1234567u + (uint32_t)cv.pool_offset * 0x632BE5ABu;
     const long long threads = cv.P_seq * (sub > 0 ? PAGE / sub : 1);
     dim3 gs((unsigned)((threads + 255) / 256), cv.B);
     sample_kernel<<<gs, 256, 0, st>>>(src, sb.sel, sb.sample, sub, thresh, seed, skip_newest);
+    count_launch();
+}
+
+void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,
+                                long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st) {
+    launch_sample_only(cv, sb, t, n_total, skip_newest, st);
     // 7 sigma: a miss costs the single-CTA exact redo of the whole sequence, so it must be next to impossible
     bracket_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.sample, k_evict, n_total, distrust_sample, 7.0f);
-    count_launch(2);
+    count_launch();
+}
+
+void launch_shard_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, u64* keys_out,
+                         int32_t* counts_out, cudaStream_t st) {
+    launch_sample_only(cv, sb, t, n_total, 0, st);
+    launch_shard_export_sample(cv, sb, keys_out, counts_out, st);
 }
 
 void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
@@ -786,9 +1062,8 @@ void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long
     dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
     filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
     resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
-                                                 sb.stats, compact_cursor, cv.err);
-    redo_kernel<<<cv.B, 1024, 0, st>>>(src, sb.sel, cv.evict_mask, cv.P_seq, k_evict, cv.err);
-    count_launch(3);
+                                                 sb.stats, compact_cursor, cv.err, src, 1);
+    count_launch(2);
 }
 
 void launch_select_cache(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total,

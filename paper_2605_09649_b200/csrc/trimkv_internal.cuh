@@ -118,6 +118,8 @@ struct CacheView {
     int row_bytes;         // d * sizeof(element)
     int swizzle;           // 1 if rows are chunk-permuted
     int pool_bits;         // bits that hold layer*H+head in the tie-break word
+    int pool_offset;       // added to the local layer*H+head in that word: > 0 when the handle holds a slice of a
+                           // sequence's layers (the pool id of the tie-break is the id within the whole model)
 };
 
 __device__ __forceinline__ size_t kv_row_offset(const CacheView& cv, int b, long long page, int part, int off) {
@@ -164,8 +166,12 @@ void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st);
 
 // Second half of the gate alone: z_scratch holds nchunk partial pre-activations per (row, hidden unit).
+// to_cache != null (decode step, one row per sequence): lambda and c are also written to the newest entry of every pool.
 void launch_gate_out(const GateParams& gp, const float* z_scratch, int nchunk, int layer0, int nlayers, int rows_per_layer,
-                     float* beta, float* lam, float* c, cudaStream_t st);
+                     float* beta, float* lam, float* c, cudaStream_t st, const CacheView* to_cache = nullptr);
+// First half of the gate alone (the hidden layer's partial pre-activations into z_scratch).
+void launch_gate_hidden(const GateParams& gp, const float* x, float* z_scratch, int layer0, int nlayers, int rows_per_layer,
+                        cudaStream_t st);
 
 // Tensor-core (tcgen05, 3xTF32) form of the hidden layer for calls with many rows of one layer.
 struct GateTcState;
@@ -194,6 +200,24 @@ void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, lo
                                 long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st);
 void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
                               int32_t* compact_cursor, cudaStream_t st);
+// Rank-local stages of the selection of a sequence whose layers are sharded over ranks (see select.cu).
+int shard_sample_cap();
+void launch_shard_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, u64* keys_out,
+                         int32_t* counts_out, cudaStream_t st);
+void launch_shard_export_sample(const CacheView& cv, const SelectBuffers& sb, u64* keys_out, int32_t* counts_out, cudaStream_t st);
+void launch_shard_bracket(const CacheView& cv, const SelectBuffers& sb, const u64* gkeys, const int32_t* gcounts, int world,
+                          long long n_total, long long k_evict, int distrust, cudaStream_t st);
+void launch_shard_filter(const CacheView& cv, const SelectBuffers& sb, long long t, long long* n_below_out,
+                         int32_t* cand_count_out, cudaStream_t st);
+void launch_shard_export_cands(const CacheView& cv, const SelectBuffers& sb, void* out, long long cap, cudaStream_t st);
+void launch_shard_resolve(const CacheView& cv, const SelectBuffers& sb, const void* gcand, const int32_t* gcounts,
+                          const long long* n_below_global, int world, int rank, long long cap, long long k_evict,
+                          int32_t* compact_cursor, int32_t* resolved_out, cudaStream_t st);
+void launch_shard_hist(const CacheView& cv, const SelectBuffers& sb, long long t, const u64* prefix, int top, unsigned* hist_out,
+                       cudaStream_t st);
+void launch_shard_digit(int B, const unsigned* hist, u64* prefix, long long* rank, int top, cudaStream_t st);
+void launch_shard_mark(const CacheView& cv, const SelectBuffers& sb, long long t, const u64* tau, int32_t* compact_cursor,
+                       cudaStream_t st);
 // Fixed per-pool budget: every pool keeps its keep_per_pool best entries (masks as for launch_select_cache).
 void launch_select_pools(const CacheView& cv, long long t, int keep_per_pool, int32_t* compact_cursor, cudaStream_t st);
 // evictions_per_seq: how many entries the selection just flagged per sequence (sizes the CTAs).

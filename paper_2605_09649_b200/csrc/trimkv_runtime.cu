@@ -121,6 +121,7 @@ struct trimkv {
     cudaStream_t side_hi = nullptr;                                 // `side` at the priority of `fast` (gate-heavy steps)
     bool overlap = true;
     int test_hooks = 0;              // TRIMKV_TEST_* switches of this handle
+    bool shard = false;              // the handle holds a slice of the layers of sequences sharded over ranks
     char* pool_stage = nullptr;      // device staging of trimkv_get_pool, grown on demand
     size_t pool_stage_bytes = 0;
     cudaEvent_t ev_fork = nullptr, ev_append = nullptr, ev_side = nullptr, ev_done = nullptr, ev_sample = nullptr;
@@ -220,6 +221,7 @@ long long eviction_due(const trimkv* h) {
 
 // Entries per sequence the cache has room for between two eviction rounds: what survives a round plus one chunk.
 long long capacity_entries(const trimkv* h) {
+    if (h->shard) return h->n_max;
     const long long LH = (long long)h->L * h->H;
     return (h->cfg.per_pool_budget > 0 ? (long long)h->cfg.per_pool_budget * LH : h->M) + h->e_max;
 }
@@ -247,6 +249,7 @@ trimkv_status compact_impl(trimkv* h, cudaStream_t st) {
 }
 
 trimkv_status evict_impl(trimkv* h, cudaStream_t st) {
+    if (h->shard) return fail(TRIMKV_E_STATE, "this handle holds a slice of the layers: run the eviction round with the trimkv_shard_* calls");
     const long long t = h->tokens[0];
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layer %d holds %lld tokens, layer 0 holds %lld", l, h->tokens[l], t);
@@ -317,6 +320,11 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
                                      (long long)cfg->per_pool_budget * cfg->layers * cfg->kv_heads > cfg->budget_entries))
         return fail(TRIMKV_E_ARG, "per_pool_budget * layers * kv_heads must not exceed budget_entries (which sizes the cache)");
 
+    if (cfg->shard_total_layers < 0 || (cfg->shard_total_layers > 0 &&
+                                        (cfg->shard_layer0 < 0 || cfg->shard_layer0 + cfg->layers > cfg->shard_total_layers ||
+                                         cfg->per_pool_budget > 0)))
+        return fail(TRIMKV_E_ARG, "shard_layer0 + layers must lie within shard_total_layers (global budget only)");
+    if ((long long)cfg->shard_total_layers * cfg->kv_heads > 65536) return fail(TRIMKV_E_UNSUPPORTED, "layers * kv_heads too large");
     trimkv* h = new (std::nothrow) trimkv();
     if (!h) return fail(TRIMKV_E_NOMEM, "host allocation failed");
     h->cfg = *cfg;
@@ -325,12 +333,15 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     h->elt = cfg->kv_dtype == TRIMKV_DTYPE_BF16 ? 2 : 4;
     h->M = cfg->budget_entries;
     const long long LH = (long long)h->L * h->H;
-    h->e_max = (long long)cfg->max_chunk * LH;
-    h->n_max = h->M + h->e_max;
+    h->shard = cfg->shard_total_layers > 0;
+    const long long LH_all = h->shard ? (long long)cfg->shard_total_layers * h->H : LH;   // pools of the whole model
+    // a round may evict, on this handle, as many entries as the WHOLE model gained since the last round
+    h->e_max = (long long)cfg->max_chunk * LH_all;
+    h->n_max = h->M + (long long)cfg->max_chunk * LH;
     h->P_seq = (h->n_max + PAGE - 1) / PAGE + LH + 8;
     h->maxpp = cfg->max_pool_pages > 0 ? std::min<long long>(cfg->max_pool_pages, h->P_seq) : h->P_seq;
     h->slots_seq = h->P_seq * PAGE;
-    h->pool_bits = std::max(1, ceil_log2(LH));
+    h->pool_bits = std::max(1, ceil_log2(LH_all));
     h->max_pos = std::min<long long>((1LL << 24) - 1, (1LL << (32 - h->pool_bits)) - 1);
     h->tokens.assign(h->L, 0);
     h->gate_set.assign(h->L, 0);
@@ -345,6 +356,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     cv.row_bytes = h->d * h->elt;
     cv.swizzle = (cfg->kv_dtype == TRIMKV_DTYPE_BF16 && cv.row_bytes % 128 == 0) ? 1 : 0;
     cv.pool_bits = h->pool_bits;
+    cv.pool_offset = h->shard ? cfg->shard_layer0 * h->H : 0;
     const size_t pools = (size_t)h->B * LH;
     const size_t slots = (size_t)h->B * h->slots_seq;
     trimkv_status s = TRIMKV_OK;
@@ -573,6 +585,7 @@ struct HostArgs {
 
 trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, const void* k, const void* v, const void* q,
                             void* out, void* stream, const HostArgs* host) {
+    if (h->shard) return fail(TRIMKV_E_STATE, "this handle holds a slice of the layers: use the per-layer calls and the trimkv_shard_* calls");
     const long long t = h->tokens[0];
     for (int l = 1; l < h->L; ++l)
         if (h->tokens[l] != t) return fail(TRIMKV_E_STATE, "layers hold different token counts");
@@ -636,11 +649,13 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     const float* lam = lambda;
     const float* cc = nullptr;
     if (x) {
+        // the hidden layer streams its weights beside the K/V append; the output kernel then writes the retention terms
+        // straight into the new entries' slots, which exist once the K/V half of the append has run
         if (h->prof.on) h->prof.mark(PH_GATE, 0, sd);
-        launch_gate(gate_params(h), x, h->u, 0, h->L, h->B, nullptr, h->g_lam, h->g_c, sd);
+        launch_gate_hidden(gate_params(h), x, h->u, 0, h->L, h->B, sd);
+        if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
+        launch_gate_out(gate_params(h), h->u, gate_chunks(h->D), 0, h->L, h->B, nullptr, nullptr, nullptr, sd, &h->cv);
         if (h->prof.on) h->prof.mark(PH_GATE, 1, sd);
-        lam = h->g_lam;
-        cc = h->g_c;
     }
     // The selection's sample and rank bracket need only the page records of this step (final once the K/V half of the
     // append has run), not the new entries' retention terms: they run on a third stream beside the gate.
@@ -650,8 +665,10 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
         launch_select_cache_sample(h->cv, h->sb, h->tokens[0], h->entries, kev, 1, h->test_hooks & TRIMKV_TEST_DISTRUST_SAMPLE, h->side2);
         CUDA_TRY(cudaEventRecord(h->ev_sample, h->side2));
     }
-    if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
-    launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, APPEND_META, sd);
+    if (!x) {
+        if (two) CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_append, 0));
+        launch_append(h->cv, 0, h->L, 1, t, lam, cc, h->cfg.horizon, k, v, APPEND_META, sd);
+    }
     if (early_sample) {
         CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_sample, 0));
         if (h->prof.on) h->prof.mark(PH_SELECT, 0, sd);
@@ -787,6 +804,109 @@ trimkv_status trimkv_set_horizon(trimkv_t* h, int horizon, void* stream) {
     launch_rehorizon(h->cv, horizon, (cudaStream_t)stream);
     CUDA_TRY(cudaGetLastError());
     return TRIMKV_OK;
+}
+
+// ---- one sequence sharded by layer over ranks: the rank-local stages of an eviction round ----------------------------
+static trimkv_status shard_ready(trimkv* h) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!h->shard) return fail(TRIMKV_E_STATE, "the handle was not created with shard_total_layers > 0");
+    for (int l = 1; l < h->L; ++l)
+        if (h->tokens[l] != h->tokens[0]) return fail(TRIMKV_E_STATE, "layers hold different token counts");
+    return TRIMKV_OK;
+}
+
+int32_t trimkv_shard_sample_cap(void) { return shard_sample_cap(); }
+
+trimkv_status trimkv_shard_sample(trimkv_t* h, int64_t n_total, int64_t k_evict, uint64_t* keys_out, int32_t* counts_out,
+                                  void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (!keys_out || !counts_out || n_total < 1 || k_evict < 1 || k_evict > n_total) return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_sample(h->cv, h->sb, h->tokens[0], n_total, (u64*)keys_out, counts_out, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_bracket(trimkv_t* h, int world, const uint64_t* gathered_keys, const int32_t* gathered_counts,
+                                   int64_t n_total, int64_t k_evict, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (world < 1 || !gathered_keys || !gathered_counts || n_total < 1 || k_evict < 1) return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_bracket(h->cv, h->sb, (const u64*)gathered_keys, gathered_counts, world, n_total, k_evict,
+                         h->test_hooks & TRIMKV_TEST_DISTRUST_SAMPLE, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_filter(trimkv_t* h, int64_t* n_below_out, int32_t* cand_count_out, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (!n_below_out || !cand_count_out) return fail(TRIMKV_E_ARG, "NULL output");
+    launch_shard_filter(h->cv, h->sb, h->tokens[0], (long long*)n_below_out, cand_count_out, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_candidates(trimkv_t* h, int64_t cap, void* cand_out, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (cap < 1 || !cand_out) return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_export_cands(h->cv, h->sb, cand_out, cap, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_resolve(trimkv_t* h, int world, int rank, int64_t cap, const void* gathered_cand,
+                                   const int32_t* gathered_counts, const int64_t* n_below_global, int64_t k_evict,
+                                   int32_t* resolved_out, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (world < 1 || rank < 0 || rank >= world || world > 255 || cap < 1 || !gathered_cand || !gathered_counts || !n_below_global ||
+        !resolved_out)
+        return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_resolve(h->cv, h->sb, gathered_cand, gathered_counts, (const long long*)n_below_global, world, rank, cap, k_evict,
+                         h->cursor, resolved_out, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_hist(trimkv_t* h, const uint64_t* prefix, int top, uint32_t* hist_out, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (!prefix || !hist_out || top < 1 || top > 64) return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_hist(h->cv, h->sb, h->tokens[0], (const u64*)prefix, top, hist_out, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_digit(trimkv_t* h, const uint32_t* hist, uint64_t* prefix, int64_t* rank, int top, void* stream) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (!hist || !prefix || !rank || top < 1 || top > 64) return fail(TRIMKV_E_ARG, "bad argument");
+    launch_shard_digit(h->B, hist, (u64*)prefix, (long long*)rank, top, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_mark(trimkv_t* h, const uint64_t* tau, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    if (!tau) return fail(TRIMKV_E_ARG, "NULL tau");
+    launch_shard_mark(h->cv, h->sb, h->tokens[0], (const u64*)tau, h->cursor, (cudaStream_t)stream);
+    CUDA_TRY(cudaGetLastError());
+    return TRIMKV_OK;
+}
+
+trimkv_status trimkv_shard_compact(trimkv_t* h, int64_t* local_entries_out_host, void* stream) {
+    if (trimkv_status s = shard_ready(h)) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    launch_compact(h->cv, h->hole, h->mover, h->cursor, h->e_max, h->e_max, st);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaStreamSynchronize(st));
+    const size_t LH = (size_t)h->L * h->H;
+    std::vector<int32_t> len((size_t)h->B * LH);
+    CUDA_TRY(cudaMemcpy(len.data(), h->cv.len, len.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    long long worst = 0;
+    for (int b = 0; b < h->B; ++b) {
+        long long e = 0;
+        for (size_t p = 0; p < LH; ++p) e += len[(size_t)b * LH + p];
+        if (local_entries_out_host) local_entries_out_host[b] = e;
+        worst = std::max(worst, e);
+    }
+    h->entries = worst;              // sequences may keep different numbers here: the fullest one bounds the next append
+    return device_status(h);
 }
 
 trimkv_status trimkv_set_test_hooks(trimkv_t* h, int flags) {
