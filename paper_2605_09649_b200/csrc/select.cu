@@ -26,12 +26,18 @@ struct CacheSrc {
     static constexpr bool FLAT = false;
     CacheView cv;
     long long t1;   // t + 1
+    int skip_newest = 0;   // > 0: leave out the last skip_newest entries of every pool (their retention terms are not written yet)
     __device__ long long pages() const { return cv.P_seq; }
     // {pool, logical page, live entries, -}; pool < 0: the page is free
     __device__ int4 info(int b, long long p) const { return __ldg(cv.owner + (size_t)b * cv.P_seq + p); }
     // returns the valid-entry bits (4) of this lane; sc = orderable score (high key word), tie = ~low key word
     __device__ unsigned load4(int b, long long p, int e0, const int4& inf, uint32_t (&sc)[4], uint32_t (&tie)[4]) const {
-        if (inf.x < 0 || e0 >= inf.z) return 0u;
+        int live = inf.z;                                 // entries of this page that take part
+        if (skip_newest > 0 && inf.x >= 0) {
+            const int rest = cv.len[(size_t)b * cv.L * cv.H + inf.x] - skip_newest - inf.y * PAGE;   // entries left for this page
+            live = rest < live ? (rest > 0 ? rest : 0) : live;
+        }
+        if (inf.x < 0 || e0 >= live) return 0u;
         const size_t s = ((size_t)b * cv.P_seq + p) * PAGE + e0;
         const float4 lm = *reinterpret_cast<const float4*>(cv.lam + s);
         const float4 cc = *reinterpret_cast<const float4*>(cv.c + s);
@@ -45,10 +51,10 @@ struct CacheSrc {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float S = retention_score(l4[j], c4[j], (float)(t1i - p4[j]));
-            bad |= (S != S) && (e0 + j < inf.z);
+            bad |= (S != S) && (e0 + j < live);
             sc[j] = orderable_key(S);
             tie[j] = ((uint32_t)p4[j] << cv.pool_bits) | (uint32_t)(inf.x + cv.pool_offset);
-            if (e0 + j < inf.z) vm |= 1u << j;
+            if (e0 + j < live) vm |= 1u << j;
         }
         if (bad) latch_error(cv.err, TRIMKV_E_NONFINITE);
         return vm;
@@ -166,6 +172,42 @@ filter_kernel(Src src, SelState* __restrict__ sel, Cand* __restrict__ cand, long
 }
 
 
+
+// The newest entry of every pool, classified after a filter pass that left it out (its retention terms arrived later):
+// one thread per pool; flagged, listed or left alone exactly as the filter pass would have done.
+__global__ void filter_newest_kernel(CacheSrc src, SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap,
+                                     u64* __restrict__ evict_mask, long long mask_stride, int32_t* err) {
+    const CacheView& cv = src.cv;
+    const int LH = cv.L * cv.H;
+    const int gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= cv.B * LH) return;
+    const int b = gid / LH, pool_local = gid % LH;
+    const int n = cv.len[gid];
+    if (n <= 0) return;
+    const int idx = n - 1;
+    const int page = cv.block_table[(size_t)gid * cv.maxpp + idx / PAGE];
+    const int off = idx % PAGE;
+    const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + off;
+    const int pos = cv.pos[slot];
+    const float S = retention_score(cv.lam[slot], cv.c[slot], (float)(src.t1 - (long long)pos));
+    if (S != S) latch_error(cv.err, TRIMKV_E_NONFINITE);
+    const u64 key = make_key(S, ((uint32_t)pos << cv.pool_bits) | (uint32_t)(pool_local + cv.pool_offset));
+    SelState* st = sel + b;
+    if (key < st->cand_lo) {
+        atomicOr(reinterpret_cast<unsigned long long*>(evict_mask + (size_t)b * mask_stride + page), 1ull << off);
+        atomicAdd(reinterpret_cast<unsigned long long*>(&st->n_below), 1ull);
+    } else if (key <= st->cand_hi) {
+        const unsigned w = atomicAdd(&st->cand_count, 1u);
+        if ((long long)w < cand_cap) {
+            Cand cnd;
+            cnd.key = key;
+            cnd.slot = (u64)((long long)page * PAGE + off);
+            cand[(size_t)b * cand_cap + w] = cnd;
+        } else {
+            latch_error(err, TRIMKV_E_NOMEM);
+        }
+    }
+}
 
 // ------------------------------------------------------------------ sample bracket (cache path)
 // One full pass suffices when a candidate range that surely holds the k-th smallest key is known beforehand.
@@ -1052,6 +1094,31 @@ void launch_shard_sample(const CacheView& cv, const SelectBuffers& sb, long long
                          int32_t* counts_out, cudaStream_t st) {
     launch_sample_only(cv, sb, t, n_total, 0, st);
     launch_shard_export_sample(cv, sb, keys_out, counts_out, st);
+}
+
+void launch_select_cache_filter(const CacheView& cv, const SelectBuffers& sb, long long t, int skip_newest, cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
+    src.skip_newest = skip_newest;
+    dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
+    filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
+    count_launch();
+}
+
+void launch_select_cache_finish(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
+                                int32_t* compact_cursor, int newest_left_out, cudaStream_t st) {
+    CacheSrc src;
+    src.cv = cv;
+    src.t1 = t + 1;
+    if (newest_left_out) {
+        const int pools = cv.B * cv.L * cv.H;
+        filter_newest_kernel<<<(pools + 127) / 128, 128, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
+        count_launch();
+    }
+    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
+                                                 sb.stats, compact_cursor, cv.err, src, 1);
+    count_launch();
 }
 
 void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,

@@ -277,7 +277,7 @@ flat_bracket_kernel(const float* __restrict__ s, long long n, long long k_evict,
 // bracket's histogram layout, keys below it are counted, and the last CTA reads the narrower bracket off the bins that
 // hold the sample ranks several standard deviations around the expected one.  Any outcome is a valid bracket or the
 // first one unchanged; the exact stages after it check whatever they are given.
-constexpr int REFINE_CTAS = 64, REFINE_THREADS = 256, REFINE_PER = 16;     // 2^18 samples
+constexpr int REFINE_CTAS = 128, REFINE_THREADS = 256, REFINE_PER = 8;     // 2^18 samples
 __global__ void __launch_bounds__(REFINE_THREADS)
 flat_refine_kernel(const float* __restrict__ s, long long n, long long k_evict, FlatState* __restrict__ st,
                    uint32_t* __restrict__ hist2, long long* __restrict__ stats, float sigmas) {
@@ -538,8 +538,46 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
     // After a trip's keep words are written: the scores that may be inside.  Every lane lists the positions of its own;
     // the warp then classifies the listed scores exactly, 32 at a time.  xs: the trip's scores in shared memory (null for
     // the ragged last trip, which re-reads them from global memory).
+    // exact classification of one score that may be inside; returns true if it is a candidate (key: its key)
+    auto classify = [&](float xv, uint32_t idx, u64& key) -> bool {
+        bad |= xv != xv;
+        key = flat_key(xv, idx);
+        const bool fast_ev = xv < mid_lt;
+        const bool ev = key < mid;
+        adj += (key < lo ? 1 : 0) - (fast_ev ? 1 : 0);
+        const bool cnd = key >= lo && key <= hi;
+        if (cnd) atomicAdd(&sm.sh[flat_bin(key, bin_base, shift)], 1u);
+        if (ev != fast_ev) {                                     // equal score words, the index decides: settle the bit now
+            unsigned long long* wp = reinterpret_cast<unsigned long long*>(keep_bits + (idx >> 6));
+            if (ev) atomicAnd(wp, ~(1ull << (idx & 63))); else atomicOr(wp, 1ull << (idx & 63));
+        }
+        return cnd;
+    };
     auto handle_inside = [&](unsigned m, long long base, const float* xs) {
-        if (!__any_sync(0xffffffffu, m != 0u)) return;
+        const int tot_in = __reduce_add_sync(0xffffffffu, __popc(m));
+        if (!tot_in) return;
+        if (tot_in <= 8) {
+            // a handful: every lane that has some takes its own, one per round (rounds = the most any lane has, mostly one)
+            if (nbuf + tot_in > FBUF) {
+                flat_flush(sm.wb, nbuf, st, cand, cand_cap);
+                nbuf = 0;
+            }
+            __syncwarp();                                        // the trip's keep words are written
+            while (__any_sync(0xffffffffu, m != 0u)) {
+                bool cnd = false;
+                u64 key = 0ull;
+                if (m) {
+                    const int p = 32 * (__ffs(m) - 1) + lane;
+                    m &= m - 1;
+                    cnd = classify(xs ? xs[p] : __ldg(s + base + p), (uint32_t)base + (uint32_t)p, key);
+                }
+                const unsigned cdb = __ballot_sync(0xffffffffu, cnd);
+                if (cnd) sm.wb[nbuf + __popc(cdb & ((1u << lane) - 1u))] = key;
+                nbuf += __popc(cdb);
+            }
+            __syncwarp();
+            return;
+        }
         if (lane0) *sm.ecount = 0u;
         __syncwarp();
         if (m) {
@@ -562,19 +600,7 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
             u64 key = 0ull;
             if (e < tot) {
                 const int p = sm.elist[e];
-                const uint32_t idx = (uint32_t)base + (uint32_t)p;
-                const float xv = xs ? xs[p] : __ldg(s + base + p);
-                bad |= xv != xv;
-                key = flat_key(xv, idx);
-                const bool fast_ev = xv < mid_lt;
-                const bool ev = key < mid;
-                adj += (key < lo ? 1 : 0) - (fast_ev ? 1 : 0);
-                cnd = key >= lo && key <= hi;
-                if (cnd) atomicAdd(&sm.sh[flat_bin(key, bin_base, shift)], 1u);
-                if (ev != fast_ev) {                             // equal score words, the index decides: settle the bit now
-                    unsigned long long* wp = reinterpret_cast<unsigned long long*>(keep_bits + (idx >> 6));
-                    if (ev) atomicAnd(wp, ~(1ull << (idx & 63))); else atomicOr(wp, 1ull << (idx & 63));
-                }
+                cnd = classify(xs ? xs[p] : __ldg(s + base + p), (uint32_t)base + (uint32_t)p, key);
             }
             const unsigned cdb = __ballot_sync(0xffffffffu, cnd);
             if (cnd) sm.wb[nbuf + __popc(cdb & ((1u << lane) - 1u))] = key;

@@ -200,6 +200,11 @@ void launch_select_cache_sample(const CacheView& cv, const SelectBuffers& sb, lo
                                 long long k_evict, int skip_newest, int distrust_sample, cudaStream_t st);
 void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
                               int32_t* compact_cursor, cudaStream_t st);
+// ... or in three parts: the filter pass may leave out the newest entry of every pool as well (skip_newest) and run beside
+// the gate; the finish then classifies those entries (newest_left_out) and ranks the candidates.
+void launch_select_cache_filter(const CacheView& cv, const SelectBuffers& sb, long long t, int skip_newest, cudaStream_t st);
+void launch_select_cache_finish(const CacheView& cv, const SelectBuffers& sb, long long t, long long k_evict,
+                                int32_t* compact_cursor, int newest_left_out, cudaStream_t st);
 // Rank-local stages of the selection of a sequence whose layers are sharded over ranks (see select.cu).
 int shard_sample_cap();
 void launch_shard_sample(const CacheView& cv, const SelectBuffers& sb, long long t, long long n_total, u64* keys_out,

@@ -663,6 +663,8 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     if (early_sample) {
         CUDA_TRY(cudaStreamWaitEvent(h->side2, h->ev_append, 0));
         launch_select_cache_sample(h->cv, h->sb, h->tokens[0], h->entries, kev, 1, h->test_hooks & TRIMKV_TEST_DISTRUST_SAMPLE, h->side2);
+        // ... and so does the filter pass over every entry but the newest of each pool: only those wait for the gate
+        launch_select_cache_filter(h->cv, h->sb, h->tokens[0], 1, h->side2);
         CUDA_TRY(cudaEventRecord(h->ev_sample, h->side2));
     }
     if (!x) {
@@ -672,7 +674,7 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     if (early_sample) {
         CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_sample, 0));
         if (h->prof.on) h->prof.mark(PH_SELECT, 0, sd);
-        launch_select_cache_rest(h->cv, h->sb, h->tokens[0], kev, h->cursor, sd);
+        launch_select_cache_finish(h->cv, h->sb, h->tokens[0], kev, h->cursor, 1, sd);
         if (h->prof.on) h->prof.mark(PH_SELECT, 1, sd);
     } else if (kev > 0) {
         select_impl(h, kev, sd);
