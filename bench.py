@@ -478,6 +478,15 @@ def measure_workload(args, w, K, W, rank, world, local_rank, main):
     assert int(lens[0].sum()) == min(w.budget_entries, entries), "budget invariant violated"
     assert per_pool == 0 or int(lens.max()) <= per_pool
 
+    modality = None
+    if w.visual_period > 0 and rank == 0:
+        # what the global budget kept of each modality (sequence 0): a token's modality follows from its position and
+        # the workload's layout; the cache itself stores no modality tag
+        pos = torch.cat([cache.kept(0, l, h, int(lens[0, l, h]) + 1) for l in range(w.layers) for h in range(w.kv_heads)])
+        vis = workloads.is_visual(w, pos.to(torch.int64) - 1)
+        prompt = workloads.is_visual(w, torch.arange(tokens_seen + done_steps[0]))
+        modality = {"kept_entries": int(pos.numel()), "kept_visual_entries": int(vis.sum()),
+                    "kept_visual_share": float(vis.float().mean()), "visual_share_of_tokens_seen": float(prompt.float().mean())}
     peak, peak_kind = load_peaks()
     ab = algorithmic_bytes(w, entries + w.layers * w.kv_heads)
     if args.retention_bias:                                        # lambda and position of every entry ride along
@@ -496,7 +505,7 @@ def measure_workload(args, w, K, W, rank, world, local_rank, main):
            "phases": {k: v[0] / KP for k, v in phases.items() if v[1]}, "peak": peak, "peak_kind": peak_kind,
            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "steps": KE, "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "breakdown": breakdown},
-           "per_pool": per_pool, "seqs": [seq_lo, seq_hi], "cpu": None}
+           "per_pool": per_pool, "seqs": [seq_lo, seq_hi], "cpu": None, "modality": modality}
     if main and rank == 0 and not args.no_cpu_baseline:
         res["cpu"] = oracle_beside_gpu(cache, w, per_layer, w_g, lambda i: step_inputs(done_steps[0] + i),
                                        tokens_seen + done_steps[0])
@@ -550,7 +559,7 @@ def run_ours(args, w):
                                    "frac_of_sustained": (attn_stats["last_flops"] / (attn_stats["last_ms"] * 1e-3) / 1e12 / tpk["sustained"])
                                                         if attn_stats["last_ms"] > 0 else None,
                                    "flops": "causal: 4 d per (query head, visible entry); masked tile parts not counted"}},
-                   "earlier_turn_decode_ms_per_step": r["early_decode"]},
+                   "earlier_turn_decode_ms_per_step": r["early_decode"], "kept_by_modality": r["modality"]},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": r["achieved"], "peak": peak, "unit": "GB/s",
                      "frac": r["achieved"] / peak, "peak_kind": f"of {peak_kind} (a copy's read + write rate: a read-only stream can exceed it)",
                      "traffic": recorded_traffic(w.name) if default_config else None,
@@ -587,6 +596,8 @@ def other_workloads(args):
                      "e2e_ms_per_step": r["e2e"]["ms_per_step"], "e2e_tokens_per_s": r["e2e"]["value"],
                      "gpu_launches": r["launches"], "clocks": r["clocks"], "setup_s": round(r["t_setup"], 1),
                      "earlier_turn_decode_ms_per_step": r["early_decode"]}
+        if r["modality"]:
+            out[name]["kept_by_modality"] = r["modality"]
     rows, clocks = select_sweep_rows(args, (20, 24, 28), 5, 3)
     out["select_sweep"] = {"rows": rows, "clocks": clocks, "l2": "flushed between timed calls",
                            "what": "trimkv_select_topk over n fp32 scores uniform in [-8, 0]; gbs counts one pass of 4 n bytes per call"}
