@@ -368,7 +368,6 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
         st->cand_hi = hi;
         st->n_below = 0;
         st->cand_count = 0;
-        st->cand_expected = 0;
         st->resolved = 0;
         st->passes = ns;
     }
@@ -377,16 +376,15 @@ bracket_kernel(SelState* __restrict__ sel, const u64* __restrict__ sample, long 
 constexpr int SHARD_TAG_SHIFT = 56;      // a sharded selection tags a candidate's slot with its rank above this bit
 
 // ------------------------------------------------------------------ exact ranking of the candidates
-// One CTA per sequence.  STRICT (histogram path): the candidate range is known to hold the k-th key; any
-// inconsistency is an internal error.  Otherwise (sample-bracket path): an inconsistent count means the range
-// missed; resolved stays 0 and (redo_inline) this CTA redoes its sequence exactly, or the caller runs its own fallback.
+// One CTA per sequence.  An inconsistent count (the k-th key is not among the candidates, or the list overflowed) means
+// the sampled range missed: resolved stays 0 and (redo_inline) this CTA redoes its sequence exactly, or the caller runs
+// its own fallback.
 __device__ void redo_body(CacheSrc src, SelState* __restrict__ sel, u64* __restrict__ evict_mask, long long mask_stride,
                           long long k_evict, int32_t* err);
 
-template <bool STRICT>
 __global__ void __launch_bounds__(1024)
 resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long cand_cap, u64* __restrict__ evict_mask,
-               long long mask_stride, long long k_evict, unsigned next_aim, long long* __restrict__ stats,
+               long long mask_stride, long long k_evict, long long* __restrict__ stats,
                int32_t* __restrict__ cursor, int32_t* err, CacheSrc src, int redo_inline, int my_rank = -1) {
     constexpr int DB = 11, NBIN = 1 << DB;
     __shared__ unsigned hist[NBIN];
@@ -401,25 +399,20 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
     const long long craw = (long long)st->cand_count;
     const long long C = min(craw, cand_cap);
     long long r = k_evict - st->n_below;
-    const bool ok = r >= 0 && r <= C && craw <= cand_cap && (!STRICT || (long long)st->cand_expected == craw);
+    const bool ok = r >= 0 && r <= C && craw <= cand_cap;
     const int sample_n = st->passes;
     if (!ok) {
-        if (STRICT) {
-            if (tid == 0) latch_error(err, TRIMKV_E_STATE);
-            r = r < 0 ? 0 : (r > C ? C : r);
-        } else {
-            if (tid == 0) {
-                st->resolved = 0;
-                st->sample_count = 0;
-                if (stats) { stats[b * 4 + 0] = 1; stats[b * 4 + 1] = C; stats[b * 4 + 2] = k_evict; stats[b * 4 + 3] = sample_n; }
-                if (cursor) cursor[b] = 0;
-            }
-            // the bracket missed (next to never): this CTA redoes its sequence exactly, at once, instead of a further
-            // kernel that every call would have to launch just to find nothing to do
-            __syncthreads();
-            if (redo_inline) redo_body(src, sel, evict_mask, mask_stride, k_evict, err);
-            return;
+        if (tid == 0) {
+            st->resolved = 0;
+            st->sample_count = 0;
+            if (stats) { stats[b * 4 + 0] = 1; stats[b * 4 + 1] = C; stats[b * 4 + 2] = k_evict; stats[b * 4 + 3] = sample_n; }
+            if (cursor) cursor[b] = 0;
         }
+        // the bracket missed (next to never): this CTA redoes its sequence exactly, at once, instead of a further
+        // kernel that every call would have to launch just to find nothing to do
+        __syncthreads();
+        if (redo_inline) redo_body(src, sel, evict_mask, mask_stride, k_evict, err);
+        return;
     }
     u64 tau = 0ull;
     if (r > 0) {
@@ -539,30 +532,14 @@ resolve_kernel(SelState* __restrict__ sel, Cand* __restrict__ cand, long long ca
     __syncthreads();
     if (tid == 0) {
         if (stats) {
-            stats[b * 4 + 0] = STRICT ? st->passes : 0;
+            stats[b * 4 + 0] = 0;
             stats[b * 4 + 1] = C;
             stats[b * 4 + 2] = k_evict;
-            stats[b * 4 + 3] = STRICT ? st->shift : sample_n;
+            stats[b * 4 + 3] = sample_n;
         }
-        if (STRICT) {
-            // centre the next call's first histogram on this threshold; aim for ~next_aim candidates
-            int shift = st->shift;
-            const int want = 31 - __clz((int)max(next_aim, 1u));
-            const int have = 31 - __clz((int)max((unsigned)min(C, 0x7fffffffLL), 1u));
-            shift += want - have;
-            shift = shift < 0 ? 0 : (shift > INIT_SHIFT ? INIT_SHIFT : shift);
-            const u64 half = (u64)(REG_BINS / 2) << shift;
-            st->lo = tau > half ? tau - half : 0ull;
-            st->shift = shift;
-            st->resolved = 0;
-            st->passes = 0;
-        } else {
-            st->resolved = 1;
-        }
+        st->resolved = 1;
         st->cand_count = 0;
         st->sample_count = 0;
-        st->kmin = ~0ull;
-        st->kmax = 0ull;
         if (cursor) cursor[b] = 0;
     }
 }
@@ -791,8 +768,8 @@ __global__ void state_init_kernel(SelState* sel, int B) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     SelState s;
-    s.lo = 0ull; s.kmin = ~0ull; s.kmax = 0ull; s.cand_lo = 0ull; s.cand_hi = 0ull; s.n_below = 0;
-    s.shift = INIT_SHIFT; s.resolved = 0; s.passes = 0; s.cand_count = 0; s.cand_expected = 0; s.sample_count = 0;
+    s.cand_lo = 0ull; s.cand_hi = 0ull; s.n_below = 0;
+    s.resolved = 0; s.passes = 0; s.cand_count = 0; s.sample_count = 0;
     sel[b] = s;
 }
 
@@ -1027,7 +1004,7 @@ void launch_shard_resolve(const CacheView& cv, const SelectBuffers& sb, const vo
     CacheSrc none;
     none.cv = cv;
     none.t1 = 0;
-    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u, sb.stats,
+    resolve_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, sb.stats,
                                                  compact_cursor, cv.err, none, 0, rank);
     shard_export_resolved_kernel<<<(cv.B + 127) / 128, 128, 0, st>>>(sb.sel, resolved_out, cv.B);
     count_launch(3);
@@ -1116,7 +1093,7 @@ void launch_select_cache_finish(const CacheView& cv, const SelectBuffers& sb, lo
         filter_newest_kernel<<<(pools + 127) / 128, 128, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
         count_launch();
     }
-    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
+    resolve_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict,
                                                  sb.stats, compact_cursor, cv.err, src, 1);
     count_launch();
 }
@@ -1128,7 +1105,7 @@ void launch_select_cache_rest(const CacheView& cv, const SelectBuffers& sb, long
     src.t1 = t + 1;
     dim3 grid(grid_x_for(cv.P_seq, cv.B), cv.B);
     filter_kernel<CacheSrc, true><<<grid, 256, 0, st>>>(src, sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, cv.err);
-    resolve_kernel<false><<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict, 0u,
+    resolve_kernel<<<cv.B, 1024, 0, st>>>(sb.sel, sb.cand, sb.cand_cap, cv.evict_mask, cv.P_seq, k_evict,
                                                  sb.stats, compact_cursor, cv.err, src, 1);
     count_launch(2);
 }

@@ -5,7 +5,8 @@
 // One pass over the scores:
 //   1. flat_bracket_kernel (one CTA): ranks a stratified sample of the scores (one hashed position per stratum) and
 //      brackets the k-th smallest key between two sample keys, several standard deviations of the sample rank apart;
-//      the sample key at the expected rank (`mid`) serves as a first estimate of the threshold.
+//      the bracket's midpoint (`mid`) serves as a first estimate of the threshold.  (1b, largest arrays only:
+//      flat_refine_kernel narrows the bracket with a 32 times larger sample gathered by many CTAs.)
 //   2. flat_main_kernel (whole GPU, reads the scores once): writes the keep bits against `mid`, counts the keys below
 //      the bracket, appends the keys inside it to a candidate list and bins them (shared-memory histogram of 4096 equal
 //      bins over the bracket); the last CTA finds the bin of the k-th key: a fine bracket with a few thousand keys.
@@ -391,9 +392,9 @@ flat_refine_kernel(const float* __restrict__ s, long long n, long long k_evict, 
 }
 
 // ------------------------------------------------------------------ 2. the pass over the scores
-constexpr int FBUF = 512;         // candidate keys a warp stages before it takes a slice of the global list (>= 32 * FJ)
+constexpr int FBUF = 128;         // candidate keys a warp stages before it takes a slice of the global list
 constexpr int FJ = 16;            // ballots per warp trip: a warp takes 32 * FJ = 512 consecutive scores
-constexpr int MAIN_WARPS = 16;
+constexpr int MAIN_WARPS = 24;
 constexpr int MAIN_THREADS = MAIN_WARPS * 32;
 
 // Appends the warp's staged keys to the candidate list (one atomic per flush).  Keys beyond the list's capacity are
@@ -414,14 +415,17 @@ __device__ void flat_pick_bin(FlatState* st, const uint32_t* hist, long long k_e
     __shared__ int s_bin;
     __shared__ unsigned long long s_before;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int PERT = FB / MAIN_THREADS;
+    constexpr int PICK_THREADS = 512, PERT = FB / PICK_THREADS;          // the first 512 threads hold eight bins each
+    static_assert(MAIN_THREADS >= PICK_THREADS, "the scan needs 512 threads");
     unsigned v[PERT];
     unsigned long long local = 0;
 #pragma unroll
     for (int i = 0; i < PERT; ++i) {
         v[i] = 0u;
+        if (tid < PICK_THREADS) {
 #pragma unroll
-        for (int r = 0; r < HREP; ++r) v[i] += __ldcg(hist + r * FB + tid * PERT + i);
+            for (int r = 0; r < HREP; ++r) v[i] += __ldcg(hist + r * FB + tid * PERT + i);
+        }
         local += v[i];
     }
     unsigned long long incl = local;
@@ -443,7 +447,7 @@ __device__ void flat_pick_bin(FlatState* st, const uint32_t* hist, long long k_e
         unsigned long long cum = excl;
 #pragma unroll
         for (int i = 0; i < PERT; ++i) {
-            if ((unsigned long long)r1 > cum && (unsigned long long)r1 <= cum + v[i]) { s_bin = tid * PERT + i; s_before = cum; }
+            if (tid < PICK_THREADS && (unsigned long long)r1 > cum && (unsigned long long)r1 <= cum + v[i]) { s_bin = tid * PERT + i; s_before = cum; }
             cum += v[i];
         }
     }
@@ -590,11 +594,11 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
         }
         __syncwarp();
         const int tot = (int)*((volatile unsigned*)sm.ecount);
-        if (nbuf + tot > FBUF) {
-            flat_flush(sm.wb, nbuf, st, cand, cand_cap);
-            nbuf = 0;
-        }
         for (int e0 = 0; e0 < tot; e0 += 32) {
+            if (nbuf + 32 > FBUF) {                              // room for this batch (warp-uniform)
+                flat_flush(sm.wb, nbuf, st, cand, cand_cap);
+                nbuf = 0;
+            }
             const int e = e0 + lane;
             bool cnd = false;
             u64 key = 0ull;

@@ -12,27 +12,16 @@ namespace tkv {
 
 // ------------------------------------------------------------------ constants
 constexpr int PAGE = 64;                 // entries per page
-constexpr int NB = 4096;                 // histogram bins: 0 = below range, 1..NB-2 regular, NB-1 = above range (not counted)
-constexpr int REG_BINS = NB - 2;
-constexpr int ZOOM_BITS = 11;            // a zoom maps the surviving key range onto <= 2^11 regular bins
-constexpr int MAX_HIST_PASSES = 3;       // histogram passes per selection; the last one resolves unconditionally
-constexpr int INIT_SHIFT = 64 - ZOOM_BITS;
-
 typedef unsigned long long u64;
 
-// Per-sequence selection state (device resident, persists between calls so that the first
-// histogram pass of a call can be centred on the previous call's threshold).
+// Per-sequence state of the cache's selection (device resident).
 struct SelState {
-    u64 lo;            // key at the lower edge of regular bin 1
-    u64 kmin, kmax;    // min / max key seen during the running pass
     u64 cand_lo;       // candidate range [cand_lo, cand_hi]: keys below are evicted, above are kept
     u64 cand_hi;
     long long n_below; // number of keys < cand_lo
-    int shift;         // bin width = 2^shift keys
-    int resolved;      // 1 once the candidate range is final for this call
-    int passes;        // histogram passes run in this call (sample-bracket path: keys sampled)
+    int resolved;      // 1 once the threshold of this call is settled
+    int passes;        // keys sampled in this call (reported in the statistics)
     unsigned int cand_count;   // candidates appended by the filter pass
-    unsigned int cand_expected;
     unsigned int sample_count; // keys drawn by the sampling pass of this call
 };
 
@@ -86,12 +75,6 @@ __device__ __forceinline__ float horizon_term_f32(float lam, int horizon) {
     float acc = 1.0f;
     for (int k = 1; k < horizon; ++k) acc += expf((float)k * lam);
     return logf(acc);
-}
-
-__device__ __forceinline__ int bin_of(u64 key, u64 lo, int shift) {
-    if (key < lo) return 0;
-    u64 idx = (key - lo) >> shift;
-    return idx >= (u64)REG_BINS ? NB - 1 : (int)idx + 1;
 }
 
 // ------------------------------------------------------------------ cache geometry
@@ -183,8 +166,6 @@ void launch_gate_gemm_tc(GateTcState* s, const float* x, int R, int layer, float
 
 struct SelectBuffers {
     SelState* sel;        // [B]
-    uint32_t* hist;       // [B][NB]
-    unsigned int* done;   // [B]
     Cand* cand;           // [B][cand_cap]
     long long cand_cap;
     long long* stats;     // [B][4]

@@ -160,8 +160,6 @@ trimkv_status init_cache_state(trimkv* h) {
     CUDA_TRY(cudaMemset(h->cv.len, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->cv.err, 0, sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->cv.append_failed, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
-    CUDA_TRY(cudaMemset(h->sb.hist, 0, (size_t)h->B * NB * sizeof(uint32_t)));
-    CUDA_TRY(cudaMemset(h->sb.done, 0, (size_t)h->B * sizeof(unsigned)));
     CUDA_TRY(cudaMemset(h->sb.stats, 0, (size_t)h->B * 4 * sizeof(long long)));
     CUDA_TRY(cudaMemset(h->cursor, 0, (size_t)h->B * sizeof(int32_t)));
     CUDA_TRY(cudaMemset(h->ab.pool_done, 0, (size_t)h->B * h->L * h->H * sizeof(int32_t)));
@@ -376,8 +374,6 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     SelectBuffers& sb = h->sb;
     sb.cand_cap = h->n_max;
     A(dev_alloc(h, &sb.sel, (size_t)h->B, true));
-    A(dev_alloc(h, &sb.hist, (size_t)h->B * NB, true));
-    A(dev_alloc(h, &sb.done, (size_t)h->B, true));
     A(dev_alloc(h, &sb.cand, (size_t)h->B * sb.cand_cap, false));
     A(dev_alloc(h, &sb.stats, (size_t)h->B * 4, true));
     A(dev_alloc(h, &sb.sample, (size_t)h->B * 4096, false));
