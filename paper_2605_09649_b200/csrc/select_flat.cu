@@ -523,7 +523,7 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
     const long long my_trips = c0 < nfull ? (nfull - c0 + W - 1) / W : 0;
     const bool lane0 = lane == 0;
     int nbuf = 0;                                // warp-uniform fill of the staging buffer
-    long long ev_fast = 0;                       // lanes < 8: scores of their words with the keep bit clear
+    unsigned ev_fast = 0;                        // lanes < 8: scores of their words with the keep bit clear
     int adj = 0;                                 // per lane: (inside scores below lo) - (inside scores with the keep bit clear)
     bool bad = false, failed = false;
 
@@ -613,13 +613,14 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
         __syncwarp();
     };
     // the 16 ballots of a trip sit in shared memory (written by lane 0); lanes 0..7 turn them into keep words
-    auto write_words = [&](long long word0, long long live_scores) {
+    // (full: a whole trip of 512 scores, every word inside the array)
+    auto write_words = [&](long long word0, int live_scores, bool full) {
         __syncwarp();
-        if (lane < FJ / 2 && word0 + lane < words) {
+        if (lane < FJ / 2 && (full || word0 + lane < words)) {
             const u64 wv = *reinterpret_cast<const u64*>(sm.words + 2 * lane);
             keep_bits[word0 + lane] = wv;
-            const long long lb = live_scores - 64LL * lane;
-            ev_fast += (lb >= 64 ? 64 : (lb > 0 ? lb : 0)) - __popcll(wv);
+            const int lb = full ? 64 : min(64, max(0, live_scores - 64 * lane));
+            ev_fast += (unsigned)(lb - __popcll(wv));
         }
     };
 
@@ -645,7 +646,7 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
 #pragma unroll
             for (int j = 0; j < FJ; j += 4) *reinterpret_cast<uint4*>(sm.words + j) = make_uint4(kb[j], kb[j + 1], kb[j + 2], kb[j + 3]);
         }
-        write_words(c * (FJ / 2), TRIP);
+        write_words(c * (FJ / 2), TRIP, true);
         handle_inside(m, c * TRIP, xs);
         __syncwarp();                                            // every lane is done with this stage before it is refilled
     }
@@ -666,13 +667,13 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
             const unsigned kb = __ballot_sync(0xffffffffu, live && !(xv < mid_lt));
             if (lane0) sm.words[j] = kb;
         }
-        write_words(nfull * (FJ / 2), rem);
+        write_words(nfull * (FJ / 2), (int)rem, false);
         handle_inside(m, base, nullptr);
     }
     if (nbuf > 0) flat_flush(sm.wb, nbuf, st, cand, cand_cap);
     if (bad) latch_error(status, TRIMKV_E_NONFINITE);
     // keys below lo = (scores whose keep bit the fast compare cleared) corrected by the scores classified exactly
-    long long nb = ev_fast + (long long)adj;
+    long long nb = (long long)ev_fast + (long long)adj;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) nb += __shfl_xor_sync(0xffffffffu, nb, o);
     if (lane0 && nb) atomicAdd(&st->n_below, (unsigned long long)nb);
