@@ -674,6 +674,33 @@ def test_select_topk_exact_fallbacks_match_full_sort():
         np.testing.assert_array_equal(got, _oracle_keep_bits(s.cpu().numpy(), n - k_evict))
 
 
+@pytest.mark.parametrize("kind", ["ascending", "descending", "periodic", "few_values", "wide_range", "spikes"])
+def test_select_topk_structured_inputs_match_full_sort(kind):
+    """Inputs a sample could misjudge: sorted scores, a period that matches the sampling strata, a handful of distinct
+    values, magnitudes spread over many binades, rare large spikes.  The result never depends on the sample: whichever
+    path decides (bracket, crowded-bin fallback, full fallback), the kept set is the full sort's."""
+    n = (1 << 21) + 777
+    base = workloads.selection_scores(n, seed=21, device=DEV)
+    idx = torch.arange(n, device=DEV)
+    if kind == "ascending":
+        s = torch.sort(base).values
+    elif kind == "descending":
+        s = torch.sort(base, descending=True).values
+    elif kind == "periodic":
+        s = -8.0 * ((idx % 256).float() / 256.0) + base * 1e-3           # period = the sampling stratum of this size
+    elif kind == "few_values":
+        s = torch.round(base)                                            # nine distinct values, huge tie groups
+    elif kind == "wide_range":
+        s = -torch.exp(base * 8.0 + 20.0)                                # -e^-44 .. -e^20: ~90 binades
+    else:
+        s = torch.where(idx % 1009 == 0, base * 1e6, base * 1e-6)
+    s = s.contiguous()
+    s_np = s.cpu().numpy()
+    for k in (1, n // 8, n // 2, n - 512):
+        got, stats = _select_with_stats(s, k)
+        np.testing.assert_array_equal(got, _oracle_keep_bits(s_np, k), err_msg=f"{kind} k={k} stats={stats}")
+
+
 def test_select_topk_rejects_nan_and_bad_args():
     s = torch.tensor([0.0, float("nan"), -1.0, -2.0] * 64, device=DEV)
     bits, status = binding.select_topk(s, 100)
