@@ -386,6 +386,11 @@ def measure_workload(args, w, K, W, rank, world, local_rank, main):
         cache.decode_step_all(Kt, Vt, Q, out, x=X)
         done_steps[0] += 1
 
+    # the decode loop runs on the handle's own highest-priority stream (a serving loop would do the same): the step's
+    # attention chain then needs no hand-off from and to the caller's stream
+    torch.cuda.synchronize()
+    loop_stream = cache.step_stream()
+    torch.cuda.set_stream(loop_stream)
     for i in range(W):
         step(i)
     torch.cuda.synchronize()
@@ -509,6 +514,8 @@ def measure_workload(args, w, K, W, rank, world, local_rank, main):
     if main and rank == 0 and not args.no_cpu_baseline:
         res["cpu"] = oracle_beside_gpu(cache, w, per_layer, w_g, lambda i: step_inputs(done_steps[0] + i),
                                        tokens_seen + done_steps[0])
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
     cache.close()
     del cache, inputs, host_in
     torch.cuda.empty_cache()

@@ -171,6 +171,12 @@ TRIMKV_API trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x
  * caller's stream instead (same results; for per-kernel timing).  Synchronises. */
 TRIMKV_API trimkv_status trimkv_set_overlap(trimkv_t* h, int enable);
 
+/* The handle's own highest-priority stream (a cudaStream_t), on which trimkv_decode_step_all runs its K/V append, attention
+ * and compaction.  A caller that passes this stream -- or any stream of its own created with the device's highest
+ * priority -- as `stream` saves the step the two hand-offs between the caller's stream and that one (a few microseconds
+ * each, on the critical path of short steps).  Owned by the handle; do not destroy it. */
+TRIMKV_API void* trimkv_step_stream(trimkv_t* h);
+
 /* Changes the horizon h = T - t of the retention score (Sec. 4.2, Eq. (global_score): ln G~ = (t+1-i) ln beta +
  * ln sum_{k<h} beta^k; h = 1 gives the myopic score beta^(t+1-i), h = 0 stands for h -> infinity, the limit
  * beta^(t+1-i) / (1 - beta) stated below the equation) for an existing cache, e.g. between eviction rounds: the

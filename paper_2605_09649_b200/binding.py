@@ -26,7 +26,7 @@ EXPORTS = [
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static", "trimkv_set_test_hooks",
-    "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
+    "trimkv_step_stream", "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
     "trimkv_shard_resolve", "trimkv_shard_hist", "trimkv_shard_digit", "trimkv_shard_mark", "trimkv_shard_compact",
 ]
 
@@ -88,6 +88,8 @@ def lib() -> C.CDLL:
     L.trimkv_profile.argtypes = [vp, i32]
     L.trimkv_set_overlap.argtypes = [vp, i32]
     L.trimkv_set_test_hooks.argtypes = [vp, i32]
+    L.trimkv_step_stream.argtypes = [vp]
+    L.trimkv_step_stream.restype = vp
     L.trimkv_shard_sample_cap.argtypes = []
     L.trimkv_shard_sample.argtypes = [vp, i64, i64, vp, vp, vp]
     L.trimkv_shard_bracket.argtypes = [vp, i32, vp, vp, i64, i64, vp]
@@ -277,6 +279,10 @@ class TrimKV:
     def set_test_hooks(self, flags: int):
         """Testing aids of this handle (TEST_* flags; 0 = normal operation)."""
         _check(lib().trimkv_set_test_hooks(self._h, int(flags)))
+
+    def step_stream(self) -> "torch.cuda.ExternalStream":
+        """The handle's highest-priority stream as a torch stream: decode steps enqueued on it skip two stream hand-offs."""
+        return torch.cuda.ExternalStream(int(lib().trimkv_step_stream(self._h)))
 
     def set_overlap(self, enable: bool):
         _check(lib().trimkv_set_overlap(self._h, 1 if enable else 0))

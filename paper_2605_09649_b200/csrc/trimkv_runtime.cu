@@ -121,6 +121,7 @@ struct trimkv {
     cudaStream_t side_hi = nullptr;                                 // `side` at the priority of `fast` (gate-heavy steps)
     bool overlap = true;
     int test_hooks = 0;              // TRIMKV_TEST_* switches of this handle
+    int prio_hi = 0;                 // the device's highest stream priority
     bool shard = false;              // the handle holds a slice of the layers of sequences sharded over ranks
     char* pool_stage = nullptr;      // device staging of trimkv_get_pool, grown on demand
     size_t pool_stage_bytes = 0;
@@ -419,6 +420,7 @@ trimkv_status trimkv_create_ex(const trimkv_config* cfg, trimkv_t** out) {
     if (s == TRIMKV_OK) {
         int prio_lo = 0, prio_hi = 0;
         cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);     // numerically lower = higher priority
+        h->prio_hi = prio_hi;
         if (cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_lo) != cudaSuccess ||
             cudaStreamCreateWithPriority(&h->fast, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
             cudaStreamCreateWithPriority(&h->side2, cudaStreamNonBlocking, prio_lo) != cudaSuccess ||
@@ -607,10 +609,15 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     // 0.169 -> 0.155; llama8b_32k, where the gate is 7 % of the traffic, loses 9 us that way and keeps the low priority).
     const double kv_bytes = (double)(h->entries + (long long)h->L * h->H) * h->B * 2.0 * h->cv.row_bytes;
     const bool gate_heavy = x && (double)h->L * h->D * h->dg * 4.0 > 0.15 * kv_bytes;
-    cudaStream_t sd = two ? (gate_heavy ? h->side_hi : h->side) : st, fs = two ? h->fast : st;
+    // A caller whose own stream already has the highest priority gets the fast chain on that stream: the two hand-offs
+    // between its stream and `fast` (fork and join, a few microseconds each on the critical path) fall away.
+    int st_prio = 0;
+    const bool st_is_fast = two && st != nullptr &&
+                            (st == h->fast || (cudaStreamGetPriority(st, &st_prio) == cudaSuccess && st_prio == h->prio_hi));
+    cudaStream_t sd = two ? (gate_heavy ? h->side_hi : h->side) : st, fs = (two && !st_is_fast) ? h->fast : st;
     if (two) {
         CUDA_TRY(cudaEventRecord(h->ev_fork, st));
-        CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
+        if (!st_is_fast) CUDA_TRY(cudaStreamWaitEvent(fs, h->ev_fork, 0));
         CUDA_TRY(cudaStreamWaitEvent(sd, h->ev_fork, 0));
     }
     if (host) {
@@ -686,8 +693,10 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
         if (h->prof.on) h->prof.mark(PH_D2H, 1, fs);
     }
     if (two) {
-        CUDA_TRY(cudaEventRecord(h->ev_done, fs));
-        CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
+        if (!st_is_fast) {
+            CUDA_TRY(cudaEventRecord(h->ev_done, fs));
+            CUDA_TRY(cudaStreamWaitEvent(st, h->ev_done, 0));
+        }
     }
     if (s != TRIMKV_OK) return s;
     CUDA_TRY(cudaGetLastError());
@@ -914,6 +923,8 @@ trimkv_status trimkv_set_test_hooks(trimkv_t* h, int flags) {
     else tkv::g_test_hooks.store(flags, std::memory_order_relaxed);
     return TRIMKV_OK;
 }
+
+void* trimkv_step_stream(trimkv_t* h) { return h ? (void*)h->fast : nullptr; }
 
 trimkv_status trimkv_set_overlap(trimkv_t* h, int enable) {
     if (check_handle(h)) return TRIMKV_E_ARG;
