@@ -203,6 +203,13 @@ TRIMKV_API trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int he
  *  entries evicted, keys sampled}.  Synchronises. */
 TRIMKV_API trimkv_status trimkv_get_select_stats(trimkv_t* h, int64_t* out_host);
 
+/* Self-check of the cache's bookkeeping, for tests and debugging (the role a memory checker would play): every pool's
+ * block table against the page records and back, the free stack against the page records, page accounting (owned + free
+ * = all pages of a sequence), positions within 1..tokens and no NaN retention term among the live entries.  Synchronises,
+ * allocates a few bytes of scratch, and returns TRIMKV_E_STATE with the violated rules in trimkv_last_error, else the
+ * latched device status. */
+TRIMKV_API trimkv_status trimkv_check_invariants(trimkv_t* h);
+
 /* Waits for the handle's enqueued work (device synchronise) and returns the latched device error,
  * TRIMKV_OK if none.  The latch is cleared by trimkv_reset. */
 TRIMKV_API trimkv_status trimkv_sync_status(trimkv_t* h);

@@ -26,7 +26,7 @@ EXPORTS = [
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static", "trimkv_set_test_hooks",
-    "trimkv_step_stream", "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
+    "trimkv_step_stream", "trimkv_check_invariants", "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
     "trimkv_shard_resolve", "trimkv_shard_hist", "trimkv_shard_digit", "trimkv_shard_mark", "trimkv_shard_compact",
 ]
 
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
     L.trimkv_set_overlap.argtypes = [vp, i32]
     L.trimkv_set_test_hooks.argtypes = [vp, i32]
     L.trimkv_step_stream.argtypes = [vp]
+    L.trimkv_check_invariants.argtypes = [vp]
+    L.trimkv_check_invariants.restype = i32
     L.trimkv_step_stream.restype = vp
     L.trimkv_shard_sample_cap.argtypes = []
     L.trimkv_shard_sample.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -265,6 +267,10 @@ class TrimKV:
 
     def sync_status(self):
         _check(lib().trimkv_sync_status(self._h))
+
+    def check_invariants(self):
+        """Self-check of the cache's bookkeeping (raises TrimkvError E_STATE naming the violated rules)."""
+        _check(lib().trimkv_check_invariants(self._h))
 
     PHASES = ["gate", "append", "h2d_kvq", "attn_main", "d2h_out", "select", "compact", "h2d_x"]
 

@@ -1,6 +1,8 @@
 // Paged per-(layer, head) KV pools (Sec. 4.2 "Implementation details": fixed-size pages, one block
 // table per head, variable logical length per head): append of new tokens and compaction after an
 // eviction round.
+#include <algorithm>
+
 #include "trimkv_internal.cuh"
 
 namespace tkv {
@@ -327,7 +329,68 @@ rehorizon_kernel(CacheView cv, int horizon) {
     cv.c[slot] = horizon_term_f32(cv.lam[slot], horizon);
 }
 
+// Self-check of the cache's bookkeeping (tests run it where a memory checker would otherwise be used): every pool's
+// block table against the page records, every owned page against its pool, the free stack against the page records,
+// positions and retention terms of live entries.  viol: OR of the violated rules; owned [B]: pages with an owner.
+//   1 page id out of range   2 page record disagrees with the pool   4 owned page not referenced by its pool
+//   8 free-stack entry owned or out of range   16 position outside 1..tokens   64 NaN retention term
+__global__ void check_kernel(CacheView cv, long long tokens, unsigned* __restrict__ viol, unsigned* __restrict__ owned) {
+    const long long gid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    const int LH = cv.L * cv.H;
+    unsigned v = 0;
+    if (blockIdx.y == 0) {                                    // pools
+        if (gid < (long long)cv.B * LH) {
+            const int b = (int)(gid / LH), pool_local = (int)(gid % LH);
+            const int n = cv.len[gid];
+            if (n < 0) v |= 2;
+            for (int lp = 0; lp * PAGE < n; ++lp) {
+                const int page = cv.block_table[(size_t)gid * cv.maxpp + lp];
+                if (page < 0 || page >= cv.P_seq) { v |= 1; continue; }
+                const int4 ow = cv.owner[(size_t)b * cv.P_seq + page];
+                if (ow.x != pool_local || ow.y != lp || ow.z != min(PAGE, n - lp * PAGE)) v |= 2;
+            }
+        }
+    } else if (blockIdx.y == 1) {                             // pages
+        if (gid < (long long)cv.B * cv.P_seq) {
+            const int b = (int)(gid / cv.P_seq);
+            const int4 ow = cv.owner[gid];
+            if (ow.x >= 0) {
+                atomicAdd(owned + b, 1u);
+                if (ow.x >= LH) v |= 4;
+                else {
+                    const long long pool = (long long)b * LH + ow.x;
+                    const int n = cv.len[pool];
+                    if (ow.y < 0 || (long long)ow.y * PAGE >= n || cv.block_table[pool * cv.maxpp + ow.y] != (int)(gid % cv.P_seq)) v |= 4;
+                    for (int off = 0; off < ow.z && off < PAGE; ++off) {
+                        const size_t slot = (size_t)gid * PAGE + off;
+                        const int pos = cv.pos[slot];
+                        if (pos < 1 || pos > tokens) v |= 16;
+                        if (cv.lam[slot] != cv.lam[slot] || cv.c[slot] != cv.c[slot]) v |= 64;
+                    }
+                }
+            }
+        }
+    } else {                                                  // free stacks
+        if (gid < (long long)cv.B * cv.P_seq) {
+            const int b = (int)(gid / cv.P_seq);
+            const long long i = gid % cv.P_seq;
+            if (i < cv.free_count[b]) {
+                const int page = cv.free_stack[gid];
+                if (page < 0 || page >= cv.P_seq || cv.owner[(size_t)b * cv.P_seq + page].x >= 0) v |= 8;
+            }
+        }
+    }
+    if (v) atomicOr(viol, v);
+}
+
 }  // namespace
+
+void launch_check(const CacheView& cv, long long tokens, unsigned* viol, unsigned* owned, cudaStream_t st) {
+    const long long work = std::max<long long>((long long)cv.B * cv.P_seq, (long long)cv.B * cv.L * cv.H);
+    dim3 grid((unsigned)((work + 255) / 256), 3);
+    check_kernel<<<grid, 256, 0, st>>>(cv, tokens, viol, owned);
+    count_launch();
+}
 
 void launch_append(const CacheView& cv, int layer0, int nlayers, int n_new, long long pos0, const float* lam,
                    const float* c, int horizon, const void* k, const void* v, int mode, cudaStream_t st) {

@@ -789,6 +789,32 @@ trimkv_status trimkv_get_select_stats(trimkv_t* h, int64_t* out_host) {
     return device_status(h);
 }
 
+trimkv_status trimkv_check_invariants(trimkv_t* h) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    CUDA_TRY(cudaDeviceSynchronize());
+    std::vector<unsigned> host((size_t)h->B + 1, 0u);
+    unsigned* dev = nullptr;
+    CUDA_TRY(cudaMalloc((void**)&dev, host.size() * sizeof(unsigned)));
+    cudaError_t e = cudaMemset(dev, 0, host.size() * sizeof(unsigned));
+    long long tokens = 0;
+    for (int l = 0; l < h->L; ++l) tokens = std::max(tokens, h->tokens[l]);
+    if (e == cudaSuccess) {
+        launch_check(h->cv, tokens, dev, dev + 1, 0);
+        e = cudaDeviceSynchronize();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(host.data(), dev, host.size() * sizeof(unsigned), cudaMemcpyDeviceToHost);
+    std::vector<int32_t> free_count(h->B, 0);
+    if (e == cudaSuccess) e = cudaMemcpy(free_count.data(), h->cv.free_count, (size_t)h->B * sizeof(int32_t), cudaMemcpyDeviceToHost);
+    cudaFree(dev);
+    if (e != cudaSuccess) return fail(TRIMKV_E_CUDA, "check_invariants: %s", cudaGetErrorString(e));
+    unsigned viol = host[0];
+    for (int b = 0; b < h->B; ++b)
+        if ((long long)host[1 + b] + free_count[b] != h->P_seq) viol |= 32;      // pages neither owned nor free, or both
+    if (viol) return fail(TRIMKV_E_STATE, "cache bookkeeping violated (rules 0x%x: 1 page id, 2 page record, 4 orphan page, 8 free "
+                          "stack, 16 position, 32 page accounting, 64 NaN retention)", viol);
+    return device_status(h);
+}
+
 trimkv_status trimkv_sync_status(trimkv_t* h) {
     if (check_handle(h)) return TRIMKV_E_ARG;
     CUDA_TRY(cudaDeviceSynchronize());

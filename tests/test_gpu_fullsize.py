@@ -147,6 +147,7 @@ def test_full_size_step_matches_oracle_on_samples(name, context, seq, skew):
             got = cache.kept(seq, l, h, len(want) + 2).numpy()
             np.testing.assert_array_equal(got, want, err_msg=f"kept set differs in pool ({seq},{l},{h})")
     assert (cache.select_stats()[:, 0] == 0).all()                     # the sampled candidate range held
+    cache.check_invariants()
     cache.close()
 
 
@@ -307,5 +308,5 @@ def test_multi_turn_flow_at_full_shape():
     assert max(int(oc.kept_positions(l, h).max()) for l in range(w.layers) for h in range(w.kv_heads)
                if len(oc.kept_positions(l, h))) == tokens
     assert (cache.select_stats()[:, 0] == 0).all()
-    cache.sync_status()
+    cache.check_invariants()
     cache.close()

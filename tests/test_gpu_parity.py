@@ -923,3 +923,73 @@ def test_append_beyond_capacity_is_refused_synchronously():
     cache.append(0, k, k, lam=lam)                        # room again
     cache.sync_status()
     cache.close()
+
+
+# ------------------------------------------------------------------------------------------- determinism / self-check
+def test_same_inputs_twice_give_bit_identical_results():
+    """No result depends on scheduling: the same sequence of chunks and whole decode steps on two caches gives bit-identical
+    attention outputs, kept sets and stored rows (atomics only order work lists and counters, never a floating-point sum)."""
+    w = workloads.WORKLOADS["llama8b_32k"].replace(layers=3, batch=3, budget_entries=3 * 8 * 150, chunk=256, context=256)
+    per_layer, w_g = workloads.gate_params(w, 4, device=DEV)
+    off = workloads.head_logit_offsets(w, 4, 3.0, device=DEV)                       # ragged pools, several items per pool
+    wn = w_g / (w_g * w_g).sum()
+    per_layer = [(W1, b1, W2, (b2 + off[l][:, None] * wn[None, :]).contiguous()) for l, (W1, b1, W2, b2) in enumerate(per_layer)]
+    bank = workloads.ProjectionBank(w, 4, device=DEV)
+    outs, states = [], []
+    for run in range(2):
+        cache = binding.TrimKV.from_workload(w)
+        for l, p in enumerate(per_layer):
+            cache.set_gate(l, *p)
+        cache.set_shared_projection(w_g, 12.0)
+        for chunk in range(2):
+            for l in range(w.layers):
+                x = workloads.hidden_states(w, 4, l, chunk * 256, 256, device=DEV)
+                _, k, v = workloads.project_qkv(w, bank, l, x)
+                cache.append(l, k, v, x=x)
+            cache.score_and_evict()
+        step_out = []
+        for i in range(6):
+            xs, ks, vs, qs = [], [], [], []
+            for l in range(w.layers):
+                x = workloads.hidden_states(w, 4, l, 512 + i, 1, device=DEV)
+                q, k, v = workloads.project_qkv(w, bank, l, x)
+                xs.append(x[:, 0]); ks.append(k[:, 0]); vs.append(v[:, 0]); qs.append(q[:, 0])
+            X, K, V, Q = [torch.stack(t).contiguous() for t in (xs, ks, vs, qs)]
+            o = torch.empty_like(Q)
+            cache.decode_step_all(K, V, Q, o, x=X)
+            step_out.append(o.clone())
+        cache.check_invariants()
+        lens = cache.lengths()
+        pools = {}
+        for b in range(w.batch):
+            for l in range(w.layers):
+                for h in range(w.kv_heads):
+                    pos, lam, c, k, v = cache.pool(b, l, h, int(lens[b, l, h]) + 1)
+                    order = torch.argsort(pos)
+                    pools[(b, l, h)] = (pos[order], lam[order], c[order], k[order].float(), v[order].float())
+        outs.append(step_out)
+        states.append((lens, pools))
+        cache.close()
+    assert int(states[0][0].max()) > 4 * max(int(states[0][0].min()), 1)           # the pools really are ragged
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    assert torch.equal(states[0][0], states[1][0])
+    for key, ta in states[0][1].items():
+        for x, y in zip(ta, states[1][1][key]):
+            assert torch.equal(x, y), key
+
+
+def test_check_invariants_reports_a_violation():
+    """The self-check is not vacuous: a consistent cache passes; entries with a NaN retention term (which an append
+    latches as an error but still stores) make it report rule 64."""
+    cache = binding.TrimKV(64, 2, 1, 128, batch=1, max_chunk=8)
+    k = torch.zeros(1, 8, 1, 128, device=DEV, dtype=torch.bfloat16)
+    lam = -torch.rand(1, 8, 1, device=DEV)
+    cache.append(0, k, k, lam=lam)
+    cache.append(1, k, k, lam=lam)
+    cache.check_invariants()
+    cache.append(0, k, k, lam=torch.full((1, 8, 1), float("nan"), device=DEV))
+    with pytest.raises(binding.TrimkvError) as e:
+        cache.check_invariants()
+    assert e.value.status == binding.E_STATE and "0x40" in str(e.value)
+    cache.close()

@@ -56,7 +56,7 @@ def test_sharded_eviction_on_the_gpu_equals_single_process_oracle(world, distrus
                     for h in range(H):
                         got = cache.kept(b, l, h, 4096).numpy()
                         np.testing.assert_array_equal(got, want[rnd][b][l0 + l][h], err_msg=f"round {rnd} pool ({b},{l0 + l},{h})")
-        cache.sync_status()
+        cache.check_invariants()
         cache.close()
 
     run_ranks_in_threads(world, rank_body)

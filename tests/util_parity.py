@@ -59,7 +59,7 @@ class Pair:
                     got = self.gpu.kept(b, l, h, int(want[l, h]) + 1).numpy()
                     np.testing.assert_array_equal(got, self.orc[b].kept_positions(l, h),
                                                   err_msg=f"kept set differs in pool ({b},{l},{h})")
-        self.gpu.sync_status()
+        self.gpu.check_invariants()               # block tables, page records, free stacks, positions: all consistent
 
     def check_attention(self, layer, q, atol):
         """q [B, Hq, d] device tensor; compares the CUDA output with the oracle's fp64 result."""
