@@ -33,7 +33,7 @@ def _stale(target: str, deps) -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu to an object and link libtrimkv.so next to this file.  Returns the library path."""
     nvcc = _nvcc()
-    headers = [os.path.join(CSRC, "trimkv_internal.cuh"), os.path.join(CSRC, "async_copy.cuh"), os.path.join(ROOT, "include", "trimkv.h"), __file__]
+    headers = [os.path.join(CSRC, "trimkv_internal.cuh"), os.path.join(CSRC, "async_copy.cuh"), os.path.join(CSRC, "mma_sync.cuh"), os.path.join(ROOT, "include", "trimkv.h"), __file__]
     objs = []
     procs = []
     for src in SOURCES:

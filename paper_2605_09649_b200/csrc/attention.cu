@@ -14,6 +14,7 @@
 #include <algorithm>
 
 #include "async_copy.cuh"
+#include "mma_sync.cuh"
 #include "trimkv_internal.cuh"
 
 namespace tkv {
@@ -35,32 +36,6 @@ constexpr int ATT_META_OFF = (ATT_RING_OFF + ATT_WARPS * ATT_RING * 4 + 127) & ~
 constexpr int ATT_META_BYTES = 2 * TILE * 4;
 constexpr int ATT_SMEM = ATT_META_OFF + ATT_WARPS * ATT_STAGES * ATT_META_BYTES;
 constexpr unsigned WAIT_LIMIT_TEST = 1u << 8;  // the limit of the testing aid under which no copy is ever issued
-
-__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
-    uint32_t d;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-    return d;
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), .y = hi
-    return *reinterpret_cast<uint32_t*>(&v);
-}
 
 // ------------------------------------------------------------------ work plan
 // Scope = pools of layers [layer0, layer0 + nlayers): scope index si = (lb * B + b) * H + h.
@@ -558,19 +533,6 @@ attn_mma_kernel(CacheView cv, int layer0, int n_scope, int tpi, int gsz, int g, 
 }
 
 // ------------------------------------------------------------------ plain kernel: any d, fp32 or bf16
-template <typename T>
-__device__ __forceinline__ float to_f32(T v);
-template <>
-__device__ __forceinline__ float to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <typename T>
-__device__ __forceinline__ T from_f32(float v);
-template <>
-__device__ __forceinline__ float from_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
-
 // One warp per (pool in scope, query head of its group).  Lanes split d; per entry one warp reduction.
 template <typename T, int MAXD>
 __global__ void __launch_bounds__(128)

@@ -8,6 +8,8 @@
 // tile.  A warp owns 16 (token, query head) columns: S^T = K Q^T and O^T += V^T P^T with mma.sync m16n8k16, online softmax
 // in registers, as in the decode kernel, with the columns now spread over tokens.  Every wait is bounded.
 // Any other shape / fp32: one warp per (pool, token, query head).
+#include "async_copy.cuh"
+#include "mma_sync.cuh"
 #include "trimkv_internal.cuh"
 
 namespace tkv {
@@ -21,59 +23,6 @@ constexpr int P_STAGE_BYTES = 2 * PT * P_ROWB;  // K tile + V tile
 constexpr int P_SMEM = P_STAGES * P_STAGE_BYTES + 128;
 constexpr int P_WARPS = 4;
 constexpr int P_COLS = 16;                      // (token, head) columns per warp
-constexpr unsigned P_WAIT_LIMIT = 1u << 24;
-
-__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void pbar_init(uint64_t* bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void pbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void pbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool pbar_wait(uint64_t* bar, uint32_t parity) {      // false: gave up
-    for (unsigned it = 0; it < P_WAIT_LIMIT; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(s_u32(bar)), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void pbulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(s_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(s_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void pldsm_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void pldsm_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ uint32_t pmovmatrix_trans(uint32_t a) {
-    uint32_t d;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-    return d;
-}
-__device__ __forceinline__ void pmma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
 // grid = (token blocks, B * H pools of `layer`); q, out: [B, n_new, Hq, 128] bf16.
 __global__ void __launch_bounds__(P_WARPS * 32, 2)
 prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const __nv_bfloat16* __restrict__ q,
@@ -99,7 +48,7 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
     for (int i = threadIdx.x * 16; i < P_STAGES * P_STAGE_BYTES; i += blockDim.x * 16)
         *reinterpret_cast<uint4*>(psm + i) = make_uint4(0u, 0u, 0u, 0u);      // masked rows must hold finite values
     if (threadIdx.x == 0) {
-        for (int s = 0; s < P_STAGES; ++s) { pbar_init(full + s, 1); pbar_init(empty + s, P_WARPS); }
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, P_WARPS); }
         *s_fail = 0;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -119,9 +68,9 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
             const char* ksrc = cv.kv + kv_row_offset(cv, b, page, 0, (tt & 1) * PT);
             const char* vsrc = cv.kv + kv_row_offset(cv, b, page, 1, (tt & 1) * PT);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            pbar_expect_tx(full + s, P_STAGE_BYTES);
-            pbulk_g2s(dst, ksrc, PT * P_ROWB, full + s);
-            pbulk_g2s(dst + PT * P_ROWB, vsrc, PT * P_ROWB, full + s);
+            mbar_expect_tx(full + s, P_STAGE_BYTES);
+            bulk_g2s(dst, ksrc, PT * P_ROWB, full + s);
+            bulk_g2s(dst + PT * P_ROWB, vsrc, PT * P_ROWB, full + s);
         }
     };
     if (warp == 0) {
@@ -173,7 +122,7 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
             bool ok = true;
             if (nx >= P_STAGES) {
                 int got = 1;
-                if (lane == 0) got = pbar_wait(empty + nx % P_STAGES, ((nx / P_STAGES) - 1) & 1) ? 1 : 0;
+                if (lane == 0) got = mbar_wait_bounded(empty + nx % P_STAGES, ((nx / P_STAGES) - 1) & 1) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, got, 0) != 0;
             }
             if (!ok) { failed = true; break; }
@@ -182,10 +131,10 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
         const int s = tt % P_STAGES;
         {
             int got = 1;
-            if (lane == 0) got = pbar_wait(full + s, (tt / P_STAGES) & 1) ? 1 : 0;
+            if (lane == 0) got = mbar_wait_bounded(full + s, (tt / P_STAGES) & 1) ? 1 : 0;
             if (__shfl_sync(0xffffffffu, got, 0) == 0) { failed = true; break; }
         }
-        const uint32_t kbase = s_u32(psm + (size_t)s * P_STAGE_BYTES);
+        const uint32_t kbase = smem_u32(psm + (size_t)s * P_STAGE_BYTES);
         const uint32_t vbase = kbase + PT * P_ROWB;
         // ---- S^T[entry][column] = K Q^T
         float sacc[2][2][4];
@@ -200,9 +149,9 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
                 const int row = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
                 const int chunk = (2 * ks + (lane >> 4)) ^ (row & 7);
                 uint32_t a[4];
-                pldsm_x4(a, kbase + row * P_ROWB + chunk * 16);
+                ldsm_x4(a, kbase + row * P_ROWB + chunk * 16);
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) pmma_bf16(sacc[mt][nt], a, bq[nt][ks][0], bq[nt][ks][1]);
+                for (int nt = 0; nt < 2; ++nt) mma_bf16(sacc[mt][nt], a, bq[nt][ks][0], bq[nt][ks][1]);
             }
         }
         // ---- causal mask by entry index, online softmax per column
@@ -238,8 +187,8 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
                 const __nv_bfloat162 phi = __floats2bfloat162_rn(exp2f(sc[2] - mn0), exp2f(sc[3] - mn1));
                 ls0 += __low2float(plo) + __low2float(phi);
                 ls1 += __high2float(plo) + __high2float(phi);
-                pb[mt][nt][0] = pmovmatrix_trans(*reinterpret_cast<const uint32_t*>(&plo));
-                pb[mt][nt][1] = pmovmatrix_trans(*reinterpret_cast<const uint32_t*>(&phi));
+                pb[mt][nt][0] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&plo));
+                pb[mt][nt][1] = movmatrix_trans(*reinterpret_cast<const uint32_t*>(&phi));
             }
             l_run[nt][0] = l_run[nt][0] * f0 + ls0;
             l_run[nt][1] = l_run[nt][1] * f1 + ls1;
@@ -256,13 +205,13 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
                 const int row = mt * 16 + (lane & 7) + (lane >> 4) * 8;
                 const int chunk = (2 * dt + ((lane >> 3) & 1)) ^ (row & 7);
                 uint32_t a[4];
-                pldsm_x4_trans(a, vbase + row * P_ROWB + chunk * 16);
+                ldsm_x4_trans(a, vbase + row * P_ROWB + chunk * 16);
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) pmma_bf16(o[nt][dt], a, pb[mt][nt][0], pb[mt][nt][1]);
+                for (int nt = 0; nt < 2; ++nt) mma_bf16(o[nt][dt], a, pb[mt][nt][0], pb[mt][nt][1]);
             }
         }
         __syncwarp();
-        if (lane == 0) pbar_arrive(empty + s);               // this warp is done with the stage
+        if (lane == 0) mbar_arrive(empty + s);               // this warp is done with the stage
     }
     if (failed) {
         if (lane == 0) { *s_fail = 1; latch_error(cv.err, TRIMKV_E_TIMEOUT); }
@@ -295,19 +244,6 @@ prefill_attn_mma_kernel(CacheView cv, int layer, int n_new, int g, int Hq, const
     }
 }
 
-template <typename T>
-__device__ __forceinline__ float p_to_f32(T v);
-template <>
-__device__ __forceinline__ float p_to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float p_to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
-template <typename T>
-__device__ __forceinline__ T p_from_f32(float v);
-template <>
-__device__ __forceinline__ float p_from_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ __nv_bfloat16 p_from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
-
 // Plain form for any head size and fp32: one warp per (sequence, chunk token, query head); lanes split d.
 template <typename T, int MAXD>
 __global__ void __launch_bounds__(128)
@@ -333,7 +269,7 @@ prefill_attn_plain_kernel(CacheView cv, int layer, int n_new, int g, int Hq, con
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
         const int dd = lane + 32 * i;
-        qr[i] = dd < d ? p_to_f32<T>(qp[dd]) * scale : 0.f;
+        qr[i] = dd < d ? to_f32<T>(qp[dd]) * scale : 0.f;
         acc[i] = 0.f;
     }
     float m = -INFINITY, l = 0.f;
@@ -348,7 +284,7 @@ prefill_attn_plain_kernel(CacheView cv, int layer, int n_new, int g, int Hq, con
         for (int i = 0; i < PER; ++i) {
             const int dd = lane + 32 * i;
             pidx[i] = phys_chunk(cv, dd / epc, off) * epc + dd % epc;
-            if (dd < d) s = fmaf(qr[i], p_to_f32<T>(kr[pidx[i]]), s);
+            if (dd < d) s = fmaf(qr[i], to_f32<T>(kr[pidx[i]]), s);
         }
 #pragma unroll
         for (int o2 = 16; o2 > 0; o2 >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o2);
@@ -358,14 +294,14 @@ prefill_attn_plain_kernel(CacheView cv, int layer, int n_new, int g, int Hq, con
 #pragma unroll
         for (int i = 0; i < PER; ++i) {
             const int dd = lane + 32 * i;
-            if (dd < d) acc[i] = acc[i] * f + p * p_to_f32<T>(vr[pidx[i]]);
+            if (dd < d) acc[i] = acc[i] * f + p * to_f32<T>(vr[pidx[i]]);
         }
         m = mn;
     }
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
         const int dd = lane + 32 * i;
-        if (dd < d) op[dd] = p_from_f32<T>(acc[i] / l);
+        if (dd < d) op[dd] = from_f32<T>(acc[i] / l);
     }
 }
 
