@@ -29,16 +29,25 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-ATTENTION_SOURCE = os.path.join(ROOT, "paper_2605_09649_b200", "csrc", "attention.cu")
+_CSRC = os.path.join(ROOT, "paper_2605_09649_b200", "csrc")
+ATTENTION_SOURCES = [os.path.join(_CSRC, f) for f in ("attention.cu", "mma_sync.cuh", "async_copy.cuh")]
 TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "attn_mma_kernel_dram_traffic.txt")
+
+
+def attention_source_digest() -> str:
+    h = hashlib.sha256()
+    for f in ATTENTION_SOURCES:
+        h.update(open(f, "rb").read())
+    return h.hexdigest()
 
 
 def recorded_traffic(workload: str):
     """DRAM bytes (read + write) of one launch of the dominant kernel, as an ncu capture recorded them, or None.
-    Each record line is `<workload> <sha256 of the kernel's source file> <bytes per launch>`; a record counts only while
-    the source file still hashes to the same value, so a changed kernel reports no stale figure."""
+    Each record line is `<workload> <sha256 of the kernel's source files> <bytes per launch>`; a record counts only while
+    the sources (the kernel's file and the two helper headers it is built from, concatenated) still hash to the same value,
+    so a changed kernel reports no stale figure."""
     try:
-        digest = hashlib.sha256(open(ATTENTION_SOURCE, "rb").read()).hexdigest()
+        digest = attention_source_digest()
         for line in open(TRAFFIC_RECORD):
             f = line.split()
             if len(f) >= 3 and not line.startswith("#") and f[0] == workload and f[1] == digest:

@@ -77,7 +77,7 @@ def test_recorded_traffic_counts_only_for_the_recorded_kernel_source(tmp_path, m
     import hashlib
     sys.path.insert(0, ROOT)
     import bench
-    digest = hashlib.sha256(open(bench.ATTENTION_SOURCE, "rb").read()).hexdigest()
+    digest = bench.attention_source_digest()
     rec = tmp_path / "traffic.txt"
     rec.write_text(f"# comment\nllama8b_32k {'0' * 64} 111\nllama8b_32k {digest} 4318434000\n")
     monkeypatch.setattr(bench, "TRAFFIC_RECORD", str(rec))
