@@ -749,6 +749,27 @@ __device__ void flat_resolve(FlatState* st, const u64* cand2, u64* keep_bits, lo
         if (tid == 0) { st->mode = MODE_EXACT_ALL; stats[2] = C; }
         return;
     }
+    if (C <= 1024) {
+        // the usual case, a few hundred keys: every thread counts the keys below its own (the keys are unique, so the
+        // thread whose count is r - 1 holds the threshold); one broadcast read per key instead of several radix sweeps
+        __shared__ u64 skeys[1024];
+        __shared__ u64 s_tau;
+        const bool have = tid < C;
+        const u64 mine = have ? __ldcg(cand2 + tid) : 0ull;
+        if (have) skeys[tid] = mine;
+        __syncthreads();
+        int below = 0;
+        for (int j = 0; j < (int)C; ++j) below += skeys[j] < mine ? 1 : 0;
+        if (have && below == (int)r - 1) s_tau = mine;
+        __syncthreads();
+        const u64 tau = s_tau;
+        if (have) {
+            const bool keep = mine > tau;
+            if (keep != (mine >= mid)) set_keep(keep_bits, mine, keep);
+        }
+        if (tid == 0) stats[2] = C;
+        return;
+    }
     u64 kr[PER];
     u64 vor = 0ull, vand = ~0ull;
 #pragma unroll
@@ -1043,12 +1064,15 @@ cudaError_t launch_select_flat(const float* scores, long long n, long long k_kee
     // 8192 samples keep the bracket under 5 % of the scores (the candidate list has room for 6 %).  Where that is still
     // millions of keys (the largest arrays, threshold away from the ends), a second, 32 times larger sample gathered by
     // many CTAs narrows it about fivefold: the list's traffic and the bits settled later shrink with it.
-    flat_bracket_kernel<8><<<1, 1024, 0, stream>>>(scores, n, k_evict, st, hist, stats, status, sigmas, distrust);
     int launches = 4;
     {
         const double q = (double)k_evict / (double)n;
         const double width = 2.0 * (sigmas * std::sqrt(q * (1.0 - q) / 8192.0) + 9.0 / 8192.0);
-        if (!distrust && n >= (1LL << 26) && width * (double)n > 2.0e6) {
+        const bool refine = !distrust && n >= (1LL << 26) && width * (double)n > 2.0e6;
+        // where the refinement follows, the first bracket only has to hold the threshold: half the samples do
+        if (refine) flat_bracket_kernel<4><<<1, 1024, 0, stream>>>(scores, n, k_evict, st, hist, stats, status, sigmas, distrust);
+        else flat_bracket_kernel<8><<<1, 1024, 0, stream>>>(scores, n, k_evict, st, hist, stats, status, sigmas, distrust);
+        if (refine) {
             flat_refine_kernel<<<REFINE_CTAS, REFINE_THREADS, 0, stream>>>(scores, n, k_evict, st, hist + (size_t)HREP * FB, stats, sigmas);
             ++launches;
         }
