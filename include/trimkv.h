@@ -198,6 +198,18 @@ TRIMKV_API trimkv_status trimkv_get_kept(trimkv_t* h, int seq, int layer, int he
 TRIMKV_API trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap, int* n, int32_t* pos_host,
                               float* lambda_host, float* c_host, void* k_host, void* v_host);
 
+/* Checkpoint / resume.  The cache IS the method's whole state (which entries survive, with their retention terms), so a
+ * snapshot is every pool read back with trimkv_get_pool plus the token count.  To resume: create a handle with the same
+ * shape, set the gate weights, call trimkv_import_pool for every non-empty pool (host arrays as trimkv_get_pool wrote
+ * them: pos int32 [n], lambda and c fp32 [n], k and v [n, d] in kv_dtype; the pool must be empty), then
+ * trimkv_import_finish(tokens) with the number of tokens the sequences had seen.  Entries keep their order, positions and
+ * fp32 retention terms, so every later eviction round and attention call gives what the original cache would have given.
+ * Both calls synchronise.  Errors: a pool that is not empty (TRIMKV_E_STATE), too many entries (TRIMKV_E_NOMEM), NaN
+ * retention terms (TRIMKV_E_NONFINITE); import_finish requires every sequence to hold the same number of entries. */
+TRIMKV_API trimkv_status trimkv_import_pool(trimkv_t* h, int seq, int layer, int head, int n, const int32_t* pos_host,
+                                 const float* lambda_host, const float* c_host, const void* k_host, const void* v_host);
+TRIMKV_API trimkv_status trimkv_import_finish(trimkv_t* h, int64_t tokens);
+
 /* Per-sequence figures of the last selection, int64 [B, 4] to host:
  * {1 if the exact redo ran (the sampled candidate range missed) else 0, candidates ranked exactly,
  *  entries evicted, keys sampled}.  Synchronises. */

@@ -26,7 +26,7 @@ EXPORTS = [
     "trimkv_prefill_attention", "trimkv_decode_step_all", "trimkv_decode_step_all_host", "trimkv_get_lengths", "trimkv_get_kept", "trimkv_get_pool", "trimkv_get_select_stats",
     "trimkv_sync_status", "trimkv_set_overlap", "trimkv_set_horizon", "trimkv_profile", "trimkv_profile_read", "trimkv_last_error", "trimkv_kernel_launches", "trimkv_select_workspace_bytes",
     "trimkv_select_topk", "trimkv_select_topk_static", "trimkv_set_test_hooks",
-    "trimkv_step_stream", "trimkv_check_invariants", "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
+    "trimkv_step_stream", "trimkv_check_invariants", "trimkv_import_pool", "trimkv_import_finish", "trimkv_shard_sample_cap", "trimkv_shard_sample", "trimkv_shard_bracket", "trimkv_shard_filter", "trimkv_shard_candidates",
     "trimkv_shard_resolve", "trimkv_shard_hist", "trimkv_shard_digit", "trimkv_shard_mark", "trimkv_shard_compact",
 ]
 
@@ -91,6 +91,10 @@ def lib() -> C.CDLL:
     L.trimkv_step_stream.argtypes = [vp]
     L.trimkv_check_invariants.argtypes = [vp]
     L.trimkv_check_invariants.restype = i32
+    L.trimkv_import_pool.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.trimkv_import_pool.restype = i32
+    L.trimkv_import_finish.argtypes = [vp, i64]
+    L.trimkv_import_finish.restype = i32
     L.trimkv_step_stream.restype = vp
     L.trimkv_shard_sample_cap.argtypes = []
     L.trimkv_shard_sample.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -325,6 +329,15 @@ class TrimKV:
                                      C.c_void_p(v.data_ptr()) if with_kv else None))
         m = n.value
         return pos[:m], lam[:m], c[:m], (k[:m] if with_kv else None), (v[:m] if with_kv else None)
+
+    def import_pool(self, seq: int, layer: int, head: int, pos, lam, c, k, v):
+        """Fills the (empty) pool from host tensors as `pool` returned them (checkpoint resume)."""
+        n = int(pos.numel())
+        hp = lambda t: C.c_void_p(t.contiguous().data_ptr()) if n else None
+        _check(lib().trimkv_import_pool(self._h, seq, layer, head, n, hp(pos), hp(lam), hp(c), hp(k), hp(v)))
+
+    def import_finish(self, tokens: int):
+        _check(lib().trimkv_import_finish(self._h, int(tokens)))
 
     def select_stats(self) -> torch.Tensor:
         out = torch.empty(self.B, 4, dtype=torch.int64)

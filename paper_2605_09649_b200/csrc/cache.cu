@@ -329,6 +329,58 @@ rehorizon_kernel(CacheView cv, int horizon) {
     cv.c[slot] = horizon_term_f32(cv.lam[slot], horizon);
 }
 
+// Fills an EMPTY pool with n entries given as dense arrays (the inverse of gather_pool_kernel): takes pages from the
+// sequence's free stack, writes rows (chunk-permuted like every stored row), metadata, page records and the length.
+// One CTA.  A pool that is not empty, or a sequence without enough free pages, latches an error and changes nothing.
+__global__ void __launch_bounds__(256)
+import_pool_kernel(CacheView cv, int b, long long pool, int n, const int32_t* __restrict__ pos, const float* __restrict__ lam,
+                   const float* __restrict__ c, const char* __restrict__ k, const char* __restrict__ v) {
+    __shared__ int s_fail;
+    int32_t* bt = cv.block_table + pool * cv.maxpp;
+    const int np = (n + PAGE - 1) / PAGE;
+    if (threadIdx.x == 0) {
+        int fail = 0;
+        if (cv.len[pool] != 0) fail = TRIMKV_E_STATE;
+        else if (np > cv.maxpp) fail = TRIMKV_E_NOMEM;
+        else {
+            const int prev = atomicSub(&cv.free_count[b], np);
+            if (prev < np) { atomicAdd(&cv.free_count[b], np); fail = TRIMKV_E_NOMEM; }
+            else {
+                const int32_t* stack = cv.free_stack + (size_t)b * cv.P_seq;
+                for (int j = 0; j < np; ++j) bt[j] = stack[prev - 1 - j];
+            }
+        }
+        if (fail) latch_error(cv.err, fail);
+        s_fail = fail;
+    }
+    __syncthreads();
+    if (s_fail) return;
+    const int pool_local = (int)(pool % ((long long)cv.L * cv.H));
+    const int rc = cv.row_bytes / 16;
+    const long long work = (long long)n * (2 * rc + 1);
+    for (long long w = threadIdx.x; w < work; w += blockDim.x) {
+        const int i = (int)(w / (2 * rc + 1));
+        const int r = (int)(w % (2 * rc + 1));
+        const int page = bt[i / PAGE], off = i % PAGE;
+        if (r == 2 * rc) {
+            const size_t slot = ((size_t)b * cv.P_seq + page) * PAGE + off;
+            if (lam[i] != lam[i] || c[i] != c[i]) latch_error(cv.err, TRIMKV_E_NONFINITE);
+            cv.pos[slot] = pos[i];
+            cv.lam[slot] = lam[i];
+            cv.c[slot] = c[i];
+        } else {
+            const int part = r / rc, ci = r % rc;
+            const char* src = (part ? v : k) + (size_t)i * cv.row_bytes + (size_t)ci * 16;
+            char* dst = cv.kv + kv_row_offset(cv, b, page, part, off) + (size_t)phys_chunk(cv, ci, off) * 16;
+            *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+        }
+    }
+    for (int lp = threadIdx.x; lp < np; lp += blockDim.x)
+        cv.owner[(size_t)b * cv.P_seq + bt[lp]] = make_int4(pool_local, lp, min(PAGE, n - lp * PAGE), 0);
+    __syncthreads();
+    if (threadIdx.x == 0) cv.len[pool] = n;
+}
+
 // Self-check of the cache's bookkeeping (tests run it where a memory checker would otherwise be used): every pool's
 // block table against the page records, every owned page against its pool, the free stack against the page records,
 // positions and retention terms of live entries.  viol: OR of the violated rules; owned [B]: pages with an owner.
@@ -384,6 +436,14 @@ __global__ void check_kernel(CacheView cv, long long tokens, unsigned* __restric
 }
 
 }  // namespace
+
+void launch_import_pool(const CacheView& cv, int seq, int layer, int head, int n, const int32_t* pos, const float* lam,
+                        const float* c, const void* k, const void* v, cudaStream_t st) {
+    if (n <= 0) return;
+    const long long pool = ((long long)seq * cv.L + layer) * cv.H + head;
+    import_pool_kernel<<<1, 256, 0, st>>>(cv, seq, pool, n, pos, lam, c, (const char*)k, (const char*)v);
+    count_launch();
+}
 
 void launch_check(const CacheView& cv, long long tokens, unsigned* viol, unsigned* owned, cudaStream_t st) {
     const long long work = std::max<long long>((long long)cv.B * cv.P_seq, (long long)cv.B * cv.L * cv.H);

@@ -261,6 +261,10 @@ void launch_prefill_attention(const CacheView& cv, int layer, int n_new, int Hq,
 // Rewrites c of every stored entry from its lambda for a new horizon.
 void launch_rehorizon(const CacheView& cv, int horizon, cudaStream_t st);
 
+// Fills an empty pool from dense device arrays (pos, lambda, c [n]; k, v [n, d] in the KV dtype).
+void launch_import_pool(const CacheView& cv, int seq, int layer, int head, int n, const int32_t* pos, const float* lam,
+                        const float* c, const void* k, const void* v, cudaStream_t st);
+
 // Bookkeeping self-check (see check_kernel): viol [1] and owned [B] must be zero on entry.
 void launch_check(const CacheView& cv, long long tokens, unsigned* viol, unsigned* owned, cudaStream_t st);
 

@@ -774,6 +774,62 @@ trimkv_status trimkv_get_pool(trimkv_t* h, int seq, int layer, int head, int cap
     return device_status(h);
 }
 
+trimkv_status trimkv_import_pool(trimkv_t* h, int seq, int layer, int head, int n, const int32_t* pos_host,
+                                 const float* lambda_host, const float* c_host, const void* k_host, const void* v_host) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (seq < 0 || seq >= h->B || layer < 0 || layer >= h->L || head < 0 || head >= h->H || n < 0)
+        return fail(TRIMKV_E_ARG, "pool index out of range or negative n");
+    if (n == 0) return TRIMKV_OK;
+    if (!pos_host || !lambda_host || !c_host || !k_host || !v_host) return fail(TRIMKV_E_ARG, "NULL array");
+    if ((long long)n > h->n_max) return fail(TRIMKV_E_NOMEM, "%d entries exceed the cache's capacity of %lld per sequence", n, h->n_max);
+    for (int i = 0; i < n; ++i)
+        if (pos_host[i] < 1 || pos_host[i] > h->max_pos) return fail(TRIMKV_E_ARG, "position %d out of range", pos_host[i]);
+    CUDA_TRY(cudaDeviceSynchronize());
+    const size_t rb = (size_t)h->d * h->elt;
+    const size_t meta = ((size_t)n * 4 + 255) / 256 * 256, kvb = ((size_t)n * rb + 255) / 256 * 256;
+    const size_t need = 3 * meta + 2 * kvb;
+    if (need > h->pool_stage_bytes) {
+        if (h->pool_stage) cudaFree(h->pool_stage);
+        h->pool_stage = nullptr;
+        h->pool_stage_bytes = 0;
+        const size_t want = std::max(need, (size_t)1 << 20);
+        CUDA_TRY(cudaMalloc((void**)&h->pool_stage, want));
+        h->pool_stage_bytes = want;
+    }
+    char* tmp = h->pool_stage;
+    CUDA_TRY(cudaMemcpy(tmp, pos_host, (size_t)n * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(tmp + meta, lambda_host, (size_t)n * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(tmp + 2 * meta, c_host, (size_t)n * 4, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(tmp + 3 * meta, k_host, (size_t)n * rb, cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(tmp + 3 * meta + kvb, v_host, (size_t)n * rb, cudaMemcpyHostToDevice));
+    launch_import_pool(h->cv, seq, layer, head, n, (const int32_t*)tmp, (const float*)(tmp + meta), (const float*)(tmp + 2 * meta),
+                       tmp + 3 * meta, tmp + 3 * meta + kvb, 0);
+    CUDA_TRY(cudaDeviceSynchronize());
+    return device_status(h);
+}
+
+trimkv_status trimkv_import_finish(trimkv_t* h, int64_t tokens) {
+    if (check_handle(h)) return TRIMKV_E_ARG;
+    if (tokens < 0 || tokens > h->max_pos) return fail(TRIMKV_E_ARG, "tokens out of range");
+    CUDA_TRY(cudaDeviceSynchronize());
+    const size_t LH = (size_t)h->L * h->H;
+    std::vector<int32_t> len((size_t)h->B * LH);
+    CUDA_TRY(cudaMemcpy(len.data(), h->cv.len, len.size() * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    long long first = -1, worst = 0;
+    for (int b = 0; b < h->B; ++b) {
+        long long e = 0;
+        for (size_t p = 0; p < LH; ++p) e += len[(size_t)b * LH + p];
+        if (first < 0) first = e;
+        if (!h->shard && e != first)
+            return fail(TRIMKV_E_STATE, "sequence %d holds %lld entries, sequence 0 holds %lld: all sequences advance in lock step", b, e, first);
+        worst = std::max(worst, e);
+    }
+    if (worst > h->n_max) return fail(TRIMKV_E_NOMEM, "imported entries exceed the cache's capacity");
+    h->entries = worst;
+    std::fill(h->tokens.begin(), h->tokens.end(), (long long)tokens);
+    return device_status(h);
+}
+
 trimkv_status trimkv_get_kept(trimkv_t* h, int seq, int layer, int head, int32_t* pos_out_host, int cap, int* n) {
     if (!pos_out_host) return fail(TRIMKV_E_ARG, "NULL output");
     trimkv_status s = trimkv_get_pool(h, seq, layer, head, cap, n, pos_out_host, nullptr, nullptr, nullptr, nullptr);

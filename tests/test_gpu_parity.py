@@ -993,3 +993,71 @@ def test_check_invariants_reports_a_violation():
         cache.check_invariants()
     assert e.value.status == binding.E_STATE and "0x40" in str(e.value)
     cache.close()
+
+
+def test_checkpoint_resume_continues_bit_for_bit():
+    """Checkpoint / resume: a cache read back pool by pool (trimkv_get_pool) and rebuilt in a new handle
+    (trimkv_import_pool, trimkv_import_finish) continues exactly as the original: the same decode steps give bit-identical
+    attention outputs, pool lengths and kept sets, and both agree with the oracle that followed the original from the start."""
+    w = BF16_SMALL.replace(budget_entries=500, batch=2)
+    pair = Pair(w)
+    r = np.random.default_rng(61)
+    g = torch.Generator(device=DEV); g.manual_seed(61)
+    dt = torch.bfloat16
+    for n in (160, 90, 1, 1):
+        for l in range(w.layers):
+            k = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+            v = torch.randn(w.batch, n, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+            lam = random_lambda((w.batch, n, w.kv_heads), int(r.integers(1 << 30)), scale=0.05)
+            pair.append(l, k, v, lam, oracle_retention(lam, w.horizon))
+        pair.evict()
+    pair.check_sets()
+    tokens = 160 + 90 + 2
+    # ---- snapshot and rebuild
+    lens = pair.gpu.lengths()
+    clone = binding.TrimKV.from_workload(w)
+    for b in range(w.batch):
+        for l in range(w.layers):
+            for h in range(w.kv_heads):
+                pos, lam, c, k, v = pair.gpu.pool(b, l, h, int(lens[b, l, h]) + 1)
+                clone.import_pool(b, l, h, pos, lam, c, k, v)
+    clone.import_finish(tokens)
+    clone.check_invariants()
+    assert torch.equal(clone.lengths(), lens)
+    with pytest.raises(binding.TrimkvError) as e:                                   # a pool that is not empty is refused
+        clone.import_pool(0, 0, 0, *pair.gpu.pool(0, 0, 0, int(lens[0, 0, 0]) + 1))
+    assert e.value.status == binding.E_STATE
+    clone.reset()
+    for b in range(w.batch):                                                        # (the latch is cleared by reset: rebuild)
+        for l in range(w.layers):
+            for h in range(w.kv_heads):
+                clone.import_pool(b, l, h, *pair.gpu.pool(b, l, h, int(lens[b, l, h]) + 1))
+    clone.import_finish(tokens)
+    # ---- both continue with the same whole decode steps
+    for step in range(4):
+        K = torch.randn(w.layers, w.batch, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+        V = torch.randn(w.layers, w.batch, w.kv_heads, w.head_dim, generator=g, device=DEV).to(dt)
+        Q = torch.randn(w.layers, w.batch, w.q_heads, w.head_dim, generator=g, device=DEV).to(dt)
+        lam = random_lambda((w.layers, w.batch, w.kv_heads), int(r.integers(1 << 30)), scale=0.05)
+        lam_t = torch.from_numpy(lam).to(DEV)
+        o1, o2 = torch.empty_like(Q), torch.empty_like(Q)
+        pair.gpu.decode_step_all(K, V, Q, o1, lam=lam_t)
+        clone.decode_step_all(K, V, Q, o2, lam=lam_t)
+        assert torch.equal(o1, o2)
+        assert torch.equal(pair.gpu.lengths(), clone.lengths())
+        # the oracle follows too (horizon 2: c = ln(1 + e^lambda), which the device's fp32 routine and the oracle's fp64
+        # evaluation round to the same fp32 value for these lambdas, or the final kept sets below would differ)
+        for l in range(w.layers):
+            for b in pair.seqs:
+                pair.orc[b].append(l, to_np(K[l, b])[None], to_np(V[l, b])[None], lam=lam[l, b][None])
+        for b in pair.seqs:
+            pair.orc[b].score_and_evict()
+    for b in range(w.batch):
+        for l in range(w.layers):
+            for h in range(w.kv_heads):
+                got = clone.kept(b, l, h, 4096)
+                assert torch.equal(got, pair.gpu.kept(b, l, h, 4096))
+                np.testing.assert_array_equal(got.numpy(), pair.orc[b].kept_positions(l, h))
+    clone.check_invariants()
+    clone.close()
+    pair.close()
