@@ -419,14 +419,26 @@ __device__ void flat_pick_bin(FlatState* st, const uint32_t* hist, long long k_e
     static_assert(MAIN_THREADS >= PICK_THREADS, "the scan needs 512 threads");
     unsigned v[PERT];
     unsigned long long local = 0;
+    {
+        // every load is issued before the first sum: one round trip to L2, not one per copy and bin
+        uint4 part[HREP][PERT / 4];
+        const int t = tid < PICK_THREADS ? tid : 0;
 #pragma unroll
-    for (int i = 0; i < PERT; ++i) {
-        v[i] = 0u;
-        if (tid < PICK_THREADS) {
+        for (int r = 0; r < HREP; ++r)
 #pragma unroll
-            for (int r = 0; r < HREP; ++r) v[i] += __ldcg(hist + r * FB + tid * PERT + i);
+            for (int q = 0; q < PERT / 4; ++q) part[r][q] = __ldcg(reinterpret_cast<const uint4*>(hist + r * FB + t * PERT) + q);
+#pragma unroll
+        for (int q = 0; q < PERT / 4; ++q) {
+            uint4 a = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int r = 0; r < HREP; ++r) { a.x += part[r][q].x; a.y += part[r][q].y; a.z += part[r][q].z; a.w += part[r][q].w; }
+            v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
         }
-        local += v[i];
+#pragma unroll
+        for (int i = 0; i < PERT; ++i) {
+            if (tid >= PICK_THREADS) v[i] = 0u;
+            local += v[i];
+        }
     }
     unsigned long long incl = local;
 #pragma unroll

@@ -213,7 +213,7 @@ void launch_compact(const CacheView& cv, int32_t* hole, int32_t* mover, int32_t*
 // Standalone selection over a flat score array (select_flat.cu).  Workspace layout: 1 KB of state and counters, the
 // candidate histogram (in several copies; the exact fallback's histograms reuse the space), the keys ranked exactly,
 // then the candidate list.
-constexpr int FLAT_HIST_BINS = 4096, FLAT_HIST_REPLICAS = 8, FLAT_X_BINS = 2048, FLAT_X_PASSES = 6, FLAT_CAND2_CAP = 16384;
+constexpr int FLAT_HIST_BINS = 4096, FLAT_HIST_REPLICAS = 3, FLAT_X_BINS = 2048, FLAT_X_PASSES = 6, FLAT_CAND2_CAP = 16384;
 constexpr size_t FLAT_FIXED_BYTES = 1024 + (size_t)FLAT_HIST_REPLICAS * FLAT_HIST_BINS * 4 + (size_t)FLAT_CAND2_CAP * 8;
 constexpr long long flat_select_cand_cap(long long n) { return n / 16 + 16384; }   // keys inside the sampled bracket, with margin
 constexpr size_t flat_select_workspace_bytes(long long n) {
