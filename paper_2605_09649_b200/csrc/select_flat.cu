@@ -761,17 +761,21 @@ __device__ void flat_resolve(FlatState* st, const u64* cand2, u64* keep_bits, lo
         if (tid == 0) { st->mode = MODE_EXACT_ALL; stats[2] = C; }
         return;
     }
-    if (C <= 1024) {
-        // the usual case, a few hundred keys: every thread counts the keys below its own (the keys are unique, so the
-        // thread whose count is r - 1 holds the threshold); one broadcast read per key instead of several radix sweeps
-        __shared__ u64 skeys[1024];
+    if (C <= 512) {
+        // the usual case, a few hundred keys: every thread that holds a key counts the keys below its own (the keys are
+        // unique, so the thread whose count is r - 1 holds the threshold): C broadcast reads per key holder, cheaper than
+        // several radix sweeps of the whole CTA up to about this size
+        __shared__ u64 skeys[512];
         __shared__ u64 s_tau;
         const bool have = tid < C;
         const u64 mine = have ? __ldcg(cand2 + tid) : 0ull;
         if (have) skeys[tid] = mine;
         __syncthreads();
         int below = 0;
-        for (int j = 0; j < (int)C; ++j) below += skeys[j] < mine ? 1 : 0;
+        if (have) {                                            // whole warps beyond the list skip the loop
+#pragma unroll 8
+            for (int j = 0; j < (int)C; ++j) below += skeys[j] < mine ? 1 : 0;
+        }
         if (have && below == (int)r - 1) s_tau = mine;
         __syncthreads();
         const u64 tau = s_tau;
