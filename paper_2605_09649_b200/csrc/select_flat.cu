@@ -3,7 +3,8 @@
 // integer order is the eviction order, so the result equals a full sort and no float is compared after key construction.
 //
 // One pass over the scores:
-//   1. flat_bracket_kernel (one CTA): ranks a stratified sample of the scores (one hashed position per stratum) and
+//   0. flat_gather_kernel: a stratified sample of the scores (one hashed position per stratum), as keys.
+//   1. flat_bracket_kernel (one CTA): ranks the sample and
 //      brackets the k-th smallest key between two sample keys, several standard deviations of the sample rank apart;
 //      the bracket's midpoint (`mid`) serves as a first estimate of the threshold.  (1b, largest arrays only:
 //      flat_refine_kernel narrows the bracket with a 32 times larger sample gathered by many CTAs.)
@@ -95,15 +96,33 @@ __device__ void flat_publish(FlatState* st, u64 lo, u64 hi, u64 e_lo, u64 e_hi, 
     st->finite = (fin && isfinite(hw)) ? 1 : 0;
 }
 
+// ------------------------------------------------------------------ 0. sample gather
+// One thread per sample: a hashed position inside its stratum, the score there, its key.  Spread over many SMs because
+// the reads are scattered over the whole array (one CTA needs 8 us for 8192 of them); the same launch clears what the later
+// kernels accumulate into.  cap: the most samples (4096 or 8192); the strata are as wide as that needs.
+__global__ void __launch_bounds__(256)
+flat_gather_kernel(const float* __restrict__ s, long long n, int cap, u64* __restrict__ samples, uint32_t* __restrict__ hist,
+                   int32_t* __restrict__ status) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    for (int i = j; i < FB * (HREP + 1); i += gridDim.x * blockDim.x) hist[i] = 0u;   // + the refinement round's histogram
+    if (j == 0 && status) *status = 0;
+    const long long stride = (n + cap - 1) / cap;          // stratum width; 1 when every score is sampled
+    const int ns = (int)((n + stride - 1) / stride);
+    if (j >= ns) return;
+    const long long base = (long long)j * stride;
+    const uint32_t width = (uint32_t)min(stride, n - base);
+    const uint32_t idx = (uint32_t)base + (width > 1u ? mix32((uint32_t)j * 0x9E3779B1u + 0x7F4A7C15u) % width : 0u);
+    samples[j] = flat_key(__ldg(s + idx), idx);
+}
+
 // ------------------------------------------------------------------ 1. sample bracket
 // PER keys per thread in registers (1024 threads): 4096 or 16384 samples.  The lower and the upper end of the bracket
 // are found by ONE radix descent over the sample: while the two ranks fall into the same bin one histogram serves both;
 // after they part each key still matches at most one of the two prefixes, so a sweep costs the same.
 template <int PER>
 __global__ void __launch_bounds__(1024)
-flat_bracket_kernel(const float* __restrict__ s, long long n, long long k_evict, FlatState* __restrict__ st,
-                    uint32_t* __restrict__ hist, long long* __restrict__ stats, int32_t* __restrict__ status, float sigmas,
-                    int distrust) {
+flat_bracket_kernel(const u64* __restrict__ samples, long long n, long long k_evict, FlatState* __restrict__ st,
+                    long long* __restrict__ stats, float sigmas, int distrust) {
     constexpr int DB = 11, NBIN = 1 << DB, CAP = 1024 * PER;
     __shared__ unsigned hAB[NBIN];          // low half-word: keys under the lower end's prefix; high: the upper end's
     __shared__ unsigned wtot[32];
@@ -113,35 +132,14 @@ flat_bracket_kernel(const float* __restrict__ s, long long n, long long k_evict,
     __shared__ unsigned s_cnt[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // state of this call: everything the later kernels accumulate into starts at zero
-    for (int i = tid; i < FB * (HREP + 1); i += 1024) hist[i] = 0u;     // + the refinement round's histogram, right behind
-    if (tid == 0 && status) *status = 0;
-
     const long long stride = (n + CAP - 1) / CAP;          // stratum width; 1 when every score is sampled
     const int ns = (int)((n + stride - 1) / stride);
     u64 key[PER];
     u64 vor = 0ull, vand = ~0ull, kmin = ~0ull, kmax = 0ull;
-    // every sample is requested before the first is used: the reads are scattered over the whole array, and one after
-    // the other they would cost a memory round trip each
-    uint32_t sidx[PER];
-    float sval[PER];
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
-        const int j = tid + i * 1024;
-        sidx[i] = 0u;
-        if (j < ns) {
-            const long long base = (long long)j * stride;
-            const uint32_t width = (uint32_t)min(stride, n - base);
-            sidx[i] = (uint32_t)base + (width > 1u ? mix32((uint32_t)j * 0x9E3779B1u + 0x7F4A7C15u) % width : 0u);
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < PER; ++i) sval[i] = (tid + i * 1024 < ns) ? __ldg(s + sidx[i]) : 0.0f;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        key[i] = ~0ull;
+        key[i] = tid + i * 1024 < ns ? samples[tid + i * 1024] : ~0ull;
         if (tid + i * 1024 < ns) {
-            key[i] = flat_key(sval[i], sidx[i]);
             vor |= key[i];
             vand &= key[i];
             kmin = key[i] < kmin ? key[i] : kmin;
@@ -1086,8 +1084,12 @@ cudaError_t launch_select_flat(const float* scores, long long n, long long k_kee
         const double width = 2.0 * (sigmas * std::sqrt(q * (1.0 - q) / 8192.0) + 9.0 / 8192.0);
         const bool refine = !distrust && n >= (1LL << 26) && width * (double)n > 2.0e6;
         // where the refinement follows, the first bracket only has to hold the threshold: half the samples do
-        if (refine) flat_bracket_kernel<4><<<1, 1024, 0, stream>>>(scores, n, k_evict, st, hist, stats, status, sigmas, distrust);
-        else flat_bracket_kernel<8><<<1, 1024, 0, stream>>>(scores, n, k_evict, st, hist, stats, status, sigmas, distrust);
+        u64* samples = cand2 + FB / 2;          // behind the refinement round's histogram, which shares the space of cand2
+        const int cap = refine ? 4096 : 8192;
+        flat_gather_kernel<<<cap / 256, 256, 0, stream>>>(scores, n, cap, samples, hist, status);
+        if (refine) flat_bracket_kernel<4><<<1, 1024, 0, stream>>>(samples, n, k_evict, st, stats, sigmas, distrust);
+        else flat_bracket_kernel<8><<<1, 1024, 0, stream>>>(samples, n, k_evict, st, stats, sigmas, distrust);
+        ++launches;
         if (refine) {
             flat_refine_kernel<<<REFINE_CTAS, REFINE_THREADS, 0, stream>>>(scores, n, k_evict, st, hist + (size_t)HREP * FB, stats, sigmas);
             ++launches;
