@@ -103,6 +103,7 @@ __device__ void flat_publish(FlatState* st, u64 lo, u64 hi, u64 e_lo, u64 e_hi, 
 __global__ void __launch_bounds__(256)
 flat_gather_kernel(const float* __restrict__ s, long long n, int cap, u64* __restrict__ samples, uint32_t* __restrict__ hist,
                    int32_t* __restrict__ status) {
+    grid_dependents_may_launch();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     for (int i = j; i < FB * (HREP + 1); i += gridDim.x * blockDim.x) hist[i] = 0u;   // + the refinement round's histogram
     if (j == 0 && status) *status = 0;
@@ -131,6 +132,8 @@ flat_bracket_kernel(const u64* __restrict__ samples, long long n, long long k_ev
     __shared__ long long s_r[2];
     __shared__ unsigned s_cnt[2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    grid_dependents_may_launch();
+    grid_dependency_wait();                                // the samples come from the kernel before
 
     const long long stride = (n + CAP - 1) / CAP;          // stratum width; 1 when every score is sampled
     const int ns = (int)((n + stride - 1) / stride);
@@ -286,6 +289,8 @@ flat_refine_kernel(const float* __restrict__ s, long long n, long long k_evict, 
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr long long CAP = (long long)REFINE_CTAS * REFINE_THREADS * REFINE_PER;
+    grid_dependents_may_launch();
+    grid_dependency_wait();                                // the first bracket comes from the kernel before
     const u64 lo = st->lo, hi = st->hi, bin_base = st->bin_base;
     const int shift = st->shift;
     for (int i = tid; i < FB; i += REFINE_THREADS) sh[i] = 0u;
@@ -711,6 +716,8 @@ flat_main_kernel(const float* __restrict__ s, long long n, long long k_evict, Fl
         for (int i = 0; i < RING; ++i) mbar_init(sm.bars + i, 1);
     }
     fence_proxy_async_smem();
+    grid_dependents_may_launch();
+    grid_dependency_wait();                                // shared memory is set up; the bracket comes from the kernel before
     __syncthreads();
     if (st->finite) flat_main_body<true>(s, n, st, cand, cand_cap, keep_bits, status, sm);
     else flat_main_body<false>(s, n, st, cand, cand_cap, keep_bits, status, sm);
@@ -865,6 +872,7 @@ __global__ void __launch_bounds__(1024)
 flat_cand_kernel(FlatState* __restrict__ st, const u64* __restrict__ cand, u64* __restrict__ cand2,
                  u64* __restrict__ keep_bits, long long* __restrict__ stats) {
     __shared__ int s_last;
+    grid_dependency_wait();                                   // the list and its bin come from the kernel before
     if (st->mode != MODE_DONE) return;                        // the exact fallback over all scores takes over
     const int lane = threadIdx.x & 31;
     const long long C1 = (long long)st->cand_count;
@@ -1087,21 +1095,24 @@ cudaError_t launch_select_flat(const float* scores, long long n, long long k_kee
         u64* samples = cand2 + FB / 2;          // behind the refinement round's histogram, which shares the space of cand2
         const int cap = refine ? 4096 : 8192;
         flat_gather_kernel<<<cap / 256, 256, 0, stream>>>(scores, n, cap, samples, hist, status);
-        if (refine) flat_bracket_kernel<4><<<1, 1024, 0, stream>>>(samples, n, k_evict, st, stats, sigmas, distrust);
-        else flat_bracket_kernel<8><<<1, 1024, 0, stream>>>(samples, n, k_evict, st, stats, sigmas, distrust);
+        // every kernel after the first is a dependent launch: it is placed and set up while its predecessor finishes
+        if (refine) launch_dependent(flat_bracket_kernel<4>, dim3(1), dim3(1024), 0, stream, samples, n, k_evict, st, stats, sigmas, distrust);
+        else launch_dependent(flat_bracket_kernel<8>, dim3(1), dim3(1024), 0, stream, samples, n, k_evict, st, stats, sigmas, distrust);
         ++launches;
         if (refine) {
-            flat_refine_kernel<<<REFINE_CTAS, REFINE_THREADS, 0, stream>>>(scores, n, k_evict, st, hist + (size_t)HREP * FB, stats, sigmas);
+            launch_dependent(flat_refine_kernel, dim3(REFINE_CTAS), dim3(REFINE_THREADS), 0, stream, scores, n, k_evict, st,
+                             hist + (size_t)HREP * FB, stats, sigmas);
             ++launches;
         }
     }
     const long long nchunk = (n + 32 * FJ - 1) / (32 * FJ);
     const int grid2 = (int)std::max<long long>(1, std::min<long long>((nchunk + MAIN_WARPS - 1) / MAIN_WARPS, (long long)sms));
     if (first_use_on_device(2)) cudaFuncSetAttribute(flat_main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MAIN_SMEM_BYTES);
-    flat_main_kernel<<<grid2, MAIN_THREADS, MAIN_SMEM_BYTES, stream>>>(scores, n, k_evict, st, hist, cand, cand_cap, keep_bits, stats, status);
+    launch_dependent(flat_main_kernel, dim3(grid2), dim3(MAIN_THREADS), MAIN_SMEM_BYTES, stream, scores, n, k_evict, st, hist, cand,
+                     cand_cap, keep_bits, stats, status);
     const long long expect = n / 24 + 1024;                    // candidates the pass over the list should be sized for
     const int grid3 = (int)std::max<long long>(1, std::min<long long>((expect + 8191) / 8192, (long long)sms));
-    flat_cand_kernel<<<grid3, 1024, 0, stream>>>(st, cand, cand2, keep_bits, stats);
+    launch_dependent(flat_cand_kernel, dim3(grid3), dim3(1024), 0, stream, st, cand, cand2, keep_bits, stats);
     // exact fallback: all CTAs resident at once (cooperative launch), so that its grid barrier is safe
     static int blocks_per_sm[64] = {};
     if (dev >= 0 && dev < 64 && blocks_per_sm[dev] == 0) {

@@ -273,6 +273,33 @@ void launch_gather_pool(const CacheView& cv, int seq, int layer, int head, int32
 
 void count_launch(int n = 1);
 
+// ---- programmatic dependent launch: a chain of short kernels in one stream overlaps each kernel's launch latency and
+// prologue with the tail of the kernel before it.  A kernel launched by launch_dependent() may start while its predecessor
+// in the stream still runs; it must call grid_dependency_wait() before it touches anything a predecessor reads or writes
+// (the wait returns once every earlier grid of the stream has completed and its writes are visible).  A predecessor lets
+// the next kernel's CTAs be placed by calling grid_dependents_may_launch() in every CTA (or by exiting); that call says
+// nothing about memory.  Both are no-ops in a kernel launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t stream,
+                                    Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // TRIMKV_TEST_* switches of the handle-less calls.
 int global_test_hooks();
 
