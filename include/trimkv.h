@@ -305,9 +305,12 @@ TRIMKV_API int64_t trimkv_kernel_launches(void);
  * status_out: device int32, set to a trimkv_status by the kernels (may be NULL).
  * The scores are read once: a sampled bracket of the threshold, one pass that writes the keep bits and a short list of
  * keys near the threshold, exact ranking of that list.  If the bracket misses (about one call in 10^4) an exact
- * multi-pass fallback runs instead; the result is the same either way.  After the call, int64 workspace[64 .. 68)
+ * multi-pass fallback runs instead; the result is the same either way.  After the call, int64 workspace[64 .. 69)
  * (byte offset 512) holds counters for tests and tuning: {fallback taken: 0 none, 1 exact over the candidate list,
- * 2 exact over all scores; keys in the sampled bracket; keys ranked exactly; keys sampled}. */
+ * 2 exact over all scores; keys in the sampled bracket; keys ranked exactly; keys sampled; form of the streaming
+ * pass's per-score tests: 2 arithmetic (no warp votes: both ends of the bracket finite, and neither its half-width
+ * nor the threshold estimate under 2^-100 in magnitude), 1 one subtraction and one compare, 0 two compares (an end
+ * of the bracket is open)}. */
 TRIMKV_API size_t trimkv_select_workspace_bytes(int64_t n);
 TRIMKV_API trimkv_status trimkv_select_topk(const float* scores, int64_t n, int64_t k_keep, uint64_t* keep_bits, void* workspace,
                                  size_t workspace_bytes, int32_t* status_out, void* stream);

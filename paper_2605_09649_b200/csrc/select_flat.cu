@@ -58,7 +58,9 @@ struct FlatState {
     float lo_f, hi_f;                // x < lo_f: score word below lo's; x > hi_f: above hi's
     float mid_lt;                    // x < mid_lt  iff  score word < mid's
     float ctr, hw;                   // finite bracket: score word within [lo's, hi's] implies !(|x - ctr| > hw)
-    int finite;                      // 1 if lo_f and hi_f are finite (the one-compare test applies)
+    int finite;                      // form of the main pass's tests.  0: two compares per score with lo_f and hi_f;
+                                     // 1: both ends finite: one subtraction + one compare (ctr, hw); 2: as 1 with hw and
+                                     // |mid_lt| at least 2^-100: the arithmetic form is exact (see flat_main_body)
 };
 static_assert(sizeof(FlatState) <= 256, "FlatState must fit the reserved header");
 
@@ -92,8 +94,13 @@ __device__ void flat_publish(FlatState* st, u64 lo, u64 hi, u64 e_lo, u64 e_hi, 
         hw = (float)(h * (1.0 + 1e-6));
         hw = nextafterf(nextafterf(hw, INFINITY), INFINITY);   // rounding of x - ctr and of hw itself: stay on the safe side
     }
+    const float mid_lt = st->mid_lt;
+    const bool fin1 = fin && isfinite(hw);
+    const bool mid_ok = isfinite(mid_lt) && fabsf(mid_lt) >= 0x1p-100f;
+    int form = fin1 ? 1 : 0;
+    if (fin1 && mid_ok && hw >= 0x1p-100f) form = 2;
     st->ctr = ctr; st->hw = hw;
-    st->finite = (fin && isfinite(hw)) ? 1 : 0;
+    st->finite = form;
 }
 
 // ------------------------------------------------------------------ 0. sample gather
@@ -523,7 +530,7 @@ struct MainSmem {          // one warp's views of the CTA's dynamic shared memor
     unsigned* ecount;
 };
 
-template <bool FINITE>
+template <int FORM>
 __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long long n, FlatState* __restrict__ st,
                                                u64* __restrict__ cand, long long cand_cap, u64* __restrict__ keep_bits,
                                                int32_t* __restrict__ status, const MainSmem& sm) {
@@ -535,23 +542,30 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
     const long long nfull = n / TRIP;                            // full trips: streamed through the ring
     const long long W = (long long)gridDim.x * MAIN_WARPS;
     const long long c0 = (long long)blockIdx.x * MAIN_WARPS + warp;
-    const long long my_trips = c0 < nfull ? (nfull - c0 + W - 1) / W : 0;
+    const int my_trips = c0 < nfull ? (int)((nfull - c0 + W - 1) / W) : 0;        // at most 2^23: indices are 32 bits wide
     const bool lane0 = lane == 0;
     int nbuf = 0;                                // warp-uniform fill of the staging buffer
     unsigned ev_fast = 0;                        // lanes < 8: scores of their words with the keep bit clear
     int adj = 0;                                 // per lane: (inside scores below lo) - (inside scores with the keep bit clear)
     bool bad = false, failed = false;
 
+    constexpr bool FINITE = FORM >= 1;
     auto inside_of = [&](float xv) -> bool {
         if (FINITE) return !(fabsf(xv - ctr) > hw);                  // true for NaN as well: it is reported below
         return !(xv < lo_f) && !(xv > hi_f);
     };
-    auto issue = [&](long long t) {                                  // trip t of this warp into stage t % RING
-        if (lane0 && t < my_trips) {
-            const int stg = (int)(t % RING);
-            fence_proxy_async_smem();
-            mbar_expect_tx(sm.bars + stg, TRIP * 4);
-            bulk_g2s(sm.ring + stg * TRIP, s + (c0 + t * W) * TRIP, TRIP * 4, sm.bars + stg);
+    // lane 0 keeps the copy it issues next (RING - 1 trips ahead of the trip being read).  The stage a copy refills was
+    // read one trip earlier, and the warp barrier that ends a trip orders those reads before the copy is issued.
+    const float* src_next = s + c0 * TRIP;
+    const long long src_step = W * TRIP;
+    int issue_stg = 0, issued = 0;
+    auto issue = [&]() {
+        if (lane0 && issued < my_trips) {
+            mbar_expect_tx(sm.bars + issue_stg, TRIP * 4);
+            bulk_g2s(sm.ring + issue_stg * TRIP, src_next, TRIP * 4, sm.bars + issue_stg);
+            src_next += src_step;
+            issue_stg = issue_stg == RING - 1 ? 0 : issue_stg + 1;
+            ++issued;
         }
     };
     // After a trip's keep words are written: the scores that may be inside.  Every lane lists the positions of its own;
@@ -572,7 +586,8 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
         }
         return cnd;
     };
-    auto handle_inside = [&](unsigned m, long long base, const float* xs) {
+    // consec: bit j of m is the lane's score 16 lane + j of the trip (arithmetic form); otherwise score 32 j + lane
+    auto handle_inside = [&](unsigned m, long long base, const float* xs, bool consec) {
         const int tot_in = __reduce_add_sync(0xffffffffu, __popc(m));
         if (!tot_in) return;
         if (tot_in <= 8) {
@@ -586,7 +601,8 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
                 bool cnd = false;
                 u64 key = 0ull;
                 if (m) {
-                    const int p = 32 * (__ffs(m) - 1) + lane;
+                    const int j = __ffs(m) - 1;
+                    const int p = consec ? 16 * lane + j : 32 * j + lane;
                     m &= m - 1;
                     cnd = classify(xs ? xs[p] : __ldg(s + base + p), (uint32_t)base + (uint32_t)p, key);
                 }
@@ -604,7 +620,7 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
             while (m) {
                 const int j = __ffs(m) - 1;
                 m &= m - 1;
-                sm.elist[pos++] = (unsigned short)(32 * j + lane);
+                sm.elist[pos++] = (unsigned short)(consec ? 16 * lane + j : 32 * j + lane);
             }
         }
         __syncwarp();
@@ -639,36 +655,79 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
         }
     };
 
-    for (int t = 0; t < RING - 1; ++t) issue(t);
-    long long t = 0;
-    for (; t < my_trips; ++t) {
-        issue(t + RING - 1);                                     // its stage was read in trip t - 1 (warp barrier below)
-        const int stg = (int)(t % RING);
-        if (!mbar_wait_bounded(sm.bars + stg, (uint32_t)((t / RING) & 1))) { failed = true; break; }
+    for (int i = 0; i < RING - 1; ++i) issue();
+    long long c = c0;
+    int t = 0, stg = 0;
+    uint32_t phase = 0;
+    // arithmetic form: the four 16-byte loads of a lane, as byte offsets into a stage.  Chunk it of the lane is read as
+    // chunk it ^ r4 with r4 = (lane / 2) & 3, so that the eight lanes served together touch all banks
+    const int r4 = (lane >> 1) & 3;
+    const uint32_t off0 = (uint32_t)(lane * 64 + (r4 << 4));
+    u64* kw = keep_bits + c0 * (FJ / 2) + lane;                  // lanes 0..7: the keep word of the current trip
+    const long long kw_step = W * (FJ / 2);
+    for (; t < my_trips; ++t, c += W, kw += kw_step) {
+        issue();
+        if (!mbar_wait_bounded(sm.bars + stg, phase)) { failed = true; break; }
         const float* xs = sm.ring + stg * TRIP;
-        const long long c = c0 + t * W;
-        unsigned m = 0u;                                         // bit j: this lane's score j of the trip may be inside
-        float x[FJ];                                             // all 16 loads first: none waits behind a store
+        unsigned m = 0u;                                         // this lane's scores of the trip that may be inside
+        if (FORM == 2) {
+            // Arithmetic form: lane l takes the 16 CONSECUTIVE scores 16 l .. 16 l + 15, so its 16 keep bits are a
+            // quarter of a keep word as they stand, and no ballot is needed.  The two tests run on the FMA pipe:
+            //   evicted  <=>  x < mid_lt          <=>  saturate((mid_lt - x) * 2^126) = 1
+            //   outside  <=>  |x - ctr| > hw      <=>  saturate((|x - ctr| - hw) * 2^126) = 1
+            // (a difference of two distinct floats is never zero; with |mid_lt| and hw at least 2^-100 a positive one is
+            // at least 2^-124, so the product saturates to exactly 1; a negative one, zero or NaN gives exactly 0, and a
+            // NaN score is thereby kept and listed as possibly inside, as in the compare form.)  The bits are collected
+            // as a binary number in a float (16 bits: exact).
+            const char* xb = reinterpret_cast<const char*>(xs);
+            float4 v[4];
 #pragma unroll
-        for (int j = 0; j < FJ; ++j) x[j] = xs[32 * j + lane];
-        unsigned kb[FJ];
+            for (int it = 0; it < 4; ++it) v[it] = *reinterpret_cast<const float4*>(xb + (off0 ^ (uint32_t)(it << 4)));
+            float acc_e = 0.f, acc_o = 0.f;
 #pragma unroll
-        for (int j = 0; j < FJ; ++j) {
-            if (inside_of(x[j])) m |= 1u << j;
-            kb[j] = __ballot_sync(0xffffffffu, !(x[j] < mid_lt));
+            for (int it = 3; it >= 0; --it) {
+                const float xe[4] = {v[it].x, v[it].y, v[it].z, v[it].w};
+#pragma unroll
+                for (int e = 3; e >= 0; --e) {
+                    acc_e = fmaf(acc_e, 2.0f, __saturatef((mid_lt - xe[e]) * 0x1p126f));
+                    acc_o = fmaf(acc_o, 2.0f, __saturatef((fabsf(xe[e] - ctr) - hw) * 0x1p126f));
+                }
+            }
+            // local nibble `it` holds the scores of nibble it ^ r4: swap nibbles within bytes if r4 & 1, bytes if r4 & 2
+            // (both 16-bit masks at once, one in each half of a word)
+            unsigned eo = (unsigned)acc_e | ((unsigned)acc_o << 16);
+            if (r4 & 1) eo = ((eo & 0x0F0F0F0Fu) << 4) | ((eo >> 4) & 0x0F0F0F0Fu);
+            if (r4 & 2) eo = __byte_perm(eo, 0u, 0x2301);
+            const unsigned keep16 = ~eo & 0xFFFFu;
+            m = ~eo >> 16;
+            ev_fast += 16u - (unsigned)__popc(keep16);
+            reinterpret_cast<unsigned short*>(sm.words)[lane] = (unsigned short)keep16;
+            __syncwarp();
+            if (lane < FJ / 2) *kw = *reinterpret_cast<const u64*>(sm.words + 2 * lane);
+        } else {
+            float x[FJ];                                         // all 16 loads first: none waits behind a store
+#pragma unroll
+            for (int j = 0; j < FJ; ++j) x[j] = xs[32 * j + lane];
+            unsigned kb[FJ];
+#pragma unroll
+            for (int j = 0; j < FJ; ++j) {
+                if (inside_of(x[j])) m |= 1u << j;
+                kb[j] = __ballot_sync(0xffffffffu, !(x[j] < mid_lt));
+            }
+            if (lane0) {
+#pragma unroll
+                for (int j = 0; j < FJ; j += 4) *reinterpret_cast<uint4*>(sm.words + j) = make_uint4(kb[j], kb[j + 1], kb[j + 2], kb[j + 3]);
+            }
+            write_words(c * (FJ / 2), TRIP, true);
         }
-        if (lane0) {
-#pragma unroll
-            for (int j = 0; j < FJ; j += 4) *reinterpret_cast<uint4*>(sm.words + j) = make_uint4(kb[j], kb[j + 1], kb[j + 2], kb[j + 3]);
-        }
-        write_words(c * (FJ / 2), TRIP, true);
-        handle_inside(m, c * TRIP, xs);
+        handle_inside(m, c * TRIP, xs, FORM == 2);
         __syncwarp();                                            // every lane is done with this stage before it is refilled
+        if (stg == RING - 1) { stg = 0; phase ^= 1u; } else ++stg;
     }
     if (failed) {                                                // a wait gave up: report, and let the copies in flight land
         latch_error(status, TRIMKV_E_TIMEOUT);
-        for (long long u = t; u < my_trips && u < t + RING; ++u)             // trips issued and not yet waited for
-            mbar_wait_bounded(sm.bars + (int)(u % RING), (uint32_t)((u / RING) & 1));
+        for (int u = t; u < my_trips && u < t + RING; ++u)                  // trips issued and not yet waited for
+            mbar_wait_bounded(sm.bars + u % RING, (uint32_t)((u / RING) & 1));
     }
     // the ragged last trip (fewer than 512 scores), by the warp whose turn it would be: plain loads
     if (nfull * TRIP < n && c0 == nfull % W) {
@@ -683,7 +742,7 @@ __device__ __forceinline__ void flat_main_body(const float* __restrict__ s, long
             if (lane0) sm.words[j] = kb;
         }
         write_words(nfull * (FJ / 2), (int)rem, false);
-        handle_inside(m, base, nullptr);
+        handle_inside(m, base, nullptr, false);
     }
     if (nbuf > 0) flat_flush(sm.wb, nbuf, st, cand, cand_cap);
     if (bad) latch_error(status, TRIMKV_E_NONFINITE);
@@ -719,8 +778,11 @@ flat_main_kernel(const float* __restrict__ s, long long n, long long k_evict, Fl
     grid_dependents_may_launch();
     grid_dependency_wait();                                // shared memory is set up; the bracket comes from the kernel before
     __syncthreads();
-    if (st->finite) flat_main_body<true>(s, n, st, cand, cand_cap, keep_bits, status, sm);
-    else flat_main_body<false>(s, n, st, cand, cand_cap, keep_bits, status, sm);
+    const int form = st->finite;
+    if (blockIdx.x == 0 && threadIdx.x == 0) stats[4] = form;
+    if (form == 2) flat_main_body<2>(s, n, st, cand, cand_cap, keep_bits, status, sm);
+    else if (form == 1) flat_main_body<1>(s, n, st, cand, cand_cap, keep_bits, status, sm);
+    else flat_main_body<0>(s, n, st, cand, cand_cap, keep_bits, status, sm);
     __syncthreads();
     uint32_t* hrep = hist + (size_t)(blockIdx.x % HREP) * FB;
     for (int i = threadIdx.x; i < FB; i += MAIN_THREADS) {

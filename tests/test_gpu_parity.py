@@ -631,7 +631,7 @@ def _select_with_stats(s, k):
     bits, status = binding.select_topk(s, k, workspace=ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    stats = ws[512:512 + 32].view(torch.int64).cpu().tolist()      # {fallback taken, bracket keys, ranked keys, sampled}
+    stats = ws[512:512 + 40].view(torch.int64).cpu().tolist()      # {fallback taken, bracket keys, ranked keys, sampled, form}
     return _unpack(bits, n), stats
 
 
@@ -699,6 +699,47 @@ def test_select_topk_structured_inputs_match_full_sort(kind):
     for k in (1, n // 8, n // 2, n - 512):
         got, stats = _select_with_stats(s, k)
         np.testing.assert_array_equal(got, _oracle_keep_bits(s_np, k), err_msg=f"{kind} k={k} stats={stats}")
+
+
+@pytest.mark.parametrize("kind", ["ulps", "huge", "tiny", "near_limit", "inf_mixed"])
+def test_select_topk_streaming_forms_match_full_sort(kind):
+    """The streaming pass has three forms of its per-score tests (counter 4 of the workspace).  The arithmetic form
+    (2) replaces compares and warp votes by saturated products and claims exactness down to one ulp; it must hand over to
+    the compare forms where magnitudes under 2^-100 would break that claim.  Scores one ulp apart around the threshold,
+    magnitudes near the largest float of both signs (differences overflow), magnitudes around and far under 2^-100,
+    and infinities of both signs: the kept set is the full sort's in every case, and the expected form decided."""
+    n = (1 << 21) + 333
+    u = workloads.selection_scores(n, seed=31, device=DEV)                           # uniform in [-8, 0]
+    idx = torch.arange(n, device=DEV)
+    if kind == "ulps":
+        steps = torch.randint(-2000, 2001, (n,), device=DEV, generator=torch.Generator(device=DEV).manual_seed(5), dtype=torch.int32)
+        s = (torch.full((n,), -3.0, device=DEV).view(torch.int32) + steps).view(torch.float32)   # -3 within +-2000 ulps:
+        want_forms = {2}                                                             # neighbours one ulp apart, ~500 ties each
+    elif kind == "huge":
+        s = (u + 4.0) * 8.0e37                                                       # +-3.2e38: x - ctr may overflow
+        want_forms = {1, 2}                                                          # (the median can be exactly 0: form 1)
+    elif kind == "tiny":
+        s = (u + 4.0) * 1.0e-36                                                      # everything far under 2^-100
+        want_forms = {1}
+    elif kind == "near_limit":
+        s = (u + 4.0) * 1.0e-28                                                      # |scores| up to 4e-28; 2^-100 = 7.9e-31:
+        want_forms = {1, 2}                                                          # the median may fall under the limit
+    else:
+        s = torch.where(idx % 3 == 0, torch.full_like(u, float("inf")), u)
+        s = torch.where(idx % 3 == 1, torch.full_like(u, float("-inf")), s)
+        want_forms = {0, 1, 2}
+    s = s.contiguous()
+    s_np = s.cpu().numpy()
+    seen = set()
+    for k in (n // 8, n // 3, n // 2, n - n // 8):
+        got, stats = _select_with_stats(s, k)
+        np.testing.assert_array_equal(got, _oracle_keep_bits(s_np, k), err_msg=f"{kind} k={k} stats={stats}")
+        assert stats[4] in want_forms, (kind, k, stats)
+        seen.add(stats[4])
+    if kind in ("ulps", "huge", "near_limit", "inf_mixed"):
+        assert 2 in seen, seen
+    if kind == "inf_mixed":
+        assert 0 in seen, seen                       # a threshold among the infinities: the bracket has no finite form
 
 
 def test_select_topk_rejects_nan_and_bad_args():
