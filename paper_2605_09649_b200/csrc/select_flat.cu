@@ -147,8 +147,9 @@ flat_bracket_kernel(const u64* __restrict__ samples, long long n, long long k_ev
     u64 key[PER];
     u64 vor = 0ull, vand = ~0ull, kmin = ~0ull, kmax = 0ull;
 #pragma unroll
+    for (int i = 0; i < PER; ++i) key[i] = tid + i * 1024 < ns ? samples[tid + i * 1024] : ~0ull;   // all loads in flight at once
+#pragma unroll
     for (int i = 0; i < PER; ++i) {
-        key[i] = tid + i * 1024 < ns ? samples[tid + i * 1024] : ~0ull;
         if (tid + i * 1024 < ns) {
             vor |= key[i];
             vand &= key[i];
@@ -166,12 +167,20 @@ flat_bracket_kernel(const u64* __restrict__ samples, long long n, long long k_ev
     }
     if (lane == 0) { s_or[warp] = vor; s_and[warp] = vand; s_min[warp] = kmin; s_max[warp] = kmax; }
     __syncthreads();
-    vor = 0ull; vand = ~0ull; kmin = ~0ull; kmax = 0ull;
-    for (int w = 0; w < 32; ++w) {
-        vor |= s_or[w]; vand &= s_and[w];
-        kmin = s_min[w] < kmin ? s_min[w] : kmin;
-        kmax = s_max[w] > kmax ? s_max[w] : kmax;
+    if (warp == 0) {                                       // one warp combines the 32 partial results and publishes them
+        vor = s_or[lane]; vand = s_and[lane]; kmin = s_min[lane]; kmax = s_max[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            vor |= __shfl_xor_sync(0xffffffffu, vor, o);
+            vand &= __shfl_xor_sync(0xffffffffu, vand, o);
+            const u64 a = __shfl_xor_sync(0xffffffffu, kmin, o), b = __shfl_xor_sync(0xffffffffu, kmax, o);
+            kmin = a < kmin ? a : kmin;
+            kmax = b > kmax ? b : kmax;
+        }
+        if (lane == 0) { s_or[0] = vor; s_and[0] = vand; s_min[0] = kmin; s_max[0] = kmax; }
     }
+    __syncthreads();
+    vor = s_or[0]; vand = s_and[0]; kmin = s_min[0]; kmax = s_max[0];
     const u64 diff = vor ^ vand;
     const int top0 = diff ? 64 - __clzll((long long)diff) : 0;   // low bits in which the sample keys differ
 
