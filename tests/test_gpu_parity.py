@@ -742,6 +742,29 @@ def test_select_topk_streaming_forms_match_full_sort(kind):
         assert 0 in seen, seen                       # a threshold among the infinities: the bracket has no finite form
 
 
+def test_select_topk_calls_on_two_streams_do_not_disturb_each_other():
+    """Two selections in flight at once, each on a stream and a workspace of its own (every kernel of a call after the
+    first starts while its predecessor is still finishing, so the two calls' kernels interleave freely): both results
+    are the full sort's."""
+    sizes = [(1 << 22) + 17, (1 << 21) + 5]
+    scores = [workloads.selection_scores(n, seed=40 + i, device=DEV) for i, n in enumerate(sizes)]
+    spaces = [torch.zeros(binding.select_workspace_bytes(n), dtype=torch.uint8, device=DEV) for n in sizes]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rnd in range(6):
+        ks = [sizes[0] // (2 + rnd), sizes[1] - 100 * (rnd + 1)]
+        out = []
+        for i in range(2):
+            with torch.cuda.stream(streams[i]):
+                out.append(binding.select_topk(scores[i], ks[i], workspace=spaces[i]))
+        torch.cuda.synchronize()
+        for i in range(2):
+            bits, status = out[i]
+            assert int(status.item()) == 0
+            np.testing.assert_array_equal(_unpack(bits, sizes[i]), _oracle_keep_bits(scores[i].cpu().numpy(), ks[i]),
+                                          err_msg=f"round {rnd} stream {i}")
+
+
 def test_select_topk_rejects_nan_and_bad_args():
     s = torch.tensor([0.0, float("nan"), -1.0, -2.0] * 64, device=DEV)
     bits, status = binding.select_topk(s, 100)
