@@ -483,7 +483,10 @@ def measure_workload(args, w, K, W, rank, world, local_rank, main):
                  "gate_ms": per("gate"), "select_ms": per("select"), "compact_ms": per("compact"), "d2h_out_ms": per("d2h_out"),
                  "what": "device time of each part of trimkv_decode_step_all_host (gate, x copy and selection run beside the "
                          "attention kernel); critical path = h2d_kvq + append + attention + compact + d2h_out; the rest of "
-                         "ms_per_step is host launch and synchronisation latency"}
+                         "ms_per_step is host launch and synchronisation latency.  q and the output sit in pinned host memory "
+                         "and are read / written there by the attention kernel itself (no copy is queued: their bytes cross "
+                         "the bus inside attention_ms); K and V are copied by copy engine (h2d_kvq), or read in place by the "
+                         "append kernel when they are under 512 KB together"}
     breakdown["critical_path_ms"] = sum(breakdown[k] for k in ("h2d_kvq_ms", "append_ms", "attention_ms", "compact_ms", "d2h_out_ms"))
     breakdown["host_latency_ms"] = max(0.0, e2e_ms - breakdown["critical_path_ms"])
     breakdown["wall_ms_per_step_with_events"] = wall_prof

@@ -156,11 +156,14 @@ TRIMKV_API trimkv_status trimkv_prefill_attention(trimkv_t* h, int layer, int n_
 TRIMKV_API trimkv_status trimkv_decode_step_all(trimkv_t* h, const float* x, const float* lambda, const void* k, const void* v,
                                      const void* q, void* out, void* stream);
 
-/* The same step for callers whose per-token tensors live in HOST memory (same shapes; pinned memory makes the copies
- * asynchronous).  The library copies them to staging buffers of the handle on its internal streams, each where its consumer
- * runs (K, V, q ahead of attention; x or lambda beside it, ahead of the gate), and copies the attention output to out_host
- * at the end of the step; everything is ordered after earlier work of `stream` and complete, for `stream`, when the call's
- * work is.  The host buffers must stay untouched until then. */
+/* The same step for callers whose per-token tensors live in HOST memory (same shapes).  x (or lambda) is copied to a
+ * staging buffer of the handle beside the attention kernel, ahead of the gate.  K, V, q and the output are each touched
+ * once by one kernel.  A q_host or out_host in pinned memory the device can address (cudaHostAlloc, cudaHostRegister,
+ * torch's pin_memory) is read or written in place across the bus by the attention kernel, and no copy is queued for it;
+ * so are a pinned k_host and v_host by the append, while they are under 512 KB together (larger ones travel faster by
+ * copy engine).  Buffers in any other memory (pageable, or pinned but not 16-byte aligned) go through staging buffers:
+ * K, V, q copied ahead of the append, the output copied back at the end of the step; the results are the same either way.  Everything is ordered after earlier work of `stream` and complete, for
+ * `stream`, when the call's work is.  The host buffers must stay untouched until then. */
 TRIMKV_API trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x_host, const float* lambda_host,
                                           const void* k_host, const void* v_host, const void* q_host, void* out_host,
                                           void* stream);

@@ -574,12 +574,29 @@ trimkv_status trimkv_prefill_attention(trimkv_t* h, int layer, int n_new, const 
 
 namespace {
 
-// Host-resident arguments of trimkv_decode_step_all_host: copied to / from the handle's staging buffers on the internal
-// streams, each copy placed where its consumer runs (K, V, q ahead of attention; x or lambda ahead of the gate).
+// Host-resident arguments of trimkv_decode_step_all_host.  x (or lambda) is copied to a staging buffer of the handle on the
+// side stream, ahead of the gate.  K, V, q and the output are each touched exactly once by a kernel (K and V by the
+// append, q and the output by the attention kernel): where the caller's buffers are pinned memory that the device can
+// address (k_map .. out_map, null otherwise), those kernels can read and write them in place across the bus with no copy
+// queued (q and the output always, K and V while they are small); otherwise they go through staging buffers, K, V, q
+// ahead of the append, the output after the compaction.
 struct HostArgs {
     const void *x, *lambda, *k, *v, *q;
     void* out;
+    const void *k_map, *v_map, *q_map;
+    void* out_map;
 };
+
+// The device's address of a pinned (page-locked, mapped) host buffer; null for any other memory.
+void* device_view_of_host(const void* p) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return nullptr;
+    return aligned16(a.devicePointer) ? a.devicePointer : nullptr;
+}
 
 trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, const void* k, const void* v, const void* q,
                             void* out, void* stream, const HostArgs* host) {
@@ -623,9 +640,18 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     if (host) {
         const size_t kvb = (size_t)h->L * h->B * h->H * h->d * h->elt, qb = (size_t)h->L * h->B * h->Hq * h->d * h->elt;
         if (h->prof.on) h->prof.mark(PH_H2D, 0, fs);
-        CUDA_TRY(cudaMemcpyAsync(h->st_k, host->k, kvb, cudaMemcpyHostToDevice, fs));
-        CUDA_TRY(cudaMemcpyAsync(h->st_v, host->v, kvb, cudaMemcpyHostToDevice, fs));
-        CUDA_TRY(cudaMemcpyAsync(h->st_q, host->q, qb, cudaMemcpyHostToDevice, fs));
+        // K and V in place only while they are small: the append kernel's 16-byte reads cross the bus at about 12 GB/s
+        // (measured: 1 MB in 85 us), a copy engine moves them at 50 GB/s but costs two more calls and a hand-over to the
+        // kernel (1 MB: 34 us + 27 us).  q is read by a kernel that runs for the whole step, where the rate does not matter.
+        if (host->k_map && host->v_map && 2 * kvb < ((size_t)512 << 10)) {
+            k = host->k_map; v = host->v_map;
+        } else {
+            CUDA_TRY(cudaMemcpyAsync(h->st_k, host->k, kvb, cudaMemcpyHostToDevice, fs));
+            CUDA_TRY(cudaMemcpyAsync(h->st_v, host->v, kvb, cudaMemcpyHostToDevice, fs));
+        }
+        if (host->q_map) q = host->q_map;
+        else CUDA_TRY(cudaMemcpyAsync(h->st_q, host->q, qb, cudaMemcpyHostToDevice, fs));
+        if (host->out_map) out = host->out_map;
         if (h->prof.on) h->prof.mark(PH_H2D, 1, fs);
         if (h->prof.on) h->prof.mark(PH_H2D_SIDE, 0, sd);
         if (host->x) CUDA_TRY(cudaMemcpyAsync(h->st_x, host->x, (size_t)h->L * h->B * h->D * 4, cudaMemcpyHostToDevice, sd));
@@ -689,7 +715,8 @@ trimkv_status step_all_impl(trimkv* h, const float* x, const float* lambda, cons
     if (s == TRIMKV_OK && kev > 0) s = compact_impl(h, fs);
     if (host) {
         if (h->prof.on) h->prof.mark(PH_D2H, 0, fs);
-        CUDA_TRY(cudaMemcpyAsync(host->out, out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, cudaMemcpyDeviceToHost, fs));
+        if (!host->out_map)
+            CUDA_TRY(cudaMemcpyAsync(host->out, out, (size_t)h->L * h->B * h->Hq * h->d * h->elt, cudaMemcpyDeviceToHost, fs));
         if (h->prof.on) h->prof.mark(PH_D2H, 1, fs);
     }
     if (two) {
@@ -720,7 +747,11 @@ trimkv_status trimkv_decode_step_all_host(trimkv_t* h, const float* x_host, cons
     if (check_handle(h)) return TRIMKV_E_ARG;
     if (!k_host || !v_host || !q_host || !out_host || (!x_host && !lambda_host)) return fail(TRIMKV_E_ARG, "NULL argument");
     if (x_host && h->D <= 0) return fail(TRIMKV_E_STATE, "handle was created without a gate (hidden = 0)");
-    HostArgs ha{x_host, lambda_host, k_host, v_host, q_host, out_host};
+    HostArgs ha{x_host, lambda_host, k_host, v_host, q_host, out_host, nullptr, nullptr, nullptr, nullptr};
+    ha.k_map = device_view_of_host(k_host);
+    ha.v_map = device_view_of_host(v_host);
+    ha.q_map = device_view_of_host(q_host);
+    ha.out_map = device_view_of_host(out_host);
     return step_all_impl(h, x_host ? h->st_x : nullptr, x_host ? nullptr : h->st_x, h->st_k, h->st_v, h->st_q, h->st_out,
                          stream, &ha);
 }

@@ -529,9 +529,25 @@ def test_decode_step_all_entry_point():
         cch.close()
 
 
-def test_decode_step_all_host_buffers_entry_point():
-    """trimkv_decode_step_all_host (pinned host tensors in, host tensor out) gives what the device-pointer call gives."""
-    w = workloads.WORKLOADS["llama8b_32k"].replace(layers=2, batch=2, budget_entries=2 * 8 * 40, chunk=64, context=64)
+@pytest.mark.parametrize("memory", ["pinned", "pageable", "pinned_in_pageable_out", "pinned_offset", "pinned_large"])
+def test_decode_step_all_host_buffers_entry_point(memory):
+    """trimkv_decode_step_all_host (host tensors in, host tensor out) gives what the device-pointer call gives: with
+    pinned buffers, which the append and attention kernels read and write in place across the bus; with pageable ones,
+    which go through the handle's staging buffers; with one kind in and the other out; with pinned buffers that
+    start 32 bytes into their allocation; and with a batch large enough (K and V of a step above 512 KB) that K and V
+    travel by copy engine while q and the output stay in place."""
+    def host(t, out=False):
+        pin = memory in ("pinned", "pinned_offset", "pinned_large") or (memory == "pinned_in_pageable_out" and not out)
+        if memory == "pinned_offset":
+            pad = 32 // t.element_size()
+            big = torch.empty(t.numel() + pad, dtype=t.dtype).pin_memory()
+            view = big[pad:].view(t.shape)
+            view.copy_(t)
+            return view
+        c = t.cpu().clone()
+        return c.pin_memory() if pin else c
+    w = workloads.WORKLOADS["llama8b_32k"].replace(layers=2, batch=64 if memory == "pinned_large" else 2,
+                                                   budget_entries=2 * 8 * 40, chunk=64, context=64)
     per_layer, w_g = workloads.gate_params(w, 2, device=DEV)
     bank = workloads.ProjectionBank(w, 2, device=DEV)
     caches = [binding.TrimKV.from_workload(w) for _ in range(2)]
@@ -555,14 +571,14 @@ def test_decode_step_all_host_buffers_entry_point():
         X, K, V, Q = [torch.stack(t).contiguous() for t in (xs, ks, vs, qs)]
         out_dev = torch.empty_like(Q)
         caches[0].decode_step_all(K, V, Q, out_dev, x=X)
-        hX, hK, hV, hQ = [t.cpu().pin_memory() for t in (X, K, V, Q)]
-        out_host = torch.empty_like(hQ).pin_memory()
+        hX, hK, hV, hQ = [host(t) for t in (X, K, V, Q)]
+        out_host = host(torch.zeros_like(Q), out=True)
         caches[1].decode_step_all_host(hK, hV, hQ, out_host, x=hX)
         torch.cuda.synchronize()
         assert torch.equal(out_dev.cpu(), out_host)
         assert torch.equal(caches[0].lengths(), caches[1].lengths())
     # retention supplied instead of x
-    lam = (-torch.rand(w.layers, w.batch, w.kv_heads) * 0.01).pin_memory()
+    lam = host(-torch.rand(w.layers, w.batch, w.kv_heads) * 0.01)
     caches[0].decode_step_all(K, V, Q, out_dev, lam=lam.to(DEV))
     caches[1].decode_step_all_host(hK, hV, hQ, out_host, lam=lam)
     torch.cuda.synchronize()
