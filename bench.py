@@ -692,6 +692,136 @@ def run_select_sweep(args):
     print(json.dumps(line), flush=True)
 
 
+def run_sharded_stages(args):
+    """Layer-sharded eviction round (one sequence's layers over several GPUs, one global budget): device time of every
+    rank-local stage and the bytes each exchange moves, measured on ONE GPU with the ranks emulated as threads of this
+    process, each with a handle holding its slice of the layers and a stream of its own.  The ranks meet on the host
+    between stages (no kernel waits for another rank's kernel), and the exchanges are plain tensor stacks, so this says
+    what the stages cost and how small the exchanges are, not what a multi-GPU run takes.  One JSON line."""
+    import threading
+    import torch
+    from paper_2605_09649_b200 import binding, sharded, workloads
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the stages have no CPU fallback")
+    torch.cuda.set_device(0)
+    dev = "cuda"
+    w = workloads.WORKLOADS[args.workload]
+    world = args.emulated_ranks
+    if w.layers % world:
+        raise SystemExit("--emulated-ranks must divide the number of layers")
+    per, LH = w.layers // world, w.layers * w.kv_heads
+    rounds, warm = max(args.steps, 1), max(args.warmup, 3)
+    context = args.context if args.context is not None else (w.budget_entries // LH + 2 * w.chunk)
+    slots, barrier = [None] * world, threading.Barrier(world)
+
+    class Comm:                                           # all ranks live in this process: gather = stack
+        def __init__(self, rank):
+            self.rank, self.world, self.bytes = rank, world, {}
+
+        def all_gather(self, t, what="gather"):
+            slots[self.rank] = t
+            torch.cuda.current_stream().synchronize()
+            barrier.wait()
+            out = torch.stack(list(slots))
+            torch.cuda.current_stream().synchronize()     # the other ranks' tensors have been read before they move on
+            barrier.wait()
+            self.bytes[what] = self.bytes.get(what, 0) + t.numel() * t.element_size() * (world - 1)
+            return out
+
+        def all_reduce_sum(self, t):
+            g = self.all_gather(t.clone(), "reduce")
+            t.copy_(g.sum(0).to(t.dtype))
+            return t
+
+    class Timed(sharded.CudaStages):                      # CUDA events around every stage call, on the rank's stream
+        def __init__(self, cache):
+            super().__init__(cache)
+            self.on, self.ev = False, []
+
+    def timed(name):
+        plain = getattr(sharded.CudaStages, name)
+
+        def call(self, *a, **k):
+            if not self.on:
+                return plain(self, *a, **k)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            r = plain(self, *a, **k)
+            e1.record()
+            self.ev.append((name, e0, e1))
+            return r
+        return call
+    for name in ("sample", "bracket", "filter", "candidates", "resolve", "compact"):
+        setattr(Timed, name, timed(name))
+
+    results, errors = [None] * world, []
+
+    def rank_body(rank):
+        try:
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                cache = binding.TrimKV.from_workload(w.replace(layers=per), shard_total_layers=w.layers, shard_layer0=rank * per)
+                stages, comm = Timed(cache), Comm(rank)
+                gen = torch.Generator(device=dev)
+                gen.manual_seed(args.seed * 1000 + rank)
+                held, cands = 0, []
+
+                def one_round(n):
+                    nonlocal held
+                    kv = torch.zeros(w.batch, n, w.kv_heads, w.head_dim, device=dev, dtype=workloads.torch_dtype(w.kv_dtype))
+                    for l in range(per):
+                        lam = -torch.rand(w.batch, n, w.kv_heads, device=dev, generator=gen) * 0.05
+                        cache.append(l, kv, kv, lam=lam)
+                    n_total = held + n * LH
+                    if n_total > w.budget_entries:
+                        info = sharded.sharded_evict(stages, comm, n_total, n_total - w.budget_entries)
+                        held = w.budget_entries
+                        return info
+                    held = n_total
+                    return None
+
+                for off in range(0, context, w.chunk):
+                    one_round(w.chunk)
+                for _ in range(warm):
+                    one_round(1)
+                stages.on, comm.bytes = True, {}
+                for _ in range(rounds):
+                    info = one_round(1)
+                    cands.append(info["candidates"])
+                    assert not info["fallback"]
+                torch.cuda.synchronize()
+                per_stage = {}
+                for name, e0, e1 in stages.ev:
+                    per_stage.setdefault(name, []).append(e0.elapsed_time(e1))
+                results[rank] = ({k: sum(v) / len(v) for k, v in per_stage.items()}, dict(comm.bytes), sum(cands) / len(cands))
+                cache.check_invariants()
+                cache.close()
+        except BaseException as e:                        # noqa: BLE001
+            errors.append(e)
+            barrier.abort()
+
+    threads = [threading.Thread(target=rank_body, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    real = [e for e in errors if not isinstance(e, threading.BrokenBarrierError)]
+    if errors:
+        raise (real[0] if real else errors[0])
+    stage_ms = {k: max(r[0][k] for r in results) for k in results[0][0]}
+    line = {"metric": "layer-sharded eviction round: device ms per rank-local stage (max over emulated ranks)", "unit": "ms",
+            "value": sum(stage_ms.values()), "n_gpus": 1, "emulated_ranks": world, "steps": rounds, "warmup": warm,
+            "higher_is_better": False, "dtype": "int64", "data": "synthetic (uniform log-retention, zero K/V)",
+            "config": {"workload": w.name, "layers_per_rank": per, "budget_entries": w.budget_entries, "batch": w.batch,
+                       "round": "one decode step: 1 token appended to every layer, then the eviction round"},
+            "stage_ms": stage_ms,
+            "exchange_bytes_received_per_rank_and_round": {k: v / rounds for k, v in results[0][1].items()},
+            "candidates_per_round": results[0][2],
+            "note": "ranks emulated as threads on one GPU: their kernels share it, so a stage's time is an upper bound of what "
+                    "a rank alone would take; the exchanges are tensor stacks here (NCCL all-gather / all-reduce between GPUs)"}
+    print(json.dumps(line), flush=True)
+
+
 def spawn_ranks(args):
     """`--gpus N` outside a torchrun environment: start the N ranks here, one process per GPU (torch.distributed.run on
     this node, rendezvous on 127.0.0.1).  Returns the launcher's exit code."""
@@ -737,11 +867,16 @@ def main():
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="leave out the other named workloads and the selection sweep (they add about half a minute)")
     ap.add_argument("--select-sweep", action="store_true", help="time the standalone selection over 2^20..2^28 scores instead")
+    ap.add_argument("--sharded-stages", action="store_true",
+                    help="time the rank-local stages of the layer-sharded eviction round with ranks emulated on one GPU instead")
+    ap.add_argument("--emulated-ranks", type=int, default=2)
     ap.add_argument("--sweep-max", type=int, default=28)
     ap.add_argument("--sweep-min", type=int, default=20)
     args = ap.parse_args()
     if args.select_sweep:
         return run_select_sweep(args)
+    if args.sharded_stages:
+        return run_sharded_stages(args)
     if args.gpus < 1:
         raise SystemExit("--gpus must be at least 1")
     in_torchrun = "WORLD_SIZE" in os.environ and "RANK" in os.environ
