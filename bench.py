@@ -809,7 +809,7 @@ def run_sharded_stages(args):
     if errors:
         raise (real[0] if real else errors[0])
     stage_ms = {k: max(r[0][k] for r in results) for k in results[0][0]}
-    line = {"metric": "layer-sharded eviction round: device ms per rank-local stage (max over emulated ranks)", "unit": "ms",
+    line = {"metric": "layer-sharded eviction round: ms per rank-local stage call on the rank's stream (max over emulated ranks)", "unit": "ms",
             "value": sum(stage_ms.values()), "n_gpus": 1, "emulated_ranks": world, "steps": rounds, "warmup": warm,
             "higher_is_better": False, "dtype": "int64", "data": "synthetic (uniform log-retention, zero K/V)",
             "config": {"workload": w.name, "layers_per_rank": per, "budget_entries": w.budget_entries, "batch": w.batch,
@@ -817,8 +817,10 @@ def run_sharded_stages(args):
             "stage_ms": stage_ms,
             "exchange_bytes_received_per_rank_and_round": {k: v / rounds for k, v in results[0][1].items()},
             "candidates_per_round": results[0][2],
-            "note": "ranks emulated as threads on one GPU: their kernels share it, so a stage's time is an upper bound of what "
-                    "a rank alone would take; the exchanges are tensor stacks here (NCCL all-gather / all-reduce between GPUs)"}
+            "note": "ranks emulated as threads on one GPU: their kernels share it, and the events around a stage call also "
+                    "span the time the host needs to queue its kernels (two Python threads, one interpreter), so a stage's "
+                    "figure is an upper bound of what a rank alone would take: the kernels themselves are in the launch list "
+                    "under profiles/; the exchanges are tensor stacks here (NCCL all-gather / all-reduce between GPUs)"}
     print(json.dumps(line), flush=True)
 
 
