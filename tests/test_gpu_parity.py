@@ -529,15 +529,16 @@ def test_decode_step_all_entry_point():
         cch.close()
 
 
-@pytest.mark.parametrize("memory", ["pinned", "pageable", "pinned_in_pageable_out", "pinned_offset", "pinned_large"])
+@pytest.mark.parametrize("memory", ["pinned", "pageable", "pinned_in_pageable_out", "pinned_offset", "pinned_large", "pinned_f32"])
 def test_decode_step_all_host_buffers_entry_point(memory):
     """trimkv_decode_step_all_host (host tensors in, host tensor out) gives what the device-pointer call gives: with
     pinned buffers, which the append and attention kernels read and write in place across the bus; with pageable ones,
     which go through the handle's staging buffers; with one kind in and the other out; with pinned buffers that
     start 32 bytes into their allocation; and with a batch large enough (K and V of a step above 512 KB) that K and V
-    travel by copy engine while q and the output stay in place."""
+    travel by copy engine while q and the output stay in place; and with an fp32 cache, whose attention runs in the
+    plain one-warp-per-head kernel."""
     def host(t, out=False):
-        pin = memory in ("pinned", "pinned_offset", "pinned_large") or (memory == "pinned_in_pageable_out" and not out)
+        pin = memory in ("pinned", "pinned_offset", "pinned_large", "pinned_f32") or (memory == "pinned_in_pageable_out" and not out)
         if memory == "pinned_offset":
             pad = 32 // t.element_size()
             big = torch.empty(t.numel() + pad, dtype=t.dtype).pin_memory()
@@ -547,7 +548,8 @@ def test_decode_step_all_host_buffers_entry_point(memory):
         c = t.cpu().clone()
         return c.pin_memory() if pin else c
     w = workloads.WORKLOADS["llama8b_32k"].replace(layers=2, batch=64 if memory == "pinned_large" else 2,
-                                                   budget_entries=2 * 8 * 40, chunk=64, context=64)
+                                                   budget_entries=2 * 8 * 40, chunk=64, context=64,
+                                                   kv_dtype="f32" if memory == "pinned_f32" else "bf16")   # f32: the plain kernel
     per_layer, w_g = workloads.gate_params(w, 2, device=DEV)
     bank = workloads.ProjectionBank(w, 2, device=DEV)
     caches = [binding.TrimKV.from_workload(w) for _ in range(2)]
